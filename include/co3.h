@@ -1,0 +1,193 @@
+/*
+ * co3.h — C ABI of the CO3 uplink pipeline for NVIDIA B200 (sm_100a).
+ *
+ * CO3 ("Convert, Compress, Correct", arXiv 2204.08211) sends, per client and per round, the
+ * gradient g corrected by a decayed error memory m, converted to a low-resolution floating-point
+ * format and entropy-coded:
+ *     v = g + gamma * m            Sec. IV-A (iii), error correction with memory decay gamma
+ *     ghat = Q_fp(v)               Sec. IV-A (i), level form in Sec. V-B
+ *     b = h_Hf(ghat)               Sec. IV-A (ii), element-wise Huffman coding, one code per layer
+ *     m = v - ghat                 Algorithm 1, memory update (= gamma*m + g - ghat)
+ * and the parameter server decodes all clients and averages, Sec. II-B (iv):
+ *     avg = (1/U) * sum_u ghat^(u)
+ *
+ * Conventions for every entry point unless stated otherwise
+ *   - Pointers marked [device] are CUDA device pointers owned by the caller; pointers marked
+ *     [host] are ordinary host pointers.  The library allocates no memory and keeps no state
+ *     between calls; scratch space is the caller's `workspace` (device, 256-byte aligned, size
+ *     from co3_workspace_bytes), whose contents are undefined after a call.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Calls only enqueue
+ *     work and return; they never synchronise.
+ *   - The int return value reports what the host can see at once (null or misaligned pointers,
+ *     unsupported sizes, workspace or capacity too small for the fixed part, launch failures).
+ *     Everything that depends on device data (descriptor contents, a symbol without codeword, a
+ *     payload that does not fit, a corrupt stream) is reported in the device-side co3_result,
+ *     valid once the stream has been synchronised.  After a device-side error the outputs of
+ *     that client are undefined but nothing is written outside the buffers given.
+ *   - A gradient of one client is a flat fp32 vector of n_elem elements, cut into n_seg segments
+ *     (layers) that are contiguous and in order: segs[0].elem_off == 0,
+ *     segs[k+1].elem_off == segs[k].elem_off + segs[k].n_elem, sum of n_elem == n_elem.
+ *     Segment k uses fmts[k] and codes[k] for every client ("a different code in each layer,
+ *     the same code across users", Sec. IV-A (ii)).  Clients are batched: client u's vector
+ *     starts client_stride_elems * u elements after the base pointer.
+ *   - fp32 buffers and streams must be 16-byte aligned.
+ */
+#ifndef CO3_H_
+#define CO3_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define CO3_OK 0
+#define CO3_ERR_INVALID_ARG 1  /* bad pointer/size, or descriptor contents rejected on the device */
+#define CO3_ERR_CAPACITY 2     /* stream or workspace too small; nothing is written past the end */
+#define CO3_ERR_NO_CODEWORD 3  /* a symbol occurred whose code length is 0 */
+#define CO3_ERR_NONFINITE 4    /* NaN/Inf seen (count in n_nonfinite); the stream is still valid */
+#define CO3_ERR_CORRUPT 5      /* decoder: header/offset mismatch or a bit pattern that is no codeword */
+#define CO3_ERR_CUDA 6         /* a CUDA runtime call failed */
+
+#define CO3_MAX_CODE_LEN 16    /* longest codeword */
+#define CO3_CHUNK_SYMS 2048    /* the only chunk size supported */
+#define CO3_SUB_SYMS 128       /* symbols per sub-chunk offset */
+
+#define CO3_FMT_FLUSH_SUBNORMALS 1u
+
+/*
+ * Target format [sgn, exp, mant] of Sec. IV-A (i) / Sec. V-B, 1 + exp_bits + mant_bits <= 8,
+ * exp_bits >= 2.  Levels for the scaled input t = v * scale are c_mant * 2^c_exp with
+ * c_mant in {1 + a_1/2 + ... + a_mant/2^mant}, c_exp in {-(2^(exp-1)-2) .. 2^(exp-1)-1}; exponent
+ * code 0 holds zero and, unless CO3_FMT_FLUSH_SUBNORMALS is set, the evenly spaced values below
+ * the smallest normal level; the all-ones exponent code is never produced (inputs beyond the
+ * largest level saturate to it).  Rounding is to the nearest level, ties to the even code.
+ * `scale` is the exponent bias written as a multiplier (c_scale = 1/scale); the reconstructed
+ * value is level * inv_scale with the stored inv_scale (normally fl32(1/scale)).
+ * A symbol is sign << (exp+mant) | exponent code << mant | mantissa code; zero has sign 0.
+ */
+typedef struct {
+    uint8_t exp_bits;
+    uint8_t mant_bits;
+    uint16_t flags;
+    float scale;
+    float inv_scale;
+} co3_fmt;
+
+/* Prefix code of one layer: len[s] in 0..CO3_MAX_CODE_LEN (0 = symbol s has no codeword),
+ * bits[s] the codeword right-aligned, its most significant bit is transmitted first. */
+typedef struct {
+    uint8_t len[256];
+    uint16_t bits[256];
+} co3_code;
+
+typedef struct {
+    uint64_t elem_off;
+    uint64_t n_elem;
+} co3_seg;
+
+/* Written on the device, one per client (encode/convert) or one per call (decode). */
+typedef struct {
+    int32_t status;           /* CO3_OK or the first error seen for this client */
+    uint32_t first_bad_chunk; /* smallest chunk index that failed (CO3_ERR_CORRUPT / NO_CODEWORD) */
+    uint64_t payload_bits;    /* r: sum of the codeword lengths (Sec. II-B (iii)) */
+    uint64_t container_bytes; /* total stream size including header, tables and padding */
+    uint64_t n_saturated;     /* finite inputs beyond the largest level (Sec. V-B boundary +-B) */
+    uint64_t n_nonfinite;     /* NaN (sent as zero) and +-Inf (sent as +-B); their memory restarts at 0 */
+} co3_result;
+
+/* Text for a status code; never NULL. */
+const char* co3_status_string(int status);
+
+/*
+ * Bytes of device workspace needed by any entry point for vectors of n_elem elements in n_seg
+ * segments with n_clients clients per encode call (pass n_clients = 0 if only co3_convert,
+ * co3_decode and co3_decode_aggregate are used).  Returns CO3_ERR_INVALID_ARG for an
+ * unsupported chunk_syms or out == NULL.
+ */
+int co3_workspace_bytes(uint64_t n_elem, uint32_t n_seg, uint32_t n_clients, uint32_t chunk_syms,
+                        size_t* out /* [host] */);
+
+/* Upper bound of the size of one client's stream (every codeword CO3_MAX_CODE_LEN bits long). */
+int co3_stream_capacity_bytes(uint64_t n_elem, uint32_t n_seg, uint32_t chunk_syms,
+                              size_t* out /* [host] */);
+
+/*
+ * Correct, convert, update memory (Algorithm 1, the conversion and memory steps) for
+ * n_clients clients, without coding.
+ *   grad [device]  fp32, read only;  mem [device] fp32, updated in place: m <- v - ghat
+ *   sym_out [device, nullable]  one byte per element, same strides as grad
+ *   hist_out [device, nullable] uint64[n_seg][256]: occurrences of each symbol per segment summed
+ *                               over the clients of this call (the statistics the code is fitted
+ *                               to); overwritten, not accumulated
+ *   res [device] co3_result[n_clients]
+ */
+int co3_convert(const float* grad, float* mem, float decay,
+                const co3_fmt* fmts /* [device] n_seg */, const co3_seg* segs /* [device] n_seg */,
+                uint32_t n_seg, uint64_t n_elem, uint32_t n_clients, uint64_t client_stride_elems,
+                uint8_t* sym_out, uint64_t* hist_out, co3_result* res,
+                void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Huffman code for one layer from 256 integer weights (Sec. IV-A (ii)); host function, all
+ * pointers [host].  Every symbol fmt can produce takes part with weight max(w, 1); other symbols
+ * get length 0.  Ties: a leaf before a merged node, leaves by symbol, merged nodes by age.
+ * If the longest codeword would exceed CO3_MAX_CODE_LEN all weights are halved (not below 1) and
+ * the construction repeats.  Codewords are canonical: sorted by (length, symbol), consecutive
+ * values.  Returns CO3_ERR_INVALID_ARG for a bad fmt or a weight sum >= 2^63.
+ */
+int co3_code_build(const uint64_t* weights, const co3_fmt* fmt, co3_code* out);
+
+/*
+ * Client uplink for n_clients clients: correct + convert + encode + memory update, codes given.
+ *   streams_out [device]  client u's container starts at streams_out + u * stream_capacity
+ *                         (stream_capacity a multiple of 16); layout below
+ *   res [device] co3_result[n_clients]
+ * Container (little-endian; every section 16-byte aligned):
+ *   header 64 B: u32 magic 'CO3S', u32 version 1, u32 n_seg, u32 chunk_syms, u32 sub_syms, u32 0,
+ *                u64 n_elem, u64 n_chunks, u64 payload_words, u64 payload_bits, u64 total_bytes
+ *   n_seg x { u64 n_elem, u64 first_chunk, u64 payload_bits }
+ *   u64 word_off[n_chunks + 1]             payload word at which each chunk starts
+ *   u16 bit_off[n_chunks][16]              bit offset of each run of 128 symbols inside its chunk
+ *   u32 payload[payload_words]
+ * A chunk holds up to 2048 consecutive symbols of one segment; its codewords are concatenated in
+ * element order, bit j of the chunk is bit 31-(j%32) of its word j/32, unused bits are 0.
+ */
+int co3_encode(const float* grad, float* mem, float decay,
+               const co3_fmt* fmts, const co3_code* codes /* [device] n_seg */, const co3_seg* segs,
+               uint32_t n_seg, uint64_t n_elem, uint32_t n_clients, uint64_t client_stride_elems,
+               uint8_t* streams_out, size_t stream_capacity, uint32_t chunk_syms,
+               void* workspace, size_t workspace_bytes, co3_result* res, void* stream);
+
+/* Same container from symbols already converted (the flow in which the code is fitted to this
+ * round's histogram between conversion and coding).  sym [device]: one byte per element. */
+int co3_encode_symbols(const uint8_t* sym, const co3_code* codes, const co3_seg* segs,
+                       uint32_t n_seg, uint64_t n_elem, uint32_t n_clients, uint64_t client_stride_elems,
+                       uint8_t* streams_out, size_t stream_capacity, uint32_t chunk_syms,
+                       void* workspace, size_t workspace_bytes, co3_result* res, void* stream);
+
+/*
+ * Parameter server: decode n_clients streams and average (Sec. II-B (iv), Algorithm 1):
+ * avg_out[i] = (ghat_i^(0) + ghat_i^(1) + ...) / n_clients, fp32 additions in client order and
+ * one fp32 division.
+ *   streams [device]  array of n_clients device pointers, each to a container of at least
+ *                     stream_bytes readable bytes
+ *   res [device]      one co3_result (payload_bits and container_bytes summed over clients)
+ */
+int co3_decode_aggregate(const uint8_t* const* streams, size_t stream_bytes, uint32_t n_clients,
+                         const co3_fmt* fmts, const co3_code* codes, const co3_seg* segs,
+                         uint32_t n_seg, uint64_t n_elem, uint32_t chunk_syms, float* avg_out,
+                         void* workspace, size_t workspace_bytes, co3_result* res, void* stream);
+
+/* One stream: reconstructed values and/or symbols (either output may be NULL, not both). */
+int co3_decode(const uint8_t* stream_in, size_t stream_bytes,
+               const co3_fmt* fmts, const co3_code* codes, const co3_seg* segs,
+               uint32_t n_seg, uint64_t n_elem, uint32_t chunk_syms,
+               float* ghat_out, uint8_t* sym_out,
+               void* workspace, size_t workspace_bytes, co3_result* res, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CO3_H_ */

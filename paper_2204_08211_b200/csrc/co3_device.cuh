@@ -1,0 +1,145 @@
+// Shared device-side definitions of the CO3 kernels: workspace layout, derived per-segment
+// tables, the bit-exact converter and small block primitives.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "co3.h"
+
+namespace co3 {
+
+constexpr int kC = CO3_CHUNK_SYMS;                           // symbols per chunk
+constexpr int kS = CO3_SUB_SYMS;                             // symbols per sub-chunk offset
+constexpr int kSubs = kC / kS;                               // 16
+constexpr int kSlotWords = kC * CO3_MAX_CODE_LEN / 32;       // worst-case words of one chunk
+constexpr int kDecBits = 12;                                 // decode LUT is indexed by 12 stream bits
+constexpr int kDecLut = 1 << kDecBits;
+constexpr int kLongStride = 260;                             // u32 per segment: count + up to 256 long codewords
+constexpr uint32_t kMagic = 0x53334F43u;                     // 'C','O','3','S'
+constexpr uint32_t kHeaderBytes = 64;
+constexpr int kThreads = 256;
+
+// Call-wide state in the workspace, cleared at the start of every call.
+struct Ctrl {
+    uint32_t abort;     // set when descriptor validation failed: later kernels return at once
+    uint32_t n_chunks;  // chunks per client
+    uint32_t n_tiles;   // decode tiles per client
+    uint32_t pad;
+    uint64_t chunk_off, sub_off, payload_off;  // byte offsets of the container sections
+};
+
+// Converter constants of one segment, derived from co3_fmt by the prepare kernel.
+struct FmtDev {
+    uint32_t mant_bits;        // M
+    uint32_t mag_bits;         // E + M
+    uint32_t min_normal_bits;  // fp32 pattern of 2^emin
+    uint32_t code_bias;        // (emin + 126) << M : fp32 (exp|mant>>drop) minus this is the magnitude code
+    uint32_t max_code;         // largest magnitude code
+    uint32_t top_bits;         // fp32 pattern of the largest level
+    uint32_t flush;            // 1: no sub-normal levels
+    uint32_t half_min_bits;    // fp32 pattern of 2^(emin-1)
+    float magic;               // 2^(emin - M + 23): adding it rounds to a multiple of the sub-normal step
+    float scale, inv_scale;
+};
+
+// Workspace sections (device pointers), computed on the host from sizes only.
+struct Ws {
+    Ctrl* ctrl;
+    uint32_t* first_chunk;  // [n_seg + 1]
+    uint32_t* first_tile;   // [n_seg + 1]
+    FmtDev* fmt;            // [n_seg]
+    uint32_t* enc_lut;      // [n_seg][256]   bits << 8 | len
+    uint16_t* dec_lut;      // [n_seg][4096]  len << 8 | sym ; len 0 = no codeword, 255 = longer than 12 bits
+    uint32_t* dec_long;     // [n_seg][kLongStride]  [0] = count, then bits << 16 | len << 8 | sym
+    float* val_lut;         // [n_seg][256]   reconstructed value of each symbol
+    uint32_t* client_fail;  // [n_clients]
+    uint32_t* chunk_bits;   // [n_clients][n_chunks_max]
+    uint64_t* bit_prefix;   // [n_clients][n_chunks_max + 1]
+    uint32_t* slots;        // [n_clients][n_chunks_max][kSlotWords]
+    uint32_t n_chunks_max;
+};
+
+__host__ __device__ inline uint64_t align16(uint64_t x) { return (x + 15u) & ~(uint64_t)15u; }
+
+// First error wins, except that the soft "non-finite input" status yields to any other error.
+__device__ inline void set_status(co3_result* r, int code) {
+    const int old = atomicCAS(&r->status, CO3_OK, code);
+    if (old == CO3_ERR_NONFINITE && code != CO3_ERR_NONFINITE) atomicCAS(&r->status, CO3_ERR_NONFINITE, code);
+}
+
+// Index of the segment that owns item `x`: largest k with first[k] <= x (empty segments are skipped).
+__device__ inline uint32_t find_seg(const uint32_t* __restrict__ first, uint32_t n_seg, uint32_t x) {
+    uint32_t lo = 0, hi = n_seg;  // invariant: first[lo] <= x < first[hi]
+    while (hi - lo > 1) {
+        const uint32_t mid = (lo + hi) >> 1;
+        if (first[mid] <= x) lo = mid; else hi = mid;
+    }
+    return lo;
+}
+
+// One element of Algorithm 1's client update:
+//   v = g + gamma*m (one FMA); t = v*scale; nearest level by integer work on the fp32 pattern
+//   (ties to the even code); ghat = level*inv_scale; returns m_new = v - ghat and the symbol.
+// flags: bit 0 = finite input beyond the largest level, bit 1 = NaN/Inf input.
+__device__ __forceinline__ float convert_one(float g, float m, float decay, const FmtDev& f,
+                                             uint32_t& sym, uint32_t& flags) {
+    const float v = __fmaf_rn(decay, m, g);
+    const uint32_t vb = __float_as_uint(v) & 0x7fffffffu;
+    const float t = __fmul_rn(v, f.scale);
+    const uint32_t tb = __float_as_uint(t);
+    const uint32_t a = tb & 0x7fffffffu;
+    uint32_t code;
+    float qmag;
+    if (a >= f.min_normal_bits) {
+        const uint32_t drop = 23u - f.mant_bits;
+        const uint32_t r = a + ((1u << (drop - 1u)) - 1u) + ((a >> drop) & 1u);  // round half to even
+        code = (r >> drop) - f.code_bias;
+        flags |= (a > f.top_bits) ? 1u : 0u;  // beyond the boundary, even if it would round back onto it
+        code = min(code, f.max_code);
+        qmag = __uint_as_float((code + f.code_bias) << drop);
+    } else if (!f.flush) {
+        const float s = __fadd_rn(__uint_as_float(a), f.magic);  // rounds |t| to the sub-normal step, ties to even
+        code = __float_as_uint(s) - __float_as_uint(f.magic);
+        qmag = __fsub_rn(s, f.magic);
+    } else {
+        code = (a > f.half_min_bits) ? (1u << f.mant_bits) : 0u;  // zero or the smallest normal level; tie to zero
+        qmag = code ? __uint_as_float(f.min_normal_bits) : 0.0f;
+    }
+    uint32_t sign = (code != 0u) ? (tb >> 31) : 0u;
+    float ghat = __fmul_rn(sign ? -qmag : qmag, f.inv_scale);
+    float m_new = __fsub_rn(v, ghat);
+    if (vb >= 0x7f800000u) {  // NaN is sent as zero, +-Inf as the boundary level; their memory restarts
+        flags = (flags & ~1u) | 2u;
+        m_new = 0.0f;
+        if (vb > 0x7f800000u) { code = 0u; sign = 0u; }
+    }
+    sym = (sign << f.mag_bits) | code;
+    return m_new;
+}
+
+// Exclusive prefix sum over the 256 threads of a block; *total receives the block sum.
+// scratch: 8 words of shared memory.  Contains two __syncthreads().
+__device__ __forceinline__ uint32_t block_exclusive_scan_256(uint32_t x, uint32_t* scratch, uint32_t* total) {
+    const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+    uint32_t inc = x;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const uint32_t y = __shfl_up_sync(0xffffffffu, inc, d);
+        if (lane >= (uint32_t)d) inc += y;
+    }
+    if (lane == 31u) scratch[warp] = inc;
+    __syncthreads();
+    uint32_t base = 0, sum = 0;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) {
+        const uint32_t s = scratch[w];
+        if ((uint32_t)w < warp) base += s;
+        sum += s;
+    }
+    __syncthreads();
+    *total = sum;
+    return base + inc - x;
+}
+
+}  // namespace co3

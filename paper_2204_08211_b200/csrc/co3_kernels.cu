@@ -1,0 +1,1110 @@
+// CUDA kernels of the CO3 uplink pipeline and its parameter-server inverse (sm_100a).
+//
+//   prepare_kernel        descriptor validation + derived tables (chunk map, encode/decode LUTs)
+//   convert_kernel        v = g + gamma*m, ghat = Q_fp(v), m = v - ghat, symbols, histogram
+//   pack_kernel           (convert +) codeword lookup, block scan of lengths, bit packing of one chunk
+//   scan_kernel           chunk word offsets, header and tables of one client's container
+//   compact_kernel        chunk payloads from their worst-case slots to their final place
+//   check_streams_kernel  header / table validation before decoding
+//   decode_kernel         chunk-indexed prefix-code decoder fused with the ordered cross-client sum
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "co3.h"
+#include "co3_device.cuh"
+
+namespace co3 {
+
+// ------------------------------------------------------------------------------------------------
+// prepare: one block per segment builds that segment's tables; block 0 also lays out the chunks.
+// ------------------------------------------------------------------------------------------------
+struct PrepArgs {
+    const co3_fmt* fmts;    // nullable (encode from symbols)
+    const co3_code* codes;  // nullable (convert only)
+    const co3_seg* segs;
+    uint32_t n_seg;
+    uint64_t n_elem;
+    uint32_t tile_chunks;  // chunks per decode tile
+    co3_result* res;
+    uint32_t n_res;
+    Ws ws;
+};
+
+__device__ void fail_all(const PrepArgs& a, int code) {
+    a.ws.ctrl->abort = 1u;
+    for (uint32_t u = 0; u < a.n_res; ++u) set_status(&a.res[u], code);
+}
+
+__global__ void __launch_bounds__(kThreads) prepare_kernel(PrepArgs a) {
+    __shared__ uint32_t s_part[kThreads][2];
+    __shared__ uint32_t s_kraft;
+    __shared__ uint32_t s_nlong;
+    const uint32_t tid = threadIdx.x;
+    const uint32_t k = blockIdx.x;
+
+    if (k == 0) {
+        for (uint32_t u = tid; u < a.n_res; u += kThreads) a.res[u].first_bad_chunk = 0xffffffffu;
+        // chunk and tile layout: exclusive scans over the segments, kThreads contiguous ranges
+        const uint32_t per = (a.n_seg + kThreads - 1) / kThreads;
+        const uint32_t lo = min(tid * per, a.n_seg), hi = min(lo + per, a.n_seg);
+        uint32_t nc = 0, nt = 0;
+        bool bad = false;
+        for (uint32_t i = lo; i < hi; ++i) {
+            const uint64_t n = a.segs[i].n_elem;
+            if (n > a.n_elem) bad = true;
+            const uint32_t c = (uint32_t)((n + kC - 1) / kC);
+            nc += c;
+            nt += (c + a.tile_chunks - 1) / a.tile_chunks;
+        }
+        s_part[tid][0] = nc;
+        s_part[tid][1] = nt;
+        __syncthreads();
+        uint32_t bc = 0, bt = 0;
+        for (uint32_t i = 0; i < tid; ++i) { bc += s_part[i][0]; bt += s_part[i][1]; }
+        // segments must be contiguous, in order, and cover n_elem
+        uint64_t expect_off = (lo < a.n_seg) ? a.segs[lo].elem_off : 0;
+        for (uint32_t i = lo; i < hi; ++i) {
+            const co3_seg sg = a.segs[i];
+            if (sg.elem_off != expect_off) bad = true;
+            expect_off = sg.elem_off + sg.n_elem;
+            a.ws.first_chunk[i] = bc;
+            a.ws.first_tile[i] = bt;
+            const uint32_t c = (uint32_t)((sg.n_elem + kC - 1) / kC);
+            bc += c;
+            bt += (c + a.tile_chunks - 1) / a.tile_chunks;
+        }
+        if (lo < hi) {
+            if (lo == 0 && a.segs[0].elem_off != 0) bad = true;
+            const uint64_t next_off = (hi < a.n_seg) ? a.segs[hi].elem_off : a.n_elem;
+            if (expect_off != next_off) bad = true;
+        }
+        if (a.n_seg == 0 && tid == 0 && a.n_elem != 0) bad = true;
+        if (bc > a.ws.n_chunks_max) bad = true;
+        const bool owner = (a.n_seg == 0) ? (tid == 0) : (lo < hi && hi == a.n_seg);  // owns the end of the table
+        if (owner) {
+            a.ws.first_chunk[a.n_seg] = bc;
+            a.ws.first_tile[a.n_seg] = bt;
+            Ctrl* c = a.ws.ctrl;
+            c->n_chunks = bc;
+            c->n_tiles = bt;
+            c->chunk_off = align16(kHeaderBytes + 24ull * a.n_seg);
+            c->sub_off = align16(c->chunk_off + 8ull * (bc + 1ull));
+            c->payload_off = align16(c->sub_off + 2ull * bc * kSubs);
+        }
+        if (bad) fail_all(a, CO3_ERR_INVALID_ARG);
+    }
+    if (k >= a.n_seg) return;
+
+    // ---- format constants and value table
+    bool fmt_ok = true;
+    FmtDev fd{};
+    if (a.fmts) {
+        const co3_fmt f = a.fmts[k];
+        const uint32_t E = f.exp_bits, M = f.mant_bits;
+        fmt_ok = E >= 2 && 1 + E + M <= 8 && (f.flags & ~CO3_FMT_FLUSH_SUBNORMALS) == 0 && f.scale > 0.0f &&
+                 f.inv_scale > 0.0f && !isinf(f.scale) && !isinf(f.inv_scale);
+        const int emin = fmt_ok ? -((1 << (E - 1)) - 2) : 0;
+        if (fmt_ok) {
+            fd.mant_bits = M;
+            fd.mag_bits = E + M;
+            fd.min_normal_bits = (uint32_t)(emin + 127) << 23;
+            fd.code_bias = (uint32_t)(emin + 126) << M;
+            fd.max_code = (((1u << E) - 2u) << M) | ((1u << M) - 1u);
+            fd.top_bits = (fd.max_code + fd.code_bias) << (23u - M);
+            fd.flush = (f.flags & CO3_FMT_FLUSH_SUBNORMALS) ? 1u : 0u;
+            fd.half_min_bits = (uint32_t)(emin - 1 + 127) << 23;
+            fd.magic = __uint_as_float((uint32_t)(emin - (int)M + 23 + 127) << 23);
+            fd.scale = f.scale;
+            fd.inv_scale = f.inv_scale;
+            const float top = __fmul_rn(__uint_as_float((fd.max_code + fd.code_bias) << (23u - M)), f.inv_scale);
+            if (isinf(top)) fmt_ok = false;
+        }
+        if (fmt_ok) {
+            if (tid == 0) a.ws.fmt[k] = fd;
+            // reconstructed value of symbol `tid`
+            const uint32_t sym = tid, nb = fd.mag_bits;
+            float val = 0.0f;
+            if (sym < (2u << nb)) {
+                const uint32_t sign = sym >> nb, code = sym & ((1u << nb) - 1u);
+                const uint32_t efield = code >> M, mfield = code & ((1u << M) - 1u);
+                float q = 0.0f;
+                bool valid = efield != (1u << E) - 1u && !(sign && code == 0);
+                if (efield == 0) {
+                    if (fd.flush && mfield) valid = false;
+                    q = __fmul_rn((float)mfield, __uint_as_float((uint32_t)(emin - (int)M + 127) << 23));
+                } else {
+                    q = __uint_as_float((code + fd.code_bias) << (23u - M));
+                }
+                if (valid) val = __fmul_rn(sign ? -q : q, f.inv_scale);
+            }
+            a.ws.val_lut[k * 256 + tid] = val;
+        }
+    }
+
+    // ---- code tables
+    bool code_ok = true;
+    if (a.codes) {
+        const uint32_t len = a.codes[k].len[tid], bits = a.codes[k].bits[tid];
+        if (tid == 0) { s_kraft = 0; s_nlong = 0; }
+        __syncthreads();
+        if (len > CO3_MAX_CODE_LEN || (len && (bits >> len))) code_ok = false;
+        if (code_ok && len) atomicAdd(&s_kraft, 1u << (CO3_MAX_CODE_LEN - len));
+        a.ws.enc_lut[k * 256 + tid] = code_ok ? ((bits << 8) | len) : 0u;
+        uint16_t* lut = a.ws.dec_lut + (size_t)k * kDecLut;
+        for (uint32_t i = tid; i < (uint32_t)kDecLut; i += kThreads) lut[i] = 0;
+        __syncthreads();
+        if (s_kraft > (1u << CO3_MAX_CODE_LEN)) code_ok = false;  // over-subscribed: cannot be prefix-free
+        code_ok = __syncthreads_and(code_ok);
+        if (code_ok) {
+            // short codewords fill every table entry they prefix: one warp per symbol, lanes over the span
+            for (uint32_t sym = tid >> 5; sym < 256; sym += kThreads / 32) {
+                const uint32_t l = a.codes[k].len[sym], b = a.codes[k].bits[sym];
+                if (l == 0 || l > (uint32_t)kDecBits) continue;
+                const uint32_t span = 1u << (kDecBits - l), first = b << (kDecBits - l);
+                for (uint32_t i = tid & 31u; i < span; i += 32) lut[first + i] = (uint16_t)((l << 8) | sym);
+            }
+            if (len > (uint32_t)kDecBits) {
+                lut[bits >> (len - kDecBits)] = (uint16_t)(255u << 8);
+                const uint32_t slot = atomicAdd(&s_nlong, 1u);
+                a.ws.dec_long[k * kLongStride + 1 + slot] = (bits << 16) | (len << 8) | tid;
+            }
+            __syncthreads();
+            if (tid == 0) a.ws.dec_long[k * kLongStride] = s_nlong;
+        }
+    }
+    if ((!fmt_ok || !code_ok) && tid == 0) fail_all(a, CO3_ERR_INVALID_ARG);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Element access for one thread: 8 consecutive elements of a chunk.
+// ------------------------------------------------------------------------------------------------
+struct ChunkPos {
+    uint32_t seg;
+    uint32_t cnt;    // symbols in this chunk
+    uint64_t elem0;  // index of the chunk's first element inside the client's vector
+};
+
+__device__ __forceinline__ ChunkPos locate_chunk(const Ws& ws, const co3_seg* __restrict__ segs, uint32_t n_seg,
+                                                 uint32_t chunk) {
+    ChunkPos p;
+    p.seg = find_seg(ws.first_chunk, n_seg, chunk);
+    const co3_seg sg = segs[p.seg];
+    const uint64_t start = (uint64_t)(chunk - ws.first_chunk[p.seg]) * kC;
+    p.cnt = (uint32_t)min((uint64_t)kC, sg.n_elem - start);
+    p.elem0 = sg.elem_off + start;
+    return p;
+}
+
+__device__ __forceinline__ void load8(const float* __restrict__ p, uint32_t n_valid, float (&x)[8]) {
+    if (n_valid == 8 && (reinterpret_cast<uintptr_t>(p) & 15u) == 0) {
+        const float4 a = __ldg(reinterpret_cast<const float4*>(p));
+        const float4 b = __ldg(reinterpret_cast<const float4*>(p) + 1);
+        x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w;
+        x[4] = b.x; x[5] = b.y; x[6] = b.z; x[7] = b.w;
+    } else {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) x[j] = (uint32_t)j < n_valid ? p[j] : 0.0f;
+    }
+}
+
+__device__ __forceinline__ void store8(float* __restrict__ p, uint32_t n_valid, const float (&x)[8]) {
+    if (n_valid == 8 && (reinterpret_cast<uintptr_t>(p) & 15u) == 0) {
+        reinterpret_cast<float4*>(p)[0] = make_float4(x[0], x[1], x[2], x[3]);
+        reinterpret_cast<float4*>(p)[1] = make_float4(x[4], x[5], x[6], x[7]);
+    } else {
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+            if ((uint32_t)j < n_valid) p[j] = x[j];
+    }
+}
+
+__device__ __forceinline__ void store_sym8(uint8_t* __restrict__ p, uint32_t n_valid, const uint32_t (&s)[8]) {
+    if (n_valid == 8 && (reinterpret_cast<uintptr_t>(p) & 7u) == 0) {
+        uint2 w;
+        w.x = s[0] | (s[1] << 8) | (s[2] << 16) | (s[3] << 24);
+        w.y = s[4] | (s[5] << 8) | (s[6] << 16) | (s[7] << 24);
+        *reinterpret_cast<uint2*>(p) = w;
+    } else {
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+            if ((uint32_t)j < n_valid) p[j] = (uint8_t)s[j];
+    }
+}
+
+__device__ __forceinline__ void load_sym8(const uint8_t* __restrict__ p, uint32_t n_valid, uint32_t (&s)[8]) {
+    if (n_valid == 8 && (reinterpret_cast<uintptr_t>(p) & 7u) == 0) {
+        const uint2 w = __ldg(reinterpret_cast<const uint2*>(p));
+#pragma unroll
+        for (int j = 0; j < 4; ++j) { s[j] = (w.x >> (8 * j)) & 0xffu; s[4 + j] = (w.y >> (8 * j)) & 0xffu; }
+    } else {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) s[j] = (uint32_t)j < n_valid ? p[j] : 0u;
+    }
+}
+
+// Adds the saturated / non-finite counts of a warp to the client's result.
+__device__ __forceinline__ void add_counts(co3_result* r, uint32_t n_sat, uint32_t n_nf) {
+    if (__any_sync(0xffffffffu, (n_sat | n_nf) != 0)) {
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) {
+            n_sat += __shfl_xor_sync(0xffffffffu, n_sat, d);
+            n_nf += __shfl_xor_sync(0xffffffffu, n_nf, d);
+        }
+        if ((threadIdx.x & 31u) == 0) {
+            if (n_sat) atomicAdd(reinterpret_cast<unsigned long long*>(&r->n_saturated), (unsigned long long)n_sat);
+            if (n_nf) {
+                atomicAdd(reinterpret_cast<unsigned long long*>(&r->n_nonfinite), (unsigned long long)n_nf);
+                set_status(r, CO3_ERR_NONFINITE);
+            }
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// convert: one block per (chunk, client)
+// ------------------------------------------------------------------------------------------------
+struct ConvertArgs {
+    const float* grad;
+    float* mem;
+    float decay;
+    const co3_seg* segs;
+    uint32_t n_seg;
+    uint64_t client_stride;
+    uint8_t* sym_out;    // nullable
+    uint64_t* hist_out;  // nullable
+    co3_result* res;
+    Ws ws;
+};
+
+template <bool kSym, bool kHist>
+__global__ void __launch_bounds__(kThreads) convert_kernel(ConvertArgs a) {
+    __shared__ uint32_t s_hist[256];
+    const Ctrl* ctrl = a.ws.ctrl;
+    if (ctrl->abort) return;
+    const uint32_t chunk = blockIdx.x, u = blockIdx.y, tid = threadIdx.x;
+    if (chunk >= ctrl->n_chunks) return;
+    const ChunkPos pos = locate_chunk(a.ws, a.segs, a.n_seg, chunk);
+    const FmtDev f = a.ws.fmt[pos.seg];
+    if (kHist) {
+        s_hist[tid] = 0;
+        __syncthreads();
+    }
+    const uint32_t i0 = tid * 8;
+    const uint32_t nv = pos.cnt > i0 ? min(8u, pos.cnt - i0) : 0u;
+    uint32_t n_sat = 0, n_nf = 0;
+    if (nv) {
+        const uint64_t e = (uint64_t)u * a.client_stride + pos.elem0 + i0;
+        float g[8], m[8];
+        uint32_t s[8];
+        load8(a.grad + e, nv, g);
+        load8(a.mem + e, nv, m);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            uint32_t fl = 0;
+            m[j] = convert_one(g[j], m[j], a.decay, f, s[j], fl);
+            if ((uint32_t)j < nv) { n_sat += fl & 1u; n_nf += fl >> 1; }
+        }
+        store8(a.mem + e, nv, m);
+        if (kSym) store_sym8(a.sym_out + e, nv, s);
+        if (kHist) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+                if ((uint32_t)j < nv) atomicAdd(&s_hist[s[j]], 1u);
+        }
+    }
+    add_counts(&a.res[u], n_sat, n_nf);
+    if (kHist) {
+        __syncthreads();
+        const uint32_t c = s_hist[tid];
+        if (c) atomicAdd(reinterpret_cast<unsigned long long*>(&a.hist_out[(size_t)pos.seg * 256 + tid]), (unsigned long long)c);
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// pack: one block per (chunk, client).  Thread t owns symbols 8t .. 8t+7 of the chunk.
+// ------------------------------------------------------------------------------------------------
+struct PackArgs {
+    const float* grad;   // fused path
+    float* mem;
+    float decay;
+    const uint8_t* sym;  // symbol path
+    const co3_seg* segs;
+    uint32_t n_seg;
+    uint64_t client_stride;
+    uint8_t* streams;
+    size_t stream_capacity;
+    co3_result* res;
+    Ws ws;
+};
+
+// ORs the low n bits of v (n <= 64) into the bit buffer at bit offset `off` (most significant bit first).
+__device__ __forceinline__ void put_bits(uint32_t* buf, uint32_t off, uint64_t v, uint32_t n) {
+    if (n == 0) return;
+    const uint64_t left = v << (64u - n);  // left-aligned
+    const uint32_t hi = (uint32_t)(left >> 32), lo = (uint32_t)left;
+    const uint32_t sh = off & 31u, w = off >> 5;
+    const uint32_t w0 = hi >> sh;
+    const uint32_t w1 = __funnelshift_r(lo, hi, sh);
+    const uint32_t w2 = __funnelshift_r(0u, lo, sh);
+    if (w0) atomicOr(&buf[w], w0);
+    if (n + sh > 32u && w1) atomicOr(&buf[w + 1], w1);
+    if (n + sh > 64u && w2) atomicOr(&buf[w + 2], w2);
+}
+
+template <bool kFromSym>
+__global__ void __launch_bounds__(kThreads) pack_kernel(PackArgs a) {
+    __shared__ uint32_t s_enc[256];
+    __shared__ uint32_t s_bits[kSlotWords + 4];
+    __shared__ uint32_t s_scan[8];
+    const Ctrl* ctrl = a.ws.ctrl;
+    if (ctrl->abort) return;
+    const uint32_t chunk = blockIdx.x, u = blockIdx.y, tid = threadIdx.x;
+    if (chunk >= ctrl->n_chunks) return;
+    const ChunkPos pos = locate_chunk(a.ws, a.segs, a.n_seg, chunk);
+    s_enc[tid] = a.ws.enc_lut[pos.seg * 256 + tid];
+    for (uint32_t i = tid; i < (uint32_t)kSlotWords + 4; i += kThreads) s_bits[i] = 0;
+    __syncthreads();
+
+    const uint32_t i0 = tid * 8;
+    const uint32_t nv = pos.cnt > i0 ? min(8u, pos.cnt - i0) : 0u;
+    uint32_t s[8];
+    uint32_t n_sat = 0, n_nf = 0;
+    if (nv) {
+        const uint64_t e = (uint64_t)u * a.client_stride + pos.elem0 + i0;
+        if (kFromSym) {
+            load_sym8(a.sym + e, nv, s);
+        } else {
+            const FmtDev f = a.ws.fmt[pos.seg];
+            float g[8], m[8];
+            load8(a.grad + e, nv, g);
+            load8(a.mem + e, nv, m);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                uint32_t fl = 0;
+                m[j] = convert_one(g[j], m[j], a.decay, f, s[j], fl);
+                if ((uint32_t)j < nv) { n_sat += fl & 1u; n_nf += fl >> 1; }
+            }
+            store8(a.mem + e, nv, m);
+        }
+    }
+    // codewords of this thread's symbols, concatenated in two 64-bit halves
+    uint64_t wa = 0, wb = 0;
+    uint32_t la = 0, lb = 0;
+    bool missing = false;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        if ((uint32_t)j < nv) {
+            const uint32_t ent = s_enc[s[j]];
+            const uint32_t l = ent & 0xffu;
+            missing |= (l == 0);
+            if (j < 4) { wa = (wa << l) | (ent >> 8); la += l; }
+            else       { wb = (wb << l) | (ent >> 8); lb += l; }
+        }
+    }
+    uint32_t total;
+    const uint32_t off = block_exclusive_scan_256(la + lb, s_scan, &total);
+    put_bits(s_bits, off, wa, la);
+    put_bits(s_bits, off + la, wb, lb);
+    uint8_t* stream = a.streams + (size_t)u * a.stream_capacity;
+    if ((tid & 15u) == 0)
+        *reinterpret_cast<uint16_t*>(stream + ctrl->sub_off + 2ull * ((uint64_t)chunk * kSubs + (tid >> 4))) = (uint16_t)off;
+    if (!kFromSym) add_counts(&a.res[u], n_sat, n_nf);
+    if (__syncthreads_or(missing)) {
+        if (tid == 0) {
+            set_status(&a.res[u], CO3_ERR_NO_CODEWORD);
+            atomicMin(&a.res[u].first_bad_chunk, chunk);
+            a.ws.client_fail[u] = 1u;
+        }
+    }
+    const size_t ci = (size_t)u * a.ws.n_chunks_max + chunk;
+    if (tid == 0) a.ws.chunk_bits[ci] = total;
+    const uint32_t words = (total + 31u) >> 5;
+    uint32_t* slot = a.ws.slots + ci * kSlotWords;
+    for (uint32_t i = tid; i < words; i += kThreads) slot[i] = s_bits[i];
+}
+
+// ------------------------------------------------------------------------------------------------
+// scan: one block of 1024 threads per client.  Prefix sums of the chunk sizes give every chunk its
+// place in the payload; the same block writes the header and the segment table.
+// ------------------------------------------------------------------------------------------------
+struct ScanArgs {
+    const co3_seg* segs;
+    uint32_t n_seg;
+    uint64_t n_elem;
+    uint8_t* streams;
+    size_t stream_capacity;
+    co3_result* res;
+    Ws ws;
+};
+
+constexpr int kScanThreads = 1024;
+
+__global__ void __launch_bounds__(kScanThreads) scan_kernel(ScanArgs a) {
+    __shared__ uint64_t s_w[32], s_b[32];
+    const Ctrl* ctrl = a.ws.ctrl;
+    if (ctrl->abort) return;
+    const uint32_t u = blockIdx.x, tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
+    const uint32_t n = ctrl->n_chunks;
+    const uint32_t* bits = a.ws.chunk_bits + (size_t)u * a.ws.n_chunks_max;
+    uint64_t* bit_prefix = a.ws.bit_prefix + (size_t)u * (a.ws.n_chunks_max + 1ull);
+    uint8_t* stream = a.streams + (size_t)u * a.stream_capacity;
+    uint64_t* word_off = reinterpret_cast<uint64_t*>(stream + ctrl->chunk_off);
+
+    const uint32_t per = (n + kScanThreads - 1) / kScanThreads;
+    const uint32_t lo = min(tid * per, n), hi = min(lo + per, n);
+    uint64_t sw = 0, sb = 0;
+    for (uint32_t c = lo; c < hi; ++c) {
+        const uint32_t b = bits[c];
+        sb += b;
+        sw += (b + 31u) >> 5;
+    }
+    uint64_t iw = sw, ib = sb;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const uint64_t yw = __shfl_up_sync(0xffffffffu, iw, d), yb = __shfl_up_sync(0xffffffffu, ib, d);
+        if (lane >= (uint32_t)d) { iw += yw; ib += yb; }
+    }
+    if (lane == 31u) { s_w[warp] = iw; s_b[warp] = ib; }
+    __syncthreads();
+    uint64_t bw = 0, bb = 0, tw = 0, tb = 0;
+    for (uint32_t w = 0; w < 32; ++w) {
+        if (w < warp) { bw += s_w[w]; bb += s_b[w]; }
+        tw += s_w[w];
+        tb += s_b[w];
+    }
+    uint64_t pw = bw + iw - sw, pb = bb + ib - sb;  // exclusive prefix of this thread's range
+
+    const uint64_t total_bytes = align16(ctrl->payload_off + 4ull * tw);
+    const bool fits = total_bytes <= a.stream_capacity;
+    const bool failed = a.ws.client_fail[u] != 0;
+    for (uint32_t c = lo; c < hi; ++c) {
+        word_off[c] = pw;
+        bit_prefix[c] = pb;
+        const uint32_t b = bits[c];
+        pb += b;
+        pw += (b + 31u) >> 5;
+    }
+    if (tid == 0) {
+        word_off[n] = tw;
+        bit_prefix[n] = tb;
+    }
+    __syncthreads();
+    for (uint32_t k = tid; k < a.n_seg; k += kScanThreads) {
+        uint64_t* e = reinterpret_cast<uint64_t*>(stream + kHeaderBytes + 24ull * k);
+        const uint32_t c0 = a.ws.first_chunk[k], c1 = a.ws.first_chunk[k + 1];
+        e[0] = a.segs[k].n_elem;
+        e[1] = c0;
+        e[2] = bit_prefix[c1] - bit_prefix[c0];
+    }
+    if (tid == 0) {
+        uint32_t* h32 = reinterpret_cast<uint32_t*>(stream);
+        uint64_t* h64 = reinterpret_cast<uint64_t*>(stream);
+        h32[0] = kMagic; h32[1] = 1u; h32[2] = a.n_seg; h32[3] = kC; h32[4] = kS; h32[5] = 0u;
+        h64[3] = a.n_elem; h64[4] = n; h64[5] = tw; h64[6] = tb; h64[7] = total_bytes;
+        // table padding up to the next section
+        for (uint64_t o = kHeaderBytes + 24ull * a.n_seg; o < ctrl->chunk_off; o += 8) *reinterpret_cast<uint64_t*>(stream + o) = 0;
+        for (uint64_t o = ctrl->chunk_off + 8ull * (n + 1ull); o < ctrl->sub_off; o += 8) *reinterpret_cast<uint64_t*>(stream + o) = 0;
+        for (uint64_t o = ctrl->sub_off + 2ull * n * kSubs; o < ctrl->payload_off; o += 8) *reinterpret_cast<uint64_t*>(stream + o) = 0;
+        co3_result* r = &a.res[u];
+        r->payload_bits = tb;
+        r->container_bytes = total_bytes;
+        if (!fits) {
+            set_status(r, CO3_ERR_CAPACITY);
+            a.ws.client_fail[u] = 1u;
+        } else if (!failed) {
+            for (uint64_t o = ctrl->payload_off + 4ull * tw; o < total_bytes; o += 4) *reinterpret_cast<uint32_t*>(stream + o) = 0;
+        }
+    }
+}
+
+// compact: one block per (chunk, client) moves the chunk's words to their final position.
+__global__ void __launch_bounds__(kThreads) compact_kernel(ScanArgs a) {
+    const Ctrl* ctrl = a.ws.ctrl;
+    if (ctrl->abort) return;
+    const uint32_t chunk = blockIdx.x, u = blockIdx.y, tid = threadIdx.x;
+    if (chunk >= ctrl->n_chunks || a.ws.client_fail[u]) return;
+    uint8_t* stream = a.streams + (size_t)u * a.stream_capacity;
+    const uint64_t w0 = reinterpret_cast<const uint64_t*>(stream + ctrl->chunk_off)[chunk];
+    const size_t ci = (size_t)u * a.ws.n_chunks_max + chunk;
+    const uint32_t words = (a.ws.chunk_bits[ci] + 31u) >> 5;
+    const uint32_t* slot = a.ws.slots + ci * kSlotWords;
+    uint32_t* dst = reinterpret_cast<uint32_t*>(stream + ctrl->payload_off) + w0;
+    for (uint32_t i = tid; i < words; i += kThreads) dst[i] = slot[i];
+}
+
+// ------------------------------------------------------------------------------------------------
+// decode
+// ------------------------------------------------------------------------------------------------
+struct DecArgs {
+    const uint8_t* const* streams;  // device array of n_clients pointers, or null:
+    const uint8_t* single;          // the one stream when `streams` is null
+    size_t stream_bytes;
+    uint32_t n_clients;
+    const co3_seg* segs;
+    uint32_t n_seg;
+    uint64_t n_elem;
+    float* out;        // average (or the single client's values); nullable when sym_out is given
+    uint8_t* sym_out;  // nullable; only with n_clients == 1
+    co3_result* res;
+    Ws ws;
+};
+
+__device__ __forceinline__ const uint8_t* stream_of(const DecArgs& a, uint32_t u) {
+    return a.streams ? a.streams[u] : a.single;
+}
+
+// One block per client: the header and the tables must describe exactly the expected layout.
+__global__ void __launch_bounds__(kThreads) check_streams_kernel(DecArgs a) {
+    const Ctrl* ctrl = a.ws.ctrl;
+    if (ctrl->abort) return;
+    const uint32_t u = blockIdx.x, tid = threadIdx.x;
+    const uint8_t* stream = stream_of(a, u);
+    bool bad = false;
+    if (stream == nullptr || (reinterpret_cast<uintptr_t>(stream) & 15u)) {
+        bad = true;
+    } else {
+        const uint32_t* h32 = reinterpret_cast<const uint32_t*>(stream);
+        const uint64_t* h64 = reinterpret_cast<const uint64_t*>(stream);
+        const uint64_t n = ctrl->n_chunks;
+        if (a.stream_bytes < ctrl->payload_off) {
+            bad = true;
+        } else {
+            const uint64_t cap_words = (a.stream_bytes - ctrl->payload_off) / 4;
+            if (h32[0] != kMagic || h32[1] != 1u || h32[2] != a.n_seg || h32[3] != (uint32_t)kC || h32[4] != (uint32_t)kS ||
+                h64[3] != a.n_elem || h64[4] != n || h64[5] > cap_words || h64[7] > a.stream_bytes ||
+                h64[7] != align16(ctrl->payload_off + 4ull * h64[5]))
+                bad = true;
+            if (!bad && reinterpret_cast<const uint64_t*>(stream + ctrl->chunk_off)[n] != h64[5]) bad = true;
+            if (!bad) {
+                for (uint32_t k = tid; k < a.n_seg; k += kThreads) {
+                    const uint64_t* e = reinterpret_cast<const uint64_t*>(stream + kHeaderBytes + 24ull * k);
+                    if (e[0] != a.segs[k].n_elem || e[1] != a.ws.first_chunk[k]) bad = true;
+                }
+            }
+            if (!bad && tid == 0) {
+                atomicAdd(reinterpret_cast<unsigned long long*>(&a.res->payload_bits), (unsigned long long)h64[6]);
+                atomicAdd(reinterpret_cast<unsigned long long*>(&a.res->container_bytes), (unsigned long long)h64[7]);
+            }
+        }
+    }
+    if (__syncthreads_or(bad) && tid == 0) {
+        set_status(a.res, CO3_ERR_CORRUPT);
+        a.ws.ctrl->abort = 1u;
+    }
+}
+
+// Sequential reader of one sub-chunk: a 64-bit window over the chunk's words, bounds-checked.
+struct BitReader {
+    const uint32_t* base;  // generic pointer: shared (staged) or global
+    uint32_t nwords;
+    uint32_t next;  // next word to fetch
+    uint64_t buf;   // unread bits, left-aligned
+    int have;       // number of valid bits in buf
+
+    __device__ __forceinline__ uint32_t word(uint32_t i) const { return i < nwords ? base[i] : 0u; }
+    __device__ __forceinline__ void init(const uint32_t* b, uint32_t n, uint32_t bit_off) {
+        base = b;
+        nwords = n;
+        const uint32_t w = bit_off >> 5, sh = bit_off & 31u;
+        buf = (((uint64_t)word(w) << 32) | word(w + 1)) << sh;
+        have = 64 - (int)sh;
+        next = w + 2;
+    }
+    __device__ __forceinline__ void refill() {  // keeps at least 32 valid bits
+        if (have <= 32) {
+            buf |= (uint64_t)word(next) << (32 - have);
+            ++next;
+            have += 32;
+        }
+    }
+    __device__ __forceinline__ uint32_t position() const { return next * 32u - (uint32_t)have; }
+};
+
+// Decodes one symbol.  Returns the symbol; sets err when the bits are no codeword.
+__device__ __forceinline__ uint32_t decode_one(BitReader& br, const uint16_t* __restrict__ s_lut,
+                                               const uint32_t* __restrict__ long_tab, bool& err) {
+    const uint32_t top = (uint32_t)(br.buf >> 32);
+    const uint32_t ent = s_lut[top >> (32 - kDecBits)];
+    uint32_t len = ent >> 8, sym = ent & 0xffu;
+    if (len > (uint32_t)kDecBits) {  // codeword longer than the table index: search the short list
+        const uint32_t w16 = top >> 16, cnt = min(long_tab[0], 256u);
+        len = 0;
+        for (uint32_t i = 0; i < cnt; ++i) {
+            const uint32_t e = long_tab[1 + i];
+            const uint32_t l = (e >> 8) & 0xffu;
+            if ((w16 >> (16u - l)) == (e >> 16)) { len = l; sym = e & 0xffu; break; }
+        }
+    }
+    if (len == 0) { err = true; len = 1; sym = 0; }
+    br.buf <<= len;
+    br.have -= (int)len;
+    return sym;
+}
+
+template <int B, int G>
+struct DecSmem {
+    static constexpr int kPairs = B * G;
+    static constexpr int kPayWords = kPairs * 384;  // staging for ~6 bits/symbol; larger chunks are read in place
+    uint16_t lut[kDecLut];
+    float val[256];
+    uint32_t sym[kPairs][kC / 4];
+    uint32_t pay[kPayWords];
+    const uint32_t* pair_base[kPairs];
+    uint32_t pair_words[kPairs];
+    uint32_t pair_chunk[kPairs];
+    uint32_t pair_cnt[kPairs];
+};
+
+// Position of word j of sub-chunk s in the symbol buffer of pair p: rotated so that the 32 threads of a
+// warp (2 pairs x 16 sub-chunks, all at the same j) hit 32 different banks, and so do 32 consecutive j.
+__device__ __forceinline__ uint32_t sym_slot(uint32_t p, uint32_t s, uint32_t j) {
+    return s * 32u + ((j + s + 16u * (p & 1u)) & 31u);
+}
+
+template <int B, int G>
+__global__ void __launch_bounds__(16 * B * G) decode_kernel(DecArgs a) {
+    constexpr int kPairs = B * G;
+    constexpr int kT = 16 * kPairs;
+    constexpr int kWordsPerThread = (G * (kC / 4)) / kT;  // symbol words each thread sums per tile = 32 / B
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    DecSmem<B, G>& sm = *reinterpret_cast<DecSmem<B, G>*>(smem_raw);
+
+    const Ctrl* ctrl = a.ws.ctrl;
+    if (ctrl->abort) return;
+    const uint32_t tile = blockIdx.x, tid = threadIdx.x;
+    if (tile >= ctrl->n_tiles) return;
+    const uint32_t seg = find_seg(a.ws.first_tile, a.n_seg, tile);
+    const uint32_t chunk0 = a.ws.first_chunk[seg] + (tile - a.ws.first_tile[seg]) * G;
+    const uint32_t n_chunks_tile = min((uint32_t)G, a.ws.first_chunk[seg + 1] - chunk0);
+    const co3_seg sg = a.segs[seg];
+    const uint64_t cap_words = (a.stream_bytes - ctrl->payload_off) / 4;
+
+    for (uint32_t i = tid; i < (uint32_t)kDecLut / 2; i += kT)
+        reinterpret_cast<uint32_t*>(sm.lut)[i] = reinterpret_cast<const uint32_t*>(a.ws.dec_lut + (size_t)seg * kDecLut)[i];
+    for (uint32_t i = tid; i < 256; i += kT) sm.val[i] = a.ws.val_lut[seg * 256 + i];
+    const uint32_t* long_tab = a.ws.dec_long + (size_t)seg * kLongStride;
+
+    float carry[kWordsPerThread][4];  // running sums across client batches (only when G == 1)
+    bool err = false;
+
+    for (uint32_t u0 = 0; u0 < a.n_clients; u0 += B) {
+        const uint32_t nb = min((uint32_t)B, a.n_clients - u0);
+        __syncthreads();  // previous batch fully consumed; LUTs visible
+        // ---- pair descriptors (pair = one chunk of one client) and staging plan
+        if (tid < 32) {
+            uint32_t nw = 0, cnt = 0, chunk = 0;
+            const uint32_t* base = nullptr;
+            if (tid < (uint32_t)kPairs) {
+                const uint32_t cl = tid / B, ul = tid % B;
+                if (cl < n_chunks_tile && ul < nb) {
+                    chunk = chunk0 + cl;
+                    const uint8_t* stream = stream_of(a, u0 + ul);
+                    const uint64_t* word_off = reinterpret_cast<const uint64_t*>(stream + ctrl->chunk_off);
+                    const uint64_t w0 = word_off[chunk], w1 = word_off[chunk + 1];
+                    const uint64_t start = (uint64_t)(chunk - a.ws.first_chunk[seg]) * kC;
+                    cnt = (uint32_t)min((uint64_t)kC, sg.n_elem - start);
+                    if (w0 > w1 || w1 > cap_words || w1 - w0 > (uint64_t)kSlotWords) {
+                        err = true;
+                        cnt = 0;
+                    } else {
+                        nw = (uint32_t)(w1 - w0);
+                        base = reinterpret_cast<const uint32_t*>(stream + ctrl->payload_off) + w0;
+                    }
+                }
+            }
+            uint32_t inc = nw;  // inclusive prefix of the staged sizes over the pairs
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                const uint32_t y = __shfl_up_sync(0xffffffffu, inc, d);
+                if (tid >= (uint32_t)d) inc += y;
+            }
+            if (tid < (uint32_t)kPairs) {
+                const bool staged = inc <= (uint32_t)DecSmem<B, G>::kPayWords;
+                if (staged && nw) {
+                    uint32_t* dst = sm.pay + (inc - nw);
+                    sm.pair_base[tid] = dst;
+                } else {
+                    sm.pair_base[tid] = base;  // read in place
+                }
+                sm.pair_words[tid] = (staged ? 0x80000000u : 0u) | nw;
+                sm.pair_chunk[tid] = chunk;
+                sm.pair_cnt[tid] = cnt;
+                // remember the source for the copy below
+                if (staged && nw) reinterpret_cast<const uint32_t**>(sm.sym[tid])[0] = base;
+            }
+        }
+        __syncthreads();
+        // ---- stage the payloads (coalesced)
+        for (uint32_t p = 0; p < (uint32_t)kPairs; ++p) {
+            const uint32_t pw = sm.pair_words[p];
+            if (!(pw & 0x80000000u) || !(pw & 0x7fffffffu)) continue;
+            const uint32_t* src = reinterpret_cast<const uint32_t* const*>(sm.sym[p])[0];
+            uint32_t* dst = const_cast<uint32_t*>(sm.pair_base[p]);
+            const uint32_t nw = pw & 0x7fffffffu;
+            for (uint32_t i = tid; i < nw; i += kT) dst[i] = __ldg(src + i);
+        }
+        __syncthreads();
+        // ---- decode: thread = (pair, sub-chunk)
+        {
+            const uint32_t p = tid >> 4, s = tid & 15u;
+            const uint32_t cnt = sm.pair_cnt[p];
+            const uint32_t nw = sm.pair_words[p] & 0x7fffffffu;
+            const uint32_t my = cnt > s * kS ? min((uint32_t)kS, cnt - s * kS) : 0u;
+            uint32_t* out = sm.sym[p];
+            if (my) {
+                const uint32_t cl = p / B, ul = p % B;
+                const uint8_t* stream = stream_of(a, u0 + ul);
+                const uint16_t* sub = reinterpret_cast<const uint16_t*>(stream + ctrl->sub_off) + (uint64_t)(chunk0 + cl) * kSubs;
+                const uint32_t off = sub[s];
+                const bool last = cnt <= (s + 1) * kS;
+                if (off > nw * 32u) {
+                    err = true;
+                    for (uint32_t j = 0; j < 32; ++j) out[sym_slot(p, s, j)] = 0;
+                } else {
+                    BitReader br;
+                    br.init(sm.pair_base[p], nw, off);
+                    for (uint32_t j = 0; j < 32; ++j) {  // four symbols per output word
+                        uint32_t w = 0;
+                        if (j * 4 < my) {
+                            br.refill();
+                            const uint32_t s0 = decode_one(br, sm.lut, long_tab, err);
+                            const uint32_t s1 = (j * 4 + 1 < my) ? decode_one(br, sm.lut, long_tab, err) : 0u;
+                            br.refill();
+                            const uint32_t s2 = (j * 4 + 2 < my) ? decode_one(br, sm.lut, long_tab, err) : 0u;
+                            const uint32_t s3 = (j * 4 + 3 < my) ? decode_one(br, sm.lut, long_tab, err) : 0u;
+                            w = s0 | (s1 << 8) | (s2 << 16) | (s3 << 24);
+                        }
+                        out[sym_slot(p, s, j)] = w;
+                    }
+                    const uint32_t end = br.position();
+                    if (!last) {
+                        if (end != sub[s + 1]) err = true;
+                    } else if (((end + 31u) >> 5) != nw) {
+                        err = true;
+                    }
+                }
+            } else {
+                for (uint32_t j = 0; j < 32; ++j) out[sym_slot(p, s, j)] = 0;
+            }
+        }
+        __syncthreads();
+        // ---- ordered sum over the clients of this batch; thread owns whole symbol words
+        const bool first_batch = (u0 == 0), last_batch = (u0 + B >= a.n_clients);
+#pragma unroll
+        for (int r = 0; r < kWordsPerThread; ++r) {
+            const uint32_t w = tid + r * kT;         // word index inside the tile
+            const uint32_t cl = w / (kC / 4), wi = w % (kC / 4);
+            const uint32_t s = wi >> 5, j = wi & 31u;
+            float acc[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) acc[q] = (G == 1 && !first_batch) ? carry[r][q] : 0.0f;
+            uint32_t symw = 0;
+            for (uint32_t ul = 0; ul < nb; ++ul) {
+                const uint32_t p = cl * B + ul;
+                symw = sm.sym[p][sym_slot(p, s, j)];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) acc[q] = __fadd_rn(acc[q], sm.val[(symw >> (8 * q)) & 0xffu]);
+            }
+            if (G == 1 && !last_batch) {
+#pragma unroll
+                for (int q = 0; q < 4; ++q) carry[r][q] = acc[q];
+                continue;
+            }
+            if (cl >= n_chunks_tile) continue;
+            const uint32_t cnt = sm.pair_cnt[cl * B];
+            const uint32_t i0 = wi * 4;
+            if (i0 >= cnt) continue;
+            const uint32_t nv = min(4u, cnt - i0);
+            const uint64_t e = sg.elem_off + (uint64_t)(chunk0 + cl - a.ws.first_chunk[seg]) * kC + i0;
+            if (a.out) {
+                const float U = (float)a.n_clients;
+                float* o = a.out + e;
+                if (nv == 4 && (reinterpret_cast<uintptr_t>(o) & 15u) == 0) {
+                    *reinterpret_cast<float4*>(o) = make_float4(__fdiv_rn(acc[0], U), __fdiv_rn(acc[1], U),
+                                                                __fdiv_rn(acc[2], U), __fdiv_rn(acc[3], U));
+                } else {
+                    for (uint32_t q = 0; q < nv; ++q) o[q] = __fdiv_rn(acc[q], U);
+                }
+            }
+            if (a.sym_out) {
+                uint8_t* o = a.sym_out + e;
+                if (nv == 4 && (reinterpret_cast<uintptr_t>(o) & 3u) == 0) {
+                    *reinterpret_cast<uint32_t*>(o) = symw;
+                } else {
+                    for (uint32_t q = 0; q < nv; ++q) o[q] = (uint8_t)(symw >> (8 * q));
+                }
+            }
+        }
+    }
+    if (__syncthreads_or(err) && tid == 0) {
+        set_status(a.res, CO3_ERR_CORRUPT);
+        atomicMin(&a.res->first_bad_chunk, chunk0);
+    }
+}
+
+}  // namespace co3
+
+// ================================================================================================
+// Host side: argument checks, workspace layout, launches.
+// ================================================================================================
+using namespace co3;
+
+namespace {
+
+struct WsLayout {
+    size_t ctrl, first_chunk, first_tile, fmt, enc_lut, dec_lut, dec_long, val_lut, client_fail, chunk_bits,
+        bit_prefix, slots, total;
+    uint32_t n_chunks_max;
+};
+
+size_t up256(size_t x) { return (x + 255) & ~(size_t)255; }
+
+bool ws_layout(uint64_t n_elem, uint32_t n_seg, uint32_t n_clients, WsLayout* L) {
+    if (n_elem > (1ull << 40) || n_seg > (1u << 20)) return false;
+    const uint64_t nc = n_elem / kC + n_seg;  // upper bound of the chunks of one client
+    if (nc >= (1ull << 31)) return false;
+    L->n_chunks_max = (uint32_t)nc;
+    size_t o = 0;
+    L->ctrl = o;        o += up256(sizeof(Ctrl));
+    L->first_chunk = o; o += up256(4 * ((size_t)n_seg + 1));
+    L->first_tile = o;  o += up256(4 * ((size_t)n_seg + 1));
+    L->fmt = o;         o += up256(sizeof(FmtDev) * (size_t)n_seg);
+    L->enc_lut = o;     o += up256(4 * 256 * (size_t)n_seg);
+    L->dec_lut = o;     o += up256(2 * (size_t)kDecLut * n_seg);
+    L->dec_long = o;    o += up256(4 * (size_t)kLongStride * n_seg);
+    L->val_lut = o;     o += up256(4 * 256 * (size_t)n_seg);
+    L->client_fail = o; o += up256(4 * (size_t)(n_clients ? n_clients : 1));
+    L->chunk_bits = o;  o += up256(4 * (size_t)n_clients * nc);
+    L->bit_prefix = o;  o += up256(8 * (size_t)n_clients * (nc + 1));
+    L->slots = o;       o += up256(4 * (size_t)kSlotWords * n_clients * nc);
+    L->total = o;
+    return true;
+}
+
+Ws ws_pointers(void* base, const WsLayout& L) {
+    char* b = static_cast<char*>(base);
+    Ws w;
+    w.ctrl = reinterpret_cast<Ctrl*>(b + L.ctrl);
+    w.first_chunk = reinterpret_cast<uint32_t*>(b + L.first_chunk);
+    w.first_tile = reinterpret_cast<uint32_t*>(b + L.first_tile);
+    w.fmt = reinterpret_cast<FmtDev*>(b + L.fmt);
+    w.enc_lut = reinterpret_cast<uint32_t*>(b + L.enc_lut);
+    w.dec_lut = reinterpret_cast<uint16_t*>(b + L.dec_lut);
+    w.dec_long = reinterpret_cast<uint32_t*>(b + L.dec_long);
+    w.val_lut = reinterpret_cast<float*>(b + L.val_lut);
+    w.client_fail = reinterpret_cast<uint32_t*>(b + L.client_fail);
+    w.chunk_bits = reinterpret_cast<uint32_t*>(b + L.chunk_bits);
+    w.bit_prefix = reinterpret_cast<uint64_t*>(b + L.bit_prefix);
+    w.slots = reinterpret_cast<uint32_t*>(b + L.slots);
+    w.n_chunks_max = L.n_chunks_max;
+    return w;
+}
+
+// Largest possible size of the container sections that precede the payload.
+uint64_t fixed_part_bound(uint32_t n_seg, uint64_t n_chunks_max) {
+    uint64_t o = align16(kHeaderBytes + 24ull * n_seg);
+    o = align16(o + 8ull * (n_chunks_max + 1));
+    o = align16(o + 2ull * n_chunks_max * kSubs);
+    return o;
+}
+
+bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+
+#define CO3_CUDA(call)                                  \
+    do {                                                \
+        if ((call) != cudaSuccess) return CO3_ERR_CUDA; \
+    } while (0)
+
+int begin_call(const WsLayout& L, const Ws& ws, co3_result* res, uint32_t n_res, cudaStream_t st,
+               const co3_fmt* fmts, const co3_code* codes, const co3_seg* segs, uint32_t n_seg, uint64_t n_elem,
+               uint32_t tile_chunks, uint32_t n_fail) {
+    CO3_CUDA(cudaMemsetAsync(ws.ctrl, 0, sizeof(Ctrl), st));
+    CO3_CUDA(cudaMemsetAsync(res, 0, sizeof(co3_result) * (size_t)n_res, st));
+    CO3_CUDA(cudaMemsetAsync(ws.client_fail, 0, 4 * (size_t)(n_fail ? n_fail : 1), st));
+    PrepArgs pa{fmts, codes, segs, n_seg, n_elem, tile_chunks, res, n_res, ws};
+    prepare_kernel<<<n_seg ? n_seg : 1, kThreads, 0, st>>>(pa);
+    CO3_CUDA(cudaGetLastError());
+    (void)L;
+    return CO3_OK;
+}
+
+template <int B, int G>
+int launch_decode(const DecArgs& da, uint32_t n_tiles_max, cudaStream_t st) {
+    const size_t smem = sizeof(DecSmem<B, G>);
+    CO3_CUDA(cudaFuncSetAttribute(decode_kernel<B, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    if (n_tiles_max == 0) return CO3_OK;
+    decode_kernel<B, G><<<n_tiles_max, 16 * B * G, smem, st>>>(da);
+    CO3_CUDA(cudaGetLastError());
+    return CO3_OK;
+}
+
+int decode_common(const uint8_t* const* streams, const uint8_t* single, size_t stream_bytes, uint32_t n_clients, const co3_fmt* fmts,
+                  const co3_code* codes, const co3_seg* segs, uint32_t n_seg, uint64_t n_elem, uint32_t chunk_syms,
+                  float* out, uint8_t* sym_out, void* workspace, size_t workspace_bytes, co3_result* res,
+                  cudaStream_t st) {
+    if ((!streams && !single) || !fmts || !codes || !res || !workspace || n_clients == 0 || chunk_syms != (uint32_t)kC)
+        return CO3_ERR_INVALID_ARG;
+    if ((!segs && n_seg) || (!out && !sym_out) || (sym_out && n_clients != 1)) return CO3_ERR_INVALID_ARG;
+    if (!aligned(workspace, 256) || (out && !aligned(out, 16)) || !aligned(res, 8)) return CO3_ERR_INVALID_ARG;
+    WsLayout L;
+    if (!ws_layout(n_elem, n_seg, 0, &L)) return CO3_ERR_INVALID_ARG;
+    if (workspace_bytes < L.total) return CO3_ERR_CAPACITY;
+    const Ws ws = ws_pointers(workspace, L);
+
+    // clients decoded side by side per block (B) and chunks per block (G): 16 sub-chunk threads per pair
+    int B = 1;
+    while (B < 16 && (uint32_t)B < n_clients) B <<= 1;
+    int G = 16 / B;
+    const uint64_t chunks = L.n_chunks_max;
+    if (G > 1 && chunks / G < 2 * 148) G = (4 / B) > 0 ? 4 / B : 1;  // small inputs: more, smaller blocks
+    const int rc = begin_call(L, ws, res, 1, st, fmts, codes, segs, n_seg, n_elem, (uint32_t)G, 1);
+    if (rc != CO3_OK) return rc;
+    DecArgs da{streams, single, stream_bytes, n_clients, segs, n_seg, n_elem, out, sym_out, res, ws};
+    check_streams_kernel<<<n_clients, kThreads, 0, st>>>(da);
+    CO3_CUDA(cudaGetLastError());
+    const uint32_t tiles = (uint32_t)(chunks / G + n_seg);  // upper bound; surplus blocks return at once
+#define CO3_DEC_CASE(b, g) \
+    if (B == b && G == g) return launch_decode<b, g>(da, tiles, st);
+    CO3_DEC_CASE(1, 16) CO3_DEC_CASE(1, 4) CO3_DEC_CASE(2, 8) CO3_DEC_CASE(2, 2) CO3_DEC_CASE(4, 4)
+    CO3_DEC_CASE(4, 1) CO3_DEC_CASE(8, 2) CO3_DEC_CASE(8, 1) CO3_DEC_CASE(16, 1)
+#undef CO3_DEC_CASE
+    return CO3_ERR_INVALID_ARG;
+}
+
+int encode_common(const float* grad, float* mem, float decay, const uint8_t* sym, const co3_fmt* fmts,
+                  const co3_code* codes, const co3_seg* segs, uint32_t n_seg, uint64_t n_elem, uint32_t n_clients,
+                  uint64_t client_stride, uint8_t* streams_out, size_t stream_capacity, uint32_t chunk_syms,
+                  void* workspace, size_t workspace_bytes, co3_result* res, cudaStream_t st) {
+    if (!codes || !res || !workspace || !streams_out || n_clients == 0 || n_clients > 65535u ||
+        chunk_syms != (uint32_t)kC)
+        return CO3_ERR_INVALID_ARG;
+    if (!segs && n_seg) return CO3_ERR_INVALID_ARG;
+    if (sym == nullptr && (!grad || !mem || !fmts || !aligned(grad, 16) || !aligned(mem, 16))) return CO3_ERR_INVALID_ARG;
+    if (!aligned(workspace, 256) || !aligned(streams_out, 16) || (stream_capacity & 15u) || !aligned(res, 8))
+        return CO3_ERR_INVALID_ARG;
+    if (n_clients > 1 && client_stride < n_elem) return CO3_ERR_INVALID_ARG;
+    WsLayout L;
+    if (!ws_layout(n_elem, n_seg, n_clients, &L)) return CO3_ERR_INVALID_ARG;
+    if (workspace_bytes < L.total) return CO3_ERR_CAPACITY;
+    if (stream_capacity < fixed_part_bound(n_seg, L.n_chunks_max)) return CO3_ERR_CAPACITY;
+    const Ws ws = ws_pointers(workspace, L);
+    const int rc = begin_call(L, ws, res, n_clients, st, sym ? nullptr : fmts, codes, segs, n_seg, n_elem, 1, n_clients);
+    if (rc != CO3_OK) return rc;
+    if (L.n_chunks_max) {
+        PackArgs pa{grad, mem, decay, sym, segs, n_seg, client_stride, streams_out, stream_capacity, res, ws};
+        const dim3 grid(L.n_chunks_max, n_clients);
+        if (sym) pack_kernel<true><<<grid, kThreads, 0, st>>>(pa);
+        else pack_kernel<false><<<grid, kThreads, 0, st>>>(pa);
+        CO3_CUDA(cudaGetLastError());
+    }
+    ScanArgs sa{segs, n_seg, n_elem, streams_out, stream_capacity, res, ws};
+    scan_kernel<<<n_clients, kScanThreads, 0, st>>>(sa);
+    CO3_CUDA(cudaGetLastError());
+    if (L.n_chunks_max) {
+        compact_kernel<<<dim3(L.n_chunks_max, n_clients), kThreads, 0, st>>>(sa);
+        CO3_CUDA(cudaGetLastError());
+    }
+    return CO3_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* co3_status_string(int status) {
+    switch (status) {
+        case CO3_OK: return "ok";
+        case CO3_ERR_INVALID_ARG: return "invalid argument or descriptor";
+        case CO3_ERR_CAPACITY: return "stream or workspace too small";
+        case CO3_ERR_NO_CODEWORD: return "symbol without codeword";
+        case CO3_ERR_NONFINITE: return "non-finite input (stream still valid)";
+        case CO3_ERR_CORRUPT: return "corrupt stream";
+        case CO3_ERR_CUDA: return "CUDA runtime error";
+        default: return "unknown status";
+    }
+}
+
+int co3_workspace_bytes(uint64_t n_elem, uint32_t n_seg, uint32_t n_clients, uint32_t chunk_syms, size_t* out) {
+    if (!out || chunk_syms != (uint32_t)kC) return CO3_ERR_INVALID_ARG;
+    WsLayout L;
+    if (!ws_layout(n_elem, n_seg, n_clients, &L)) return CO3_ERR_INVALID_ARG;
+    *out = L.total;
+    return CO3_OK;
+}
+
+int co3_stream_capacity_bytes(uint64_t n_elem, uint32_t n_seg, uint32_t chunk_syms, size_t* out) {
+    if (!out || chunk_syms != (uint32_t)kC) return CO3_ERR_INVALID_ARG;
+    WsLayout L;
+    if (!ws_layout(n_elem, n_seg, 0, &L)) return CO3_ERR_INVALID_ARG;
+    // every chunk rounds its bits up to a word: at most n_elem/2 words plus one per chunk
+    const uint64_t words = (n_elem * CO3_MAX_CODE_LEN + 31) / 32 + L.n_chunks_max;
+    *out = (size_t)align16(fixed_part_bound(n_seg, L.n_chunks_max) + 4ull * words);
+    return CO3_OK;
+}
+
+int co3_convert(const float* grad, float* mem, float decay, const co3_fmt* fmts, const co3_seg* segs, uint32_t n_seg,
+                uint64_t n_elem, uint32_t n_clients, uint64_t client_stride_elems, uint8_t* sym_out,
+                uint64_t* hist_out, co3_result* res, void* workspace, size_t workspace_bytes, void* stream) {
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (!grad || !mem || !fmts || !res || !workspace || n_clients == 0 || n_clients > 65535u) return CO3_ERR_INVALID_ARG;
+    if (!segs && n_seg) return CO3_ERR_INVALID_ARG;
+    if (!aligned(grad, 16) || !aligned(mem, 16) || !aligned(workspace, 256) || !aligned(res, 8) ||
+        (hist_out && !aligned(hist_out, 8)))
+        return CO3_ERR_INVALID_ARG;
+    if (n_clients > 1 && client_stride_elems < n_elem) return CO3_ERR_INVALID_ARG;
+    WsLayout L;
+    if (!ws_layout(n_elem, n_seg, 0, &L)) return CO3_ERR_INVALID_ARG;
+    if (workspace_bytes < L.total) return CO3_ERR_CAPACITY;
+    const Ws ws = ws_pointers(workspace, L);
+    if (hist_out) CO3_CUDA(cudaMemsetAsync(hist_out, 0, 8 * 256 * (size_t)n_seg, st));
+    const int rc = begin_call(L, ws, res, n_clients, st, fmts, nullptr, segs, n_seg, n_elem, 1, 1);
+    if (rc != CO3_OK) return rc;
+    if (L.n_chunks_max == 0) return CO3_OK;
+    ConvertArgs ca{grad, mem, decay, segs, n_seg, client_stride_elems, sym_out, hist_out, res, ws};
+    const dim3 grid(L.n_chunks_max, n_clients);
+    if (sym_out && hist_out) convert_kernel<true, true><<<grid, kThreads, 0, st>>>(ca);
+    else if (sym_out) convert_kernel<true, false><<<grid, kThreads, 0, st>>>(ca);
+    else if (hist_out) convert_kernel<false, true><<<grid, kThreads, 0, st>>>(ca);
+    else convert_kernel<false, false><<<grid, kThreads, 0, st>>>(ca);
+    CO3_CUDA(cudaGetLastError());
+    return CO3_OK;
+}
+
+int co3_encode(const float* grad, float* mem, float decay, const co3_fmt* fmts, const co3_code* codes,
+               const co3_seg* segs, uint32_t n_seg, uint64_t n_elem, uint32_t n_clients, uint64_t client_stride_elems,
+               uint8_t* streams_out, size_t stream_capacity, uint32_t chunk_syms, void* workspace,
+               size_t workspace_bytes, co3_result* res, void* stream) {
+    if (!grad || !mem || !fmts) return CO3_ERR_INVALID_ARG;
+    return encode_common(grad, mem, decay, nullptr, fmts, codes, segs, n_seg, n_elem, n_clients, client_stride_elems,
+                         streams_out, stream_capacity, chunk_syms, workspace, workspace_bytes, res,
+                         static_cast<cudaStream_t>(stream));
+}
+
+int co3_encode_symbols(const uint8_t* sym, const co3_code* codes, const co3_seg* segs, uint32_t n_seg, uint64_t n_elem,
+                       uint32_t n_clients, uint64_t client_stride_elems, uint8_t* streams_out, size_t stream_capacity,
+                       uint32_t chunk_syms, void* workspace, size_t workspace_bytes, co3_result* res, void* stream) {
+    if (!sym) return CO3_ERR_INVALID_ARG;
+    return encode_common(nullptr, nullptr, 0.0f, sym, nullptr, codes, segs, n_seg, n_elem, n_clients,
+                         client_stride_elems, streams_out, stream_capacity, chunk_syms, workspace, workspace_bytes, res,
+                         static_cast<cudaStream_t>(stream));
+}
+
+int co3_decode_aggregate(const uint8_t* const* streams, size_t stream_bytes, uint32_t n_clients, const co3_fmt* fmts,
+                         const co3_code* codes, const co3_seg* segs, uint32_t n_seg, uint64_t n_elem,
+                         uint32_t chunk_syms, float* avg_out, void* workspace, size_t workspace_bytes, co3_result* res,
+                         void* stream) {
+    if (!avg_out) return CO3_ERR_INVALID_ARG;
+    if (!streams) return CO3_ERR_INVALID_ARG;
+    return decode_common(streams, nullptr, stream_bytes, n_clients, fmts, codes, segs, n_seg, n_elem, chunk_syms, avg_out,
+                         nullptr, workspace, workspace_bytes, res, static_cast<cudaStream_t>(stream));
+}
+
+int co3_decode(const uint8_t* stream_in, size_t stream_bytes, const co3_fmt* fmts, const co3_code* codes,
+               const co3_seg* segs, uint32_t n_seg, uint64_t n_elem, uint32_t chunk_syms, float* ghat_out,
+               uint8_t* sym_out, void* workspace, size_t workspace_bytes, co3_result* res, void* stream) {
+    if (!stream_in || !aligned(stream_in, 16)) return CO3_ERR_INVALID_ARG;
+    return decode_common(nullptr, stream_in, stream_bytes, 1, fmts, codes, segs, n_seg, n_elem, chunk_syms, ghat_out,
+                         sym_out, workspace, workspace_bytes, res, static_cast<cudaStream_t>(stream));
+}
+
+}  // extern "C"
