@@ -1,0 +1,374 @@
+#!/usr/bin/env python
+"""Benchmark of the CO3 hot path on B200: batched client encode + parameter-server decode-aggregate.
+
+One step = one training round of the workload: every client's gradient is corrected, converted,
+entropy-coded (memory updated) in one batched `co3_encode` call, then all streams are decoded and
+averaged by `co3_decode_aggregate`.  Prints one JSON line (see README for the keys).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config 2]
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "co3_encode_decode_aggregate_throughput"
+UNIT = "gradient elements/s"
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as fh:
+            p = json.load(fh)
+        return float(p["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    return 6650.0, "fallback (6.65 TB/s, earlier measurement on this pool)"
+
+
+def workload(cfg_idx: int, clients_override=None):
+    import co3_inputs as ci
+    cfg = ci.config(cfg_idx)
+    if "cells" in cfg:      # the sweep config: one representative cell
+        cell = cfg["cells"][0]
+        cfg = dict(cfg, fmt=cell["fmt"], beta=(cell["beta"],), decay=cell["decay"])
+    sizes = cfg["sizes"]
+    E, M = cfg["fmt"]
+    fmts = []
+    for k in range(len(sizes)):
+        s, inv = ci.scale_for(E, M, cfg["beta"][k], cfg["alpha"][k])
+        fmts.append((E, M, 0, s, inv))
+    clients = cfg["clients"] if clients_override is None else clients_override
+    return cfg, sizes, fmts, clients
+
+
+def make_grads(cfg, sizes, n_clients, stride, rnd, device, rank=0):
+    """[n_clients * stride] fp32 on `device`: client u, layer k i.i.d. GenNorm(beta_k, alpha_k)."""
+    import torch
+    import co3_inputs as ci
+    out = torch.zeros(n_clients * stride, dtype=torch.float32, device=device)
+    for u in range(n_clients):
+        seed = ci.client_round_seed(cfg["seed"] + 100_000 * rank, u, rnd)
+        off = u * stride
+        for k, n in enumerate(sizes):
+            out[off:off + n] = ci.gennorm(int(n), float(cfg["beta"][k]), float(cfg["alpha"][k]),
+                                          seed * 1_000_003 + k, device,
+                                          cfg.get("outlier_frac", 0.0), cfg.get("outlier_mult", 1.0))
+            off += n
+    return out
+
+
+class ClockSampler:
+    """nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.rows = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q, "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append(line.strip())
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            f = [x.strip() for x in r.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------------------------------------------ reference arm
+def oracle_step(cfg, sizes, fmts, n_clients, codes=None):
+    """One bounded sample of the workload through the CPU oracle.  Returns (elements, seconds, codes)."""
+    import co3_inputs as ci
+    import oracle
+    ofmts = [oracle.Fmt(E, M, 0, s, inv) for (E, M, _, s, inv) in fmts]
+    offs = np.concatenate([[0], np.cumsum(sizes)]).astype(np.int64)
+    n = int(offs[-1])
+    grads = []
+    for u in range(n_clients):
+        seed = ci.client_round_seed(cfg["seed"], u, 0)
+        grads.append(np.concatenate([ci.gennorm(int(sz), float(cfg["beta"][k]), float(cfg["alpha"][k]),
+                                                seed * 1_000_003 + k).numpy() for k, sz in enumerate(sizes)]))
+    mems = [np.zeros(n, dtype=np.float32) for _ in range(n_clients)]
+    if codes is None:        # setup, untimed: fit the per-layer codes on these gradients
+        hist = np.zeros((len(sizes), 256), dtype=np.uint64)
+        for u in range(n_clients):
+            for k in range(len(sizes)):
+                r = oracle.convert(grads[u][offs[k]:offs[k + 1]], np.zeros(int(sizes[k]), dtype=np.float32),
+                                   cfg["decay"], ofmts[k])
+                hist[k] += oracle.histogram(r["sym"])
+        codes = [oracle.code_build(hist[k], ofmts[k]) for k in range(len(sizes))]
+    t0 = time.perf_counter()
+    streams = []
+    for u in range(n_clients):
+        sym = np.empty(n, dtype=np.uint8)
+        for k in range(len(sizes)):
+            m = mems[u][offs[k]:offs[k + 1]]
+            r = oracle.convert(grads[u][offs[k]:offs[k + 1]], m, cfg["decay"], ofmts[k])
+            sym[offs[k]:offs[k + 1]] = r["sym"]
+        st, s = oracle.encode(sym, sizes, codes)
+        assert st == oracle.OK
+        streams.append(s)
+    st, avg = oracle.decode_aggregate(streams, sizes, ofmts, codes)
+    assert st == oracle.OK
+    dt = time.perf_counter() - t0
+    return n * n_clients, dt, codes
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cfg, sizes, fmts, clients = workload(args.config)
+    sample_clients = 1
+    codes = None
+    _, _, codes = oracle_step(cfg, sizes, fmts, sample_clients, None)
+    for _ in range(max(0, args.warmup - 1)):
+        oracle_step(cfg, sizes, fmts, sample_clients, codes)
+    elems, secs = 0, 0.0
+    for _ in range(args.steps):
+        e, dt, _ = oracle_step(cfg, sizes, fmts, sample_clients, codes)
+        elems += e
+        secs += dt
+    value = elems / secs
+    sample = "%d of %d clients per step, full layer layout (%d elements each)" % (sample_clients, clients, sum(sizes))
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * secs / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": cfg["name"], "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------------------------ our arm
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    import paper_2204_08211_b200 as co3
+    from paper_2204_08211_b200.session import Co3Session
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; there is no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    cfg, sizes, fmts, clients = workload(args.config, args.clients)
+    sess = Co3Session(sizes, fmts, clients, cfg["decay"], dev)
+    n_rounds = 2
+    grads = [make_grads(cfg, sizes, clients, sess.stride, r, dev, rank) for r in range(n_rounds)]
+    mems = sess.new_client_buffer()
+    # setup (untimed, as the paper reuses the fitted parameters for many rounds): one code per layer from the
+    # symbol statistics of the first round, summed over the clients
+    hist = sess.histogram(grads[0], sess.new_client_buffer())
+    sess.set_codes_from_weights(hist)
+    stream = torch.cuda.current_stream()
+
+    def step(i):
+        sess.encode(grads[i % n_rounds], mems, stream)
+        sess.decode_aggregate(stream)
+
+    def check():
+        er = sess.encode_results()
+        dr = sess.decode_result()
+        if (er["status"] != co3.OK).any() or dr["status"][0] != co3.OK:
+            raise RuntimeError("device status: encode %s decode %s" % (er["status"], dr["status"]))
+        return er, dr
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for i in range(args.warmup):
+        step(i)
+    barrier()
+    check()
+
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record(stream)
+    for i in range(args.steps):
+        step(args.warmup + i)
+    e1.record(stream)
+    barrier()
+    ms = e0.elapsed_time(e1)
+    clocks = sampler.stop() if rank == 0 else None
+    er, dr = check()
+    if world > 1:
+        t = torch.tensor([ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    elems_per_step = sess.n_elem * clients * world
+    value = elems_per_step * args.steps / (ms * 1e-3)
+
+    # ---- per-kernel times: a second pass of the same steps with an event pair around every launch
+    co3.co3_profile_enable(True)
+    for i in range(args.steps):
+        step(args.warmup + i)
+    torch.cuda.synchronize()
+    prof = co3.co3_profile_read()
+    co3.co3_profile_enable(False)
+    launches_per_step = sum(n for n, _ in prof.values()) // args.steps
+
+    # ---- end to end: pinned host gradients in, averaged gradient out, every step
+    host_g = [torch.empty(clients * sess.stride, dtype=torch.float32).pin_memory() for _ in range(n_rounds)]
+    for r in range(n_rounds):
+        host_g[r].copy_(grads[r])
+    host_avg = torch.empty(sess.n_elem, dtype=torch.float32).pin_memory()
+    dev_g = torch.empty_like(grads[0])
+    e2e_steps = max(2, min(args.steps, 10))
+
+    def e2e_step(i):
+        dev_g.copy_(host_g[i % n_rounds], non_blocking=True)
+        sess.encode(dev_g, mems, stream)
+        host_avg.copy_(sess.decode_aggregate(stream), non_blocking=True)
+
+    e2e_step(0)
+    barrier()
+    e0.record(stream)
+    for i in range(e2e_steps):
+        e2e_step(i + 1)
+    e1.record(stream)
+    barrier()
+    e2e_ms = e0.elapsed_time(e1)
+    if world > 1:
+        t = torch.tensor([e2e_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    check()
+    e2e_value = elems_per_step * e2e_steps / (e2e_ms * 1e-3)
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the dominant kernel (algorithmic bytes / measured duration)
+    peak, peak_src = load_peaks()
+    n_local = sess.n_elem * clients
+    container = float(er["container_bytes"].astype(np.float64).sum())
+    alg_bytes = {
+        "pack": 12.0 * n_local + container,          # g, m in; m and the container out
+        "decode": 4.0 * sess.n_elem + container,     # all containers in; the average out
+        "convert": 13.0 * n_local,
+    }
+    kernels = {}
+    for name, (n, tot) in prof.items():
+        if n == 0:
+            continue
+        avg_ms = tot / n
+        k = {"launches_per_step": n // args.steps, "avg_ms": avg_ms}
+        if name in alg_bytes:
+            k["algorithmic_gb_per_launch"] = alg_bytes[name] / 1e9
+            k["achieved_gbs"] = alg_bytes[name] / 1e9 / (avg_ms * 1e-3)
+            k["frac_of_peak"] = k["achieved_gbs"] / peak
+        kernels[name] = k
+    dom = max((k for k in kernels if k in alg_bytes), key=lambda k: kernels[k]["avg_ms"] * kernels[k]["launches_per_step"])
+    roofline = {"kernel": dom + "_kernel", "bound": "hbm", "achieved": kernels[dom]["achieved_gbs"], "peak": peak,
+                "unit": "GB/s", "frac": kernels[dom]["frac_of_peak"], "traffic": None, "peak_source": peak_src,
+                "timed": "second pass of the same steps with CUDA events around every launch"}
+    bits = float(er["payload_bits"].astype(np.float64).sum())
+
+    # ---- CPU baseline: the oracle on a bounded sample (one client, full layer layout)
+    cpu = None
+    if not args.no_cpu_baseline:
+        elems, secs, _ = oracle_step(cfg, sizes, fmts, 1, None)
+        cpu = {"value": elems / secs, "unit": UNIT, "cores": 1, "kind": "oracle",
+               "sample": "1 of %d clients, full layer layout (%d elements): convert + encode + decode" % (clients, sess.n_elem)}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+        "config": {"workload": cfg["name"], "clients_per_gpu": clients, "elements_per_client": sess.n_elem,
+                   "layers": sess.n_seg, "format": "[1,%d,%d]" % tuple(cfg["fmt"]), "decay": cfg["decay"],
+                   "mean_code_bits": bits / n_local, "container_bits_per_element": 8.0 * container / n_local,
+                   "l2": "inputs larger than L2 (%.0f MB of gradients and memory per step)" % (8.0 * n_local / 1e6),
+                   "parallelism": "replicas" if world > 1 else "single"},
+        "gpu_launches": launches_per_step * args.steps,
+        "effective_gbs": (alg_bytes["pack"] + alg_bytes["decode"]) * world / 1e9 / (ms / args.steps * 1e-3),
+        "roofline": roofline, "kernels": kernels, "clocks": clocks,
+        "e2e": {"value": e2e_value, "unit": UNIT, "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps,
+                "h2d_bytes_per_step": int(4 * clients * sess.stride), "d2h_bytes_per_step": int(4 * sess.n_elem)},
+        "cpu_baseline": cpu,
+    }
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=2)
+    ap.add_argument("--clients", type=int, default=None, help="override the clients per GPU (profiling small cases)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -187,6 +187,25 @@ int co3_decode(const uint8_t* stream_in, size_t stream_bytes,
                float* ghat_out, uint8_t* sym_out,
                void* workspace, size_t workspace_bytes, co3_result* res, void* stream);
 
+/*
+ * Diagnostics (no counterpart in the paper).  With profiling enabled every kernel launched by the
+ * entry points above is bracketed by a CUDA event pair on the caller's stream; co3_profile_read
+ * waits for those events, adds up the elapsed time and the number of launches per kernel kind
+ * (arrays of CO3_KERNEL_COUNT entries, [host]) and clears the records.  Off by default; at most
+ * 16384 launches are recorded between reads.  Not thread-safe, and not to be left on inside a
+ * stream capture.
+ */
+#define CO3_KERNEL_PREPARE 0  /* descriptor validation and derived tables */
+#define CO3_KERNEL_CONVERT 1  /* correct + convert + memory update (+ symbols, histogram) */
+#define CO3_KERNEL_PACK 2     /* (correct + convert + memory update +) codeword lookup, scan, bit packing */
+#define CO3_KERNEL_SCAN 3     /* chunk offsets, header, tables */
+#define CO3_KERNEL_COMPACT 4  /* payload compaction */
+#define CO3_KERNEL_CHECK 5    /* stream header validation */
+#define CO3_KERNEL_DECODE 6   /* decode + cross-client accumulate */
+#define CO3_KERNEL_COUNT 7
+int co3_profile_enable(int on);
+int co3_profile_read(double* total_ms /* [host] */, uint32_t* launches /* [host] */);
+
 #ifdef __cplusplus
 }
 #endif

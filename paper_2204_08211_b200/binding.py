@@ -48,7 +48,9 @@ def _load():
     L.co3_encode_symbols.argtypes = [vp, vp, vp, u32, u64, u32, u64, vp, sz, u32, vp, sz, vp, vp]
     L.co3_decode_aggregate.argtypes = [vp, sz, u32, vp, vp, vp, u32, u64, u32, vp, vp, sz, vp, vp]
     L.co3_decode.argtypes = [vp, sz, vp, vp, vp, u32, u64, u32, vp, vp, vp, sz, vp, vp]
-    for name in ("co3_workspace_bytes", "co3_stream_capacity_bytes", "co3_convert", "co3_code_build", "co3_encode",
+    L.co3_profile_enable.argtypes = [C.c_int]
+    L.co3_profile_read.argtypes = [vp, vp]
+    for name in ("co3_profile_enable", "co3_profile_read", "co3_workspace_bytes", "co3_stream_capacity_bytes", "co3_convert", "co3_code_build", "co3_encode",
                  "co3_encode_symbols", "co3_decode_aggregate", "co3_decode"):
         getattr(L, name).restype = C.c_int
     _lib = L
@@ -173,3 +175,20 @@ def co3_decode(stream_in, stream_bytes, fmts, codes, segs, n_seg, n_elem, ghat_o
     return _load().co3_decode(_dev(stream_in), stream_bytes, _dev(fmts), _dev(codes), _dev(segs), n_seg, n_elem,
                               chunk_syms, _dev(ghat_out, True), _dev(sym_out, True), _dev(workspace),
                               workspace.numel() * workspace.element_size(), _dev(res), _stream(stream))
+
+
+KERNEL_NAMES = ("prepare", "convert", "pack", "scan", "compact", "check", "decode")
+
+
+def co3_profile_enable(on: bool) -> int:
+    return _load().co3_profile_enable(1 if on else 0)
+
+
+def co3_profile_read() -> dict:
+    """{kernel name: (launches, total ms)} since profiling was enabled or last read (synchronises)."""
+    ms = np.zeros(len(KERNEL_NAMES), dtype=np.float64)
+    n = np.zeros(len(KERNEL_NAMES), dtype=np.uint32)
+    st = _load().co3_profile_read(ms.ctypes.data, n.ctypes.data)
+    if st != OK:
+        raise RuntimeError("co3_profile_read: " + co3_status_string(st))
+    return {k: (int(n[i]), float(ms[i])) for i, k in enumerate(KERNEL_NAMES)}

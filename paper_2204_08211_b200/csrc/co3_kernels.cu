@@ -908,12 +908,47 @@ uint64_t fixed_part_bound(uint32_t n_seg, uint64_t n_chunks_max) {
     return o;
 }
 
-bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
-
 #define CO3_CUDA(call)                                  \
     do {                                                \
         if ((call) != cudaSuccess) return CO3_ERR_CUDA; \
     } while (0)
+
+bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+
+// Optional per-kernel timing (off by default): an event pair around every launch, read back by
+// co3_profile_read.  Used by benchmarks to time the kernels inside the entry points.
+struct Profiler {
+    static constexpr int kMaxRecords = 16384;
+    bool on = false;
+    int n = 0;
+    int ids[kMaxRecords];
+    cudaEvent_t ev[kMaxRecords][2];
+    int n_created = 0;
+    void begin(int id, cudaStream_t st) {
+        if (!on || n >= kMaxRecords) return;
+        if (n >= n_created) {
+            if (cudaEventCreate(&ev[n][0]) != cudaSuccess || cudaEventCreate(&ev[n][1]) != cudaSuccess) { on = false; return; }
+            ++n_created;
+        }
+        ids[n] = id;
+        cudaEventRecord(ev[n][0], st);
+    }
+    void end(cudaStream_t st) {
+        if (!on || n >= kMaxRecords) return;
+        cudaEventRecord(ev[n][1], st);
+        ++n;
+    }
+};
+Profiler g_prof;
+
+#define CO3_LAUNCH(id, st, ...)        \
+    do {                               \
+        g_prof.begin(id, st);          \
+        __VA_ARGS__;                   \
+        g_prof.end(st);                \
+        CO3_CUDA(cudaGetLastError());  \
+    } while (0)
+
 
 int begin_call(const WsLayout& L, const Ws& ws, co3_result* res, uint32_t n_res, cudaStream_t st,
                const co3_fmt* fmts, const co3_code* codes, const co3_seg* segs, uint32_t n_seg, uint64_t n_elem,
@@ -922,8 +957,7 @@ int begin_call(const WsLayout& L, const Ws& ws, co3_result* res, uint32_t n_res,
     CO3_CUDA(cudaMemsetAsync(res, 0, sizeof(co3_result) * (size_t)n_res, st));
     CO3_CUDA(cudaMemsetAsync(ws.client_fail, 0, 4 * (size_t)(n_fail ? n_fail : 1), st));
     PrepArgs pa{fmts, codes, segs, n_seg, n_elem, tile_chunks, res, n_res, ws};
-    prepare_kernel<<<n_seg ? n_seg : 1, kThreads, 0, st>>>(pa);
-    CO3_CUDA(cudaGetLastError());
+    CO3_LAUNCH(CO3_KERNEL_PREPARE, st, prepare_kernel<<<n_seg ? n_seg : 1, kThreads, 0, st>>>(pa));
     (void)L;
     return CO3_OK;
 }
@@ -933,8 +967,7 @@ int launch_decode(const DecArgs& da, uint32_t n_tiles_max, cudaStream_t st) {
     const size_t smem = sizeof(DecSmem<B, G>);
     CO3_CUDA(cudaFuncSetAttribute(decode_kernel<B, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     if (n_tiles_max == 0) return CO3_OK;
-    decode_kernel<B, G><<<n_tiles_max, 16 * B * G, smem, st>>>(da);
-    CO3_CUDA(cudaGetLastError());
+    CO3_LAUNCH(CO3_KERNEL_DECODE, st, decode_kernel<B, G><<<n_tiles_max, 16 * B * G, smem, st>>>(da));
     return CO3_OK;
 }
 
@@ -960,8 +993,7 @@ int decode_common(const uint8_t* const* streams, const uint8_t* single, size_t s
     const int rc = begin_call(L, ws, res, 1, st, fmts, codes, segs, n_seg, n_elem, (uint32_t)G, 1);
     if (rc != CO3_OK) return rc;
     DecArgs da{streams, single, stream_bytes, n_clients, segs, n_seg, n_elem, out, sym_out, res, ws};
-    check_streams_kernel<<<n_clients, kThreads, 0, st>>>(da);
-    CO3_CUDA(cudaGetLastError());
+    CO3_LAUNCH(CO3_KERNEL_CHECK, st, check_streams_kernel<<<n_clients, kThreads, 0, st>>>(da));
     const uint32_t tiles = (uint32_t)(chunks / G + n_seg);  // upper bound; surplus blocks return at once
 #define CO3_DEC_CASE(b, g) \
     if (B == b && G == g) return launch_decode<b, g>(da, tiles, st);
@@ -993,16 +1025,13 @@ int encode_common(const float* grad, float* mem, float decay, const uint8_t* sym
     if (L.n_chunks_max) {
         PackArgs pa{grad, mem, decay, sym, segs, n_seg, client_stride, streams_out, stream_capacity, res, ws};
         const dim3 grid(L.n_chunks_max, n_clients);
-        if (sym) pack_kernel<true><<<grid, kThreads, 0, st>>>(pa);
-        else pack_kernel<false><<<grid, kThreads, 0, st>>>(pa);
-        CO3_CUDA(cudaGetLastError());
+        if (sym) CO3_LAUNCH(CO3_KERNEL_PACK, st, pack_kernel<true><<<grid, kThreads, 0, st>>>(pa));
+        else CO3_LAUNCH(CO3_KERNEL_PACK, st, pack_kernel<false><<<grid, kThreads, 0, st>>>(pa));
     }
     ScanArgs sa{segs, n_seg, n_elem, streams_out, stream_capacity, res, ws};
-    scan_kernel<<<n_clients, kScanThreads, 0, st>>>(sa);
-    CO3_CUDA(cudaGetLastError());
+    CO3_LAUNCH(CO3_KERNEL_SCAN, st, scan_kernel<<<n_clients, kScanThreads, 0, st>>>(sa));
     if (L.n_chunks_max) {
-        compact_kernel<<<dim3(L.n_chunks_max, n_clients), kThreads, 0, st>>>(sa);
-        CO3_CUDA(cudaGetLastError());
+        CO3_LAUNCH(CO3_KERNEL_COMPACT, st, compact_kernel<<<dim3(L.n_chunks_max, n_clients), kThreads, 0, st>>>(sa));
     }
     return CO3_OK;
 }
@@ -1022,6 +1051,26 @@ const char* co3_status_string(int status) {
         case CO3_ERR_CUDA: return "CUDA runtime error";
         default: return "unknown status";
     }
+}
+
+int co3_profile_enable(int on) {
+    g_prof.n = 0;
+    g_prof.on = on != 0;
+    return CO3_OK;
+}
+
+int co3_profile_read(double* total_ms, uint32_t* launches) {
+    if (!total_ms || !launches) return CO3_ERR_INVALID_ARG;
+    for (int i = 0; i < CO3_KERNEL_COUNT; ++i) { total_ms[i] = 0.0; launches[i] = 0; }
+    for (int r = 0; r < g_prof.n; ++r) {
+        float ms = 0.0f;
+        CO3_CUDA(cudaEventSynchronize(g_prof.ev[r][1]));
+        CO3_CUDA(cudaEventElapsedTime(&ms, g_prof.ev[r][0], g_prof.ev[r][1]));
+        total_ms[g_prof.ids[r]] += ms;
+        launches[g_prof.ids[r]] += 1;
+    }
+    g_prof.n = 0;
+    return CO3_OK;
 }
 
 int co3_workspace_bytes(uint64_t n_elem, uint32_t n_seg, uint32_t n_clients, uint32_t chunk_syms, size_t* out) {
@@ -1062,11 +1111,10 @@ int co3_convert(const float* grad, float* mem, float decay, const co3_fmt* fmts,
     if (L.n_chunks_max == 0) return CO3_OK;
     ConvertArgs ca{grad, mem, decay, segs, n_seg, client_stride_elems, sym_out, hist_out, res, ws};
     const dim3 grid(L.n_chunks_max, n_clients);
-    if (sym_out && hist_out) convert_kernel<true, true><<<grid, kThreads, 0, st>>>(ca);
-    else if (sym_out) convert_kernel<true, false><<<grid, kThreads, 0, st>>>(ca);
-    else if (hist_out) convert_kernel<false, true><<<grid, kThreads, 0, st>>>(ca);
-    else convert_kernel<false, false><<<grid, kThreads, 0, st>>>(ca);
-    CO3_CUDA(cudaGetLastError());
+    if (sym_out && hist_out) CO3_LAUNCH(CO3_KERNEL_CONVERT, st, convert_kernel<true, true><<<grid, kThreads, 0, st>>>(ca));
+    else if (sym_out) CO3_LAUNCH(CO3_KERNEL_CONVERT, st, convert_kernel<true, false><<<grid, kThreads, 0, st>>>(ca));
+    else if (hist_out) CO3_LAUNCH(CO3_KERNEL_CONVERT, st, convert_kernel<false, true><<<grid, kThreads, 0, st>>>(ca));
+    else CO3_LAUNCH(CO3_KERNEL_CONVERT, st, convert_kernel<false, false><<<grid, kThreads, 0, st>>>(ca));
     return CO3_OK;
 }
 
