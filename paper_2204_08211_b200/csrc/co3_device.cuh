@@ -15,7 +15,12 @@ constexpr int kSubs = kC / kS;                               // 16
 constexpr int kSlotWords = kC * CO3_MAX_CODE_LEN / 32;       // worst-case words of one chunk
 constexpr int kDecBits = 12;                                 // decode LUT is indexed by 12 stream bits
 constexpr int kDecLut = 1 << kDecBits;
-constexpr int kLongStride = 260;                             // u32 per segment: count + up to 256 long codewords
+constexpr int kSubBits = CO3_MAX_CODE_LEN - kDecBits;        // second-level tables are indexed by the next 4 bits
+constexpr int kSubLut = 256 << kSubBits;                     // at most 256 second-level tables per segment
+constexpr uint32_t kEncMissing = 0x80000000u;                // encode table entry of a symbol without codeword
+constexpr uint32_t kDecLong = 0x8000u;                       // decode table entry: look in a second-level table
+constexpr uint32_t kDecInvalid = 0x4100u;                    // decode table entry: no codeword (consumes one bit)
+constexpr uint32_t kDecErrBit = 0x4000u;
 constexpr uint32_t kMagic = 0x53334F43u;                     // 'C','O','3','S'
 constexpr uint32_t kHeaderBytes = 64;
 constexpr int kThreads = 256;
@@ -29,14 +34,32 @@ struct Ctrl {
     uint64_t chunk_off, sub_off, payload_off;  // byte offsets of the container sections
 };
 
+// Where a chunk lives: written by the prepare kernel, read by every kernel that works per chunk.
+struct ChunkDesc {
+    uint32_t seg;    // segment (layer) of the chunk
+    uint32_t cnt;    // symbols in the chunk (kC except for the last chunk of a segment)
+    uint64_t elem0;  // index of its first element inside a client's vector
+};
+
+// A decode tile: up to `tile_chunks` consecutive chunks of one segment.
+struct TileDesc {
+    uint32_t seg;
+    uint32_t chunk0;
+    uint32_t n_chunks;
+    uint32_t pad;
+};
+
 // Converter constants of one segment, derived from co3_fmt by the prepare kernel.
 struct FmtDev {
     uint32_t mant_bits;        // M
     uint32_t mag_bits;         // E + M
+    uint32_t fast;             // 1: M >= 1 and sub-normal levels kept, the branch-free converter applies
+    uint32_t drop;             // 23 - M: fp32 mantissa bits below the format's
     uint32_t min_normal_bits;  // fp32 pattern of 2^emin
     uint32_t code_bias;        // (emin + 126) << M : fp32 (exp|mant>>drop) minus this is the magnitude code
     uint32_t max_code;         // largest magnitude code
     uint32_t top_bits;         // fp32 pattern of the largest level
+    uint32_t sign_shift;       // 31 - (E + M): moves the fp32 sign bit to the symbol's sign bit
     uint32_t flush;            // 1: no sub-normal levels
     uint32_t half_min_bits;    // fp32 pattern of 2^(emin-1)
     float magic;               // 2^(emin - M + 23): adding it rounds to a multiple of the sub-normal step
@@ -47,11 +70,13 @@ struct FmtDev {
 struct Ws {
     Ctrl* ctrl;
     uint32_t* first_chunk;  // [n_seg + 1]
-    uint32_t* first_tile;   // [n_seg + 1]
+    ChunkDesc* chunk_desc;  // [n_chunks_max]
+    TileDesc* tile_desc;    // [n_chunks_max]
     FmtDev* fmt;            // [n_seg]
-    uint32_t* enc_lut;      // [n_seg][256]   bits << 8 | len
-    uint16_t* dec_lut;      // [n_seg][4096]  len << 8 | sym ; len 0 = no codeword, 255 = longer than 12 bits
-    uint32_t* dec_long;     // [n_seg][kLongStride]  [0] = count, then bits << 16 | len << 8 | sym
+    uint32_t* enc_lut;      // [n_seg][256]   bits << 8 | len ; kEncMissing for a symbol without codeword
+    uint16_t* dec_lut;      // [n_seg][4096]  len << 8 | sym ; kDecInvalid where no codeword matches;
+                            //                kDecLong | index of a second-level table for longer codewords
+    uint16_t* dec_sub;      // [n_seg][256][16]  len << 8 | sym for codewords of 13..16 bits, by their bits 13..16
     float* val_lut;         // [n_seg][256]   reconstructed value of each symbol
     uint32_t* client_fail;  // [n_clients]
     uint32_t* chunk_bits;   // [n_clients][n_chunks_max]
@@ -115,6 +140,32 @@ __device__ __forceinline__ float convert_one(float g, float m, float decay, cons
         if (vb > 0x7f800000u) { code = 0u; sign = 0u; }
     }
     sym = (sign << f.mag_bits) | code;
+    return m_new;
+}
+
+// The same update without branches, for formats with M >= 1 that keep the sub-normal levels.
+// Rounding by one fp32 addition: with ae the (clamped) exponent of |t|, |t| + 2^(ae + 23 - M) is rounded by
+// the adder to a multiple of the format's step in that binade, ties to the even multiple, which has the
+// even code when M >= 1.  Saturation and non-finite inputs are only detected here (a_max > top_bits,
+// nf_acc != nf_acc); the caller then repeats the element group with convert_one, which also counts them.
+__device__ __forceinline__ float convert_fast(float g, float m, float decay, const FmtDev& f, uint32_t& sym,
+                                              uint32_t& a_max, float& nf_acc) {
+    const float v = __fmaf_rn(decay, m, g);
+    const float t = __fmul_rn(v, f.scale);
+    const uint32_t tb = __float_as_uint(t);
+    const uint32_t a = tb & 0x7fffffffu;
+    const uint32_t ac = min(a, f.top_bits);
+    a_max = max(a_max, a);  // beyond f.top_bits iff some input saturated
+    const uint32_t ae = max(ac & 0x7f800000u, f.min_normal_bits);
+    const uint32_t mg = ae + (f.drop << 23);
+    const float s = __fadd_rn(__uint_as_float(ac), __uint_as_float(mg));
+    const uint32_t code = ((ae - f.min_normal_bits) >> f.drop) + (__float_as_uint(s) - mg);
+    const float qmag = __fsub_rn(s, __uint_as_float(mg));
+    const uint32_t sgn = code ? (tb & 0x80000000u) : 0u;
+    sym = code | (sgn >> f.sign_shift);
+    const float ghat = __fmul_rn(__uint_as_float(__float_as_uint(qmag) | sgn), f.inv_scale);
+    const float m_new = __fsub_rn(v, ghat);
+    nf_acc = __fmaf_rn(m_new, 0.0f, nf_acc);  // NaN iff some m_new is not finite, i.e. some v was not
     return m_new;
 }
 

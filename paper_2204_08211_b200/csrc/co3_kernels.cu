@@ -8,6 +8,7 @@
 //   check_streams_kernel  header / table validation before decoding
 //   decode_kernel         chunk-indexed prefix-code decoder fused with the ordered cross-client sum
 #include <cuda_runtime.h>
+#include <stddef.h>
 #include <stdint.h>
 
 #include "co3.h"
@@ -16,7 +17,8 @@
 namespace co3 {
 
 // ------------------------------------------------------------------------------------------------
-// prepare: one block per segment builds that segment's tables; block 0 also lays out the chunks.
+// prepare: one block per segment validates that segment's descriptors, finds its place by a block
+// reduction over the segments before it, writes its chunk and tile descriptors and builds its tables.
 // ------------------------------------------------------------------------------------------------
 struct PrepArgs {
     const co3_fmt* fmts;    // nullable (encode from symbols)
@@ -35,65 +37,94 @@ __device__ void fail_all(const PrepArgs& a, int code) {
     for (uint32_t u = 0; u < a.n_res; ++u) set_status(&a.res[u], code);
 }
 
+__device__ __forceinline__ uint64_t block_sum_u64(uint64_t x, uint64_t* scratch /* [8] */) {
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) x += __shfl_xor_sync(0xffffffffu, x, d);
+    __syncthreads();
+    if ((threadIdx.x & 31u) == 0) scratch[threadIdx.x >> 5] = x;
+    __syncthreads();
+    uint64_t sum = 0;
+#pragma unroll
+    for (int w = 0; w < kThreads / 32; ++w) sum += scratch[w];
+    return sum;
+}
+
 __global__ void __launch_bounds__(kThreads) prepare_kernel(PrepArgs a) {
-    __shared__ uint32_t s_part[kThreads][2];
+    __shared__ uint64_t s_red[8];
     __shared__ uint32_t s_kraft;
-    __shared__ uint32_t s_nlong;
+    __shared__ uint32_t s_scan[8];
     const uint32_t tid = threadIdx.x;
     const uint32_t k = blockIdx.x;
+    const uint32_t G = a.tile_chunks;
 
-    if (k == 0) {
+    if (k == 0)
         for (uint32_t u = tid; u < a.n_res; u += kThreads) a.res[u].first_bad_chunk = 0xffffffffu;
-        // chunk and tile layout: exclusive scans over the segments, kThreads contiguous ranges
-        const uint32_t per = (a.n_seg + kThreads - 1) / kThreads;
-        const uint32_t lo = min(tid * per, a.n_seg), hi = min(lo + per, a.n_seg);
-        uint32_t nc = 0, nt = 0;
-        bool bad = false;
-        for (uint32_t i = lo; i < hi; ++i) {
-            const uint64_t n = a.segs[i].n_elem;
-            if (n > a.n_elem) bad = true;
-            const uint32_t c = (uint32_t)((n + kC - 1) / kC);
-            nc += c;
-            nt += (c + a.tile_chunks - 1) / a.tile_chunks;
-        }
-        s_part[tid][0] = nc;
-        s_part[tid][1] = nt;
-        __syncthreads();
-        uint32_t bc = 0, bt = 0;
-        for (uint32_t i = 0; i < tid; ++i) { bc += s_part[i][0]; bt += s_part[i][1]; }
-        // segments must be contiguous, in order, and cover n_elem
-        uint64_t expect_off = (lo < a.n_seg) ? a.segs[lo].elem_off : 0;
-        for (uint32_t i = lo; i < hi; ++i) {
-            const co3_seg sg = a.segs[i];
-            if (sg.elem_off != expect_off) bad = true;
-            expect_off = sg.elem_off + sg.n_elem;
-            a.ws.first_chunk[i] = bc;
-            a.ws.first_tile[i] = bt;
-            const uint32_t c = (uint32_t)((sg.n_elem + kC - 1) / kC);
-            bc += c;
-            bt += (c + a.tile_chunks - 1) / a.tile_chunks;
-        }
-        if (lo < hi) {
-            if (lo == 0 && a.segs[0].elem_off != 0) bad = true;
-            const uint64_t next_off = (hi < a.n_seg) ? a.segs[hi].elem_off : a.n_elem;
-            if (expect_off != next_off) bad = true;
-        }
-        if (a.n_seg == 0 && tid == 0 && a.n_elem != 0) bad = true;
-        if (bc > a.ws.n_chunks_max) bad = true;
-        const bool owner = (a.n_seg == 0) ? (tid == 0) : (lo < hi && hi == a.n_seg);  // owns the end of the table
-        if (owner) {
-            a.ws.first_chunk[a.n_seg] = bc;
-            a.ws.first_tile[a.n_seg] = bt;
-            Ctrl* c = a.ws.ctrl;
-            c->n_chunks = bc;
-            c->n_tiles = bt;
-            c->chunk_off = align16(kHeaderBytes + 24ull * a.n_seg);
-            c->sub_off = align16(c->chunk_off + 8ull * (bc + 1ull));
-            c->payload_off = align16(c->sub_off + 2ull * bc * kSubs);
-        }
-        if (bad) fail_all(a, CO3_ERR_INVALID_ARG);
+
+    // ---- layout: elements, chunks and tiles of the segments before this one
+    uint64_t e_before = 0, c_before = 0, t_before = 0;
+    bool bad = false;
+    for (uint32_t i = tid; i < k && i < a.n_seg; i += kThreads) {
+        const uint64_t n = a.segs[i].n_elem;
+        if (n > a.n_elem) bad = true;
+        const uint64_t c = (n + kC - 1) / kC;
+        e_before += n;
+        c_before += c;
+        t_before += (c + G - 1) / G;
     }
-    if (k >= a.n_seg) return;
+    e_before = block_sum_u64(e_before, s_red);
+    c_before = block_sum_u64(c_before, s_red);
+    t_before = block_sum_u64(t_before, s_red);
+    bad = __syncthreads_or(bad);
+    if (a.n_seg == 0) {
+        if (tid == 0) {
+            Ctrl* c = a.ws.ctrl;
+            c->n_chunks = 0;
+            c->n_tiles = 0;
+            c->chunk_off = align16(kHeaderBytes);
+            c->sub_off = align16(c->chunk_off + 8ull);
+            c->payload_off = c->sub_off;
+            a.ws.first_chunk[0] = 0;
+            if (a.n_elem != 0) fail_all(a, CO3_ERR_INVALID_ARG);
+        }
+        return;
+    }
+    const co3_seg sg = a.segs[k];
+    const uint64_t my_chunks = sg.n_elem <= a.n_elem ? (sg.n_elem + kC - 1) / kC : 0;
+    const uint64_t my_tiles = (my_chunks + G - 1) / G;
+    if (sg.n_elem > a.n_elem || sg.elem_off != e_before || c_before + my_chunks > a.ws.n_chunks_max) bad = true;
+    if (k == a.n_seg - 1 && e_before + sg.n_elem != a.n_elem) bad = true;
+    if (bad) {
+        if (tid == 0) fail_all(a, CO3_ERR_INVALID_ARG);
+        return;
+    }
+    if (tid == 0) {
+        a.ws.first_chunk[k] = (uint32_t)c_before;
+        if (k == a.n_seg - 1) {
+            const uint64_t nc = c_before + my_chunks;
+            a.ws.first_chunk[a.n_seg] = (uint32_t)nc;
+            Ctrl* c = a.ws.ctrl;
+            c->n_chunks = (uint32_t)nc;
+            c->n_tiles = (uint32_t)(t_before + my_tiles);
+            c->chunk_off = align16(kHeaderBytes + 24ull * a.n_seg);
+            c->sub_off = align16(c->chunk_off + 8ull * (nc + 1ull));
+            c->payload_off = align16(c->sub_off + 2ull * nc * kSubs);
+        }
+    }
+    for (uint64_t c = tid; c < my_chunks; c += kThreads) {
+        ChunkDesc d;
+        d.seg = k;
+        d.cnt = (uint32_t)min((uint64_t)kC, sg.n_elem - c * kC);
+        d.elem0 = sg.elem_off + c * kC;
+        a.ws.chunk_desc[c_before + c] = d;
+    }
+    for (uint64_t t = tid; t < my_tiles; t += kThreads) {
+        TileDesc d;
+        d.seg = k;
+        d.chunk0 = (uint32_t)(c_before + t * G);
+        d.n_chunks = (uint32_t)min((uint64_t)G, my_chunks - t * G);
+        d.pad = 0;
+        a.ws.tile_desc[t_before + t] = d;
+    }
 
     // ---- format constants and value table
     bool fmt_ok = true;
@@ -107,16 +138,19 @@ __global__ void __launch_bounds__(kThreads) prepare_kernel(PrepArgs a) {
         if (fmt_ok) {
             fd.mant_bits = M;
             fd.mag_bits = E + M;
+            fd.drop = 23u - M;
+            fd.sign_shift = 31u - (E + M);
             fd.min_normal_bits = (uint32_t)(emin + 127) << 23;
             fd.code_bias = (uint32_t)(emin + 126) << M;
             fd.max_code = (((1u << E) - 2u) << M) | ((1u << M) - 1u);
             fd.top_bits = (fd.max_code + fd.code_bias) << (23u - M);
             fd.flush = (f.flags & CO3_FMT_FLUSH_SUBNORMALS) ? 1u : 0u;
+            fd.fast = (M >= 1 && !fd.flush) ? 1u : 0u;
             fd.half_min_bits = (uint32_t)(emin - 1 + 127) << 23;
             fd.magic = __uint_as_float((uint32_t)(emin - (int)M + 23 + 127) << 23);
             fd.scale = f.scale;
             fd.inv_scale = f.inv_scale;
-            const float top = __fmul_rn(__uint_as_float((fd.max_code + fd.code_bias) << (23u - M)), f.inv_scale);
+            const float top = __fmul_rn(__uint_as_float(fd.top_bits), f.inv_scale);
             if (isinf(top)) fmt_ok = false;
         }
         if (fmt_ok) {
@@ -145,13 +179,15 @@ __global__ void __launch_bounds__(kThreads) prepare_kernel(PrepArgs a) {
     bool code_ok = true;
     if (a.codes) {
         const uint32_t len = a.codes[k].len[tid], bits = a.codes[k].bits[tid];
-        if (tid == 0) { s_kraft = 0; s_nlong = 0; }
+        if (tid == 0) s_kraft = 0;
         __syncthreads();
         if (len > CO3_MAX_CODE_LEN || (len && (bits >> len))) code_ok = false;
         if (code_ok && len) atomicAdd(&s_kraft, 1u << (CO3_MAX_CODE_LEN - len));
-        a.ws.enc_lut[k * 256 + tid] = code_ok ? ((bits << 8) | len) : 0u;
+        a.ws.enc_lut[k * 256 + tid] = (code_ok && len) ? ((bits << 8) | len) : kEncMissing;
         uint16_t* lut = a.ws.dec_lut + (size_t)k * kDecLut;
-        for (uint32_t i = tid; i < (uint32_t)kDecLut; i += kThreads) lut[i] = 0;
+        uint16_t* sub = a.ws.dec_sub + (size_t)k * kSubLut;
+        for (uint32_t i = tid; i < (uint32_t)kDecLut; i += kThreads) lut[i] = (uint16_t)kDecInvalid;
+        for (uint32_t i = tid; i < (uint32_t)kSubLut; i += kThreads) sub[i] = (uint16_t)kDecInvalid;
         __syncthreads();
         if (s_kraft > (1u << CO3_MAX_CODE_LEN)) code_ok = false;  // over-subscribed: cannot be prefix-free
         code_ok = __syncthreads_and(code_ok);
@@ -163,13 +199,27 @@ __global__ void __launch_bounds__(kThreads) prepare_kernel(PrepArgs a) {
                 const uint32_t span = 1u << (kDecBits - l), first = b << (kDecBits - l);
                 for (uint32_t i = tid & 31u; i < span; i += 32) lut[first + i] = (uint16_t)((l << 8) | sym);
             }
-            if (len > (uint32_t)kDecBits) {
-                lut[bits >> (len - kDecBits)] = (uint16_t)(255u << 8);
-                const uint32_t slot = atomicAdd(&s_nlong, 1u);
-                a.ws.dec_long[k * kLongStride + 1 + slot] = (bits << 16) | (len << 8) | tid;
-            }
+            // longer codewords: mark their 12-bit prefix, number the marked prefixes, fill one 16-entry
+            // second-level table per prefix
+            const bool is_long = len > (uint32_t)kDecBits;
+            const uint32_t prefix = is_long ? (bits >> (len - kDecBits)) : 0u;
+            if (is_long) lut[prefix] = (uint16_t)kDecLong;
             __syncthreads();
-            if (tid == 0) a.ws.dec_long[k * kLongStride] = s_nlong;
+            const uint32_t per = kDecLut / kThreads;
+            uint32_t marked = 0;
+            for (uint32_t i = 0; i < per; ++i) marked += (lut[tid * per + i] == kDecLong) ? 1u : 0u;
+            uint32_t total;
+            uint32_t idx = block_exclusive_scan_256(marked, s_scan, &total);
+            for (uint32_t i = 0; i < per; ++i)
+                if (lut[tid * per + i] == kDecLong) lut[tid * per + i] = (uint16_t)(kDecLong | (idx++ & 0xffu));
+            __syncthreads();
+            if (is_long) {
+                const uint32_t t = lut[prefix] & 0xffu;
+                const uint32_t rest = len - kDecBits;  // 1..4 bits beyond the prefix
+                const uint32_t first = (bits & ((1u << rest) - 1u)) << (kSubBits - rest);
+                for (uint32_t i = 0; i < (1u << (kSubBits - rest)); ++i)
+                    sub[t * (1u << kSubBits) + first + i] = (uint16_t)((len << 8) | tid);
+            }
         }
     }
     if ((!fmt_ok || !code_ok) && tid == 0) fail_all(a, CO3_ERR_INVALID_ARG);
@@ -178,68 +228,34 @@ __global__ void __launch_bounds__(kThreads) prepare_kernel(PrepArgs a) {
 // ------------------------------------------------------------------------------------------------
 // Element access for one thread: 8 consecutive elements of a chunk.
 // ------------------------------------------------------------------------------------------------
-struct ChunkPos {
-    uint32_t seg;
-    uint32_t cnt;    // symbols in this chunk
-    uint64_t elem0;  // index of the chunk's first element inside the client's vector
-};
-
-__device__ __forceinline__ ChunkPos locate_chunk(const Ws& ws, const co3_seg* __restrict__ segs, uint32_t n_seg,
-                                                 uint32_t chunk) {
-    ChunkPos p;
-    p.seg = find_seg(ws.first_chunk, n_seg, chunk);
-    const co3_seg sg = segs[p.seg];
-    const uint64_t start = (uint64_t)(chunk - ws.first_chunk[p.seg]) * kC;
-    p.cnt = (uint32_t)min((uint64_t)kC, sg.n_elem - start);
-    p.elem0 = sg.elem_off + start;
-    return p;
+__device__ __forceinline__ void load8_vec(const float* __restrict__ p, float (&x)[8]) {
+    const float4 a = __ldg(reinterpret_cast<const float4*>(p));
+    const float4 b = __ldg(reinterpret_cast<const float4*>(p) + 1);
+    x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w;
+    x[4] = b.x; x[5] = b.y; x[6] = b.z; x[7] = b.w;
 }
 
-__device__ __forceinline__ void load8(const float* __restrict__ p, uint32_t n_valid, float (&x)[8]) {
-    if (n_valid == 8 && (reinterpret_cast<uintptr_t>(p) & 15u) == 0) {
-        const float4 a = __ldg(reinterpret_cast<const float4*>(p));
-        const float4 b = __ldg(reinterpret_cast<const float4*>(p) + 1);
-        x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w;
-        x[4] = b.x; x[5] = b.y; x[6] = b.z; x[7] = b.w;
-    } else {
-#pragma unroll
-        for (int j = 0; j < 8; ++j) x[j] = (uint32_t)j < n_valid ? p[j] : 0.0f;
-    }
+__device__ __forceinline__ void store8_vec(float* __restrict__ p, const float (&x)[8]) {
+    reinterpret_cast<float4*>(p)[0] = make_float4(x[0], x[1], x[2], x[3]);
+    reinterpret_cast<float4*>(p)[1] = make_float4(x[4], x[5], x[6], x[7]);
 }
 
-__device__ __forceinline__ void store8(float* __restrict__ p, uint32_t n_valid, const float (&x)[8]) {
-    if (n_valid == 8 && (reinterpret_cast<uintptr_t>(p) & 15u) == 0) {
-        reinterpret_cast<float4*>(p)[0] = make_float4(x[0], x[1], x[2], x[3]);
-        reinterpret_cast<float4*>(p)[1] = make_float4(x[4], x[5], x[6], x[7]);
-    } else {
+__device__ __forceinline__ void load8_any(const float* __restrict__ p, uint32_t n_valid, float (&x)[8]) {
 #pragma unroll
-        for (int j = 0; j < 8; ++j)
-            if ((uint32_t)j < n_valid) p[j] = x[j];
-    }
+    for (int j = 0; j < 8; ++j) x[j] = (uint32_t)j < n_valid ? p[j] : 0.0f;
 }
 
-__device__ __forceinline__ void store_sym8(uint8_t* __restrict__ p, uint32_t n_valid, const uint32_t (&s)[8]) {
-    if (n_valid == 8 && (reinterpret_cast<uintptr_t>(p) & 7u) == 0) {
-        uint2 w;
-        w.x = s[0] | (s[1] << 8) | (s[2] << 16) | (s[3] << 24);
-        w.y = s[4] | (s[5] << 8) | (s[6] << 16) | (s[7] << 24);
-        *reinterpret_cast<uint2*>(p) = w;
-    } else {
+__device__ __forceinline__ void store8_any(float* __restrict__ p, uint32_t n_valid, const float (&x)[8]) {
 #pragma unroll
-        for (int j = 0; j < 8; ++j)
-            if ((uint32_t)j < n_valid) p[j] = (uint8_t)s[j];
-    }
+    for (int j = 0; j < 8; ++j)
+        if ((uint32_t)j < n_valid) p[j] = x[j];
 }
 
-__device__ __forceinline__ void load_sym8(const uint8_t* __restrict__ p, uint32_t n_valid, uint32_t (&s)[8]) {
-    if (n_valid == 8 && (reinterpret_cast<uintptr_t>(p) & 7u) == 0) {
-        const uint2 w = __ldg(reinterpret_cast<const uint2*>(p));
-#pragma unroll
-        for (int j = 0; j < 4; ++j) { s[j] = (w.x >> (8 * j)) & 0xffu; s[4 + j] = (w.y >> (8 * j)) & 0xffu; }
-    } else {
-#pragma unroll
-        for (int j = 0; j < 8; ++j) s[j] = (uint32_t)j < n_valid ? p[j] : 0u;
-    }
+__device__ __forceinline__ uint2 pack_sym8(const uint32_t (&s)[8]) {
+    uint2 w;
+    w.x = __byte_perm(__byte_perm(s[0], s[1], 0x0040), __byte_perm(s[2], s[3], 0x0040), 0x5410);
+    w.y = __byte_perm(__byte_perm(s[4], s[5], 0x0040), __byte_perm(s[6], s[7], 0x0040), 0x5410);
+    return w;
 }
 
 // Adds the saturated / non-finite counts of a warp to the client's result.
@@ -260,6 +276,35 @@ __device__ __forceinline__ void add_counts(co3_result* r, uint32_t n_sat, uint32
     }
 }
 
+// Correct + convert + memory update of this thread's 8 elements (Algorithm 1, client side).
+// kFull: the chunk is complete and 16-byte aligned, so the group is read and written as two float4.
+// Symbols land in s[]; the new memory is stored; counters accumulate in n_sat / n_nf.
+template <bool kFull>
+__device__ __forceinline__ void convert8(const float* __restrict__ gp, float* __restrict__ mp, uint32_t nv, float decay,
+                                         const FmtDev& f, uint32_t (&s)[8], uint32_t& n_sat, uint32_t& n_nf) {
+    float g[8], m[8], mo[8];
+    if (kFull) { load8_vec(gp, g); load8_vec(mp, m); }
+    else { load8_any(gp, nv, g); load8_any(mp, nv, m); }
+    bool redo = true;
+    if (kFull && f.fast) {
+        uint32_t a_max = 0;
+        float nf_acc = 0.0f;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) mo[j] = convert_fast(g[j], m[j], decay, f, s[j], a_max, nf_acc);
+        redo = (a_max > f.top_bits) || (nf_acc != nf_acc);
+    }
+    if (redo) {  // generic formats, ragged groups, and groups that hold a saturating or non-finite input
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            uint32_t fl = 0;
+            mo[j] = convert_one(g[j], m[j], decay, f, s[j], fl);
+            if ((uint32_t)j < nv) { n_sat += fl & 1u; n_nf += fl >> 1; }
+        }
+    }
+    if (kFull) store8_vec(mp, mo);
+    else store8_any(mp, nv, mo);
+}
+
 // ------------------------------------------------------------------------------------------------
 // convert: one block per (chunk, client)
 // ------------------------------------------------------------------------------------------------
@@ -267,8 +312,6 @@ struct ConvertArgs {
     const float* grad;
     float* mem;
     float decay;
-    const co3_seg* segs;
-    uint32_t n_seg;
     uint64_t client_stride;
     uint8_t* sym_out;    // nullable
     uint64_t* hist_out;  // nullable
@@ -276,47 +319,54 @@ struct ConvertArgs {
     Ws ws;
 };
 
+constexpr int kHistCopies = 8;    // private histograms per block, spread over the lanes
+constexpr int kHistStride = 260;  // words between copies: shifts each copy by four banks
+
 template <bool kSym, bool kHist>
 __global__ void __launch_bounds__(kThreads) convert_kernel(ConvertArgs a) {
-    __shared__ uint32_t s_hist[256];
+    __shared__ uint32_t s_hist[kHist ? kHistStride * kHistCopies : 1];
     const Ctrl* ctrl = a.ws.ctrl;
     if (ctrl->abort) return;
     const uint32_t chunk = blockIdx.x, u = blockIdx.y, tid = threadIdx.x;
     if (chunk >= ctrl->n_chunks) return;
-    const ChunkPos pos = locate_chunk(a.ws, a.segs, a.n_seg, chunk);
-    const FmtDev f = a.ws.fmt[pos.seg];
+    const ChunkDesc d = a.ws.chunk_desc[chunk];
+    const FmtDev f = a.ws.fmt[d.seg];
     if (kHist) {
-        s_hist[tid] = 0;
+        for (uint32_t i = tid; i < (uint32_t)(kHistStride * kHistCopies); i += kThreads) s_hist[i] = 0;
         __syncthreads();
     }
+    const uint64_t base = (uint64_t)u * a.client_stride + d.elem0;
+    const bool full = d.cnt == (uint32_t)kC && ((reinterpret_cast<uintptr_t>(a.grad + base) | reinterpret_cast<uintptr_t>(a.mem + base)) & 15u) == 0 &&
+                      (!kSym || (reinterpret_cast<uintptr_t>(a.sym_out + base) & 7u) == 0);
     const uint32_t i0 = tid * 8;
-    const uint32_t nv = pos.cnt > i0 ? min(8u, pos.cnt - i0) : 0u;
+    const uint32_t nv = d.cnt > i0 ? min(8u, d.cnt - i0) : 0u;
     uint32_t n_sat = 0, n_nf = 0;
-    if (nv) {
-        const uint64_t e = (uint64_t)u * a.client_stride + pos.elem0 + i0;
-        float g[8], m[8];
-        uint32_t s[8];
-        load8(a.grad + e, nv, g);
-        load8(a.mem + e, nv, m);
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            uint32_t fl = 0;
-            m[j] = convert_one(g[j], m[j], a.decay, f, s[j], fl);
-            if ((uint32_t)j < nv) { n_sat += fl & 1u; n_nf += fl >> 1; }
-        }
-        store8(a.mem + e, nv, m);
-        if (kSym) store_sym8(a.sym_out + e, nv, s);
-        if (kHist) {
+    uint32_t s[8];
+    const uint64_t e = base + i0;
+    if (full) {
+        convert8<true>(a.grad + e, a.mem + e, 8, a.decay, f, s, n_sat, n_nf);
+        if (kSym) *reinterpret_cast<uint2*>(a.sym_out + e) = pack_sym8(s);
+    } else if (nv) {
+        convert8<false>(a.grad + e, a.mem + e, nv, a.decay, f, s, n_sat, n_nf);
+        if (kSym) {
 #pragma unroll
             for (int j = 0; j < 8; ++j)
-                if ((uint32_t)j < nv) atomicAdd(&s_hist[s[j]], 1u);
+                if ((uint32_t)j < nv) a.sym_out[e + j] = (uint8_t)s[j];
         }
+    }
+    if (kHist && nv) {
+        uint32_t* h = s_hist + (tid & (kHistCopies - 1)) * kHistStride;
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+            if ((uint32_t)j < nv) atomicAdd(&h[s[j]], 1u);
     }
     add_counts(&a.res[u], n_sat, n_nf);
     if (kHist) {
         __syncthreads();
-        const uint32_t c = s_hist[tid];
-        if (c) atomicAdd(reinterpret_cast<unsigned long long*>(&a.hist_out[(size_t)pos.seg * 256 + tid]), (unsigned long long)c);
+        uint32_t c = 0;
+#pragma unroll
+        for (int i = 0; i < kHistCopies; ++i) c += s_hist[tid + i * kHistStride];
+        if (c) atomicAdd(reinterpret_cast<unsigned long long*>(&a.hist_out[(size_t)d.seg * 256 + tid]), (unsigned long long)c);
     }
 }
 
@@ -328,8 +378,6 @@ struct PackArgs {
     float* mem;
     float decay;
     const uint8_t* sym;  // symbol path
-    const co3_seg* segs;
-    uint32_t n_seg;
     uint64_t client_stride;
     uint8_t* streams;
     size_t stream_capacity;
@@ -337,74 +385,80 @@ struct PackArgs {
     Ws ws;
 };
 
-// ORs the low n bits of v (n <= 64) into the bit buffer at bit offset `off` (most significant bit first).
-__device__ __forceinline__ void put_bits(uint32_t* buf, uint32_t off, uint64_t v, uint32_t n) {
-    if (n == 0) return;
-    const uint64_t left = v << (64u - n);  // left-aligned
-    const uint32_t hi = (uint32_t)(left >> 32), lo = (uint32_t)left;
-    const uint32_t sh = off & 31u, w = off >> 5;
-    const uint32_t w0 = hi >> sh;
-    const uint32_t w1 = __funnelshift_r(lo, hi, sh);
-    const uint32_t w2 = __funnelshift_r(0u, lo, sh);
-    if (w0) atomicOr(&buf[w], w0);
-    if (n + sh > 32u && w1) atomicOr(&buf[w + 1], w1);
-    if (n + sh > 64u && w2) atomicOr(&buf[w + 2], w2);
+// ORs an n-bit value (v, right-aligned, n <= 64, bits above n clear) into the bit buffer so that its last
+// bit lands on stream bit end-1 (most significant bit first).  Words that receive only zeros are skipped.
+__device__ __forceinline__ void put_bits(uint32_t* buf, uint32_t end, uint64_t v) {
+    const uint32_t lo = (uint32_t)v, hi = (uint32_t)(v >> 32);
+    const uint32_t q = (0u - end) & 31u;  // free bits behind the value in its last word
+    const uint32_t wl = (end + 31u) >> 5;  // one past the last word touched
+    const uint32_t w2 = lo << q;
+    const uint32_t w1 = __funnelshift_l(lo, hi, q);
+    const uint32_t w0 = __funnelshift_l(hi, 0u, q);
+    if (w2) atomicOr(&buf[wl - 1], w2);
+    if (w1) atomicOr(&buf[wl - 2], w1);
+    if (w0) atomicOr(&buf[wl - 3], w0);
 }
 
 template <bool kFromSym>
 __global__ void __launch_bounds__(kThreads) pack_kernel(PackArgs a) {
     __shared__ uint32_t s_enc[256];
-    __shared__ uint32_t s_bits[kSlotWords + 4];
+    __shared__ __align__(16) uint32_t s_bits[kSlotWords + 4];
     __shared__ uint32_t s_scan[8];
     const Ctrl* ctrl = a.ws.ctrl;
     if (ctrl->abort) return;
     const uint32_t chunk = blockIdx.x, u = blockIdx.y, tid = threadIdx.x;
     if (chunk >= ctrl->n_chunks) return;
-    const ChunkPos pos = locate_chunk(a.ws, a.segs, a.n_seg, chunk);
-    s_enc[tid] = a.ws.enc_lut[pos.seg * 256 + tid];
-    for (uint32_t i = tid; i < (uint32_t)kSlotWords + 4; i += kThreads) s_bits[i] = 0;
+    const ChunkDesc d = a.ws.chunk_desc[chunk];
+    s_enc[tid] = a.ws.enc_lut[d.seg * 256 + tid];
+    reinterpret_cast<uint4*>(s_bits)[tid] = make_uint4(0, 0, 0, 0);
+    if (tid == 0) reinterpret_cast<uint4*>(s_bits)[kThreads] = make_uint4(0, 0, 0, 0);
     __syncthreads();
 
+    const uint64_t base = (uint64_t)u * a.client_stride + d.elem0;
     const uint32_t i0 = tid * 8;
-    const uint32_t nv = pos.cnt > i0 ? min(8u, pos.cnt - i0) : 0u;
+    const uint32_t nv = d.cnt > i0 ? min(8u, d.cnt - i0) : 0u;
+    const uint64_t e = base + i0;
     uint32_t s[8];
     uint32_t n_sat = 0, n_nf = 0;
-    if (nv) {
-        const uint64_t e = (uint64_t)u * a.client_stride + pos.elem0 + i0;
-        if (kFromSym) {
-            load_sym8(a.sym + e, nv, s);
+    bool full;
+    if (kFromSym) {
+        full = d.cnt == (uint32_t)kC && (reinterpret_cast<uintptr_t>(a.sym + base) & 7u) == 0;
+        if (full) {
+            const uint2 w = __ldg(reinterpret_cast<const uint2*>(a.sym + e));
+#pragma unroll
+            for (int j = 0; j < 4; ++j) { s[j] = (w.x >> (8 * j)) & 0xffu; s[4 + j] = (w.y >> (8 * j)) & 0xffu; }
         } else {
-            const FmtDev f = a.ws.fmt[pos.seg];
-            float g[8], m[8];
-            load8(a.grad + e, nv, g);
-            load8(a.mem + e, nv, m);
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                uint32_t fl = 0;
-                m[j] = convert_one(g[j], m[j], a.decay, f, s[j], fl);
-                if ((uint32_t)j < nv) { n_sat += fl & 1u; n_nf += fl >> 1; }
-            }
-            store8(a.mem + e, nv, m);
+            for (int j = 0; j < 8; ++j) s[j] = (uint32_t)j < nv ? a.sym[e + j] : 0u;
         }
+    } else {
+        const FmtDev f = a.ws.fmt[d.seg];
+        full = d.cnt == (uint32_t)kC &&
+               ((reinterpret_cast<uintptr_t>(a.grad + base) | reinterpret_cast<uintptr_t>(a.mem + base)) & 15u) == 0;
+        if (full) convert8<true>(a.grad + e, a.mem + e, 8, a.decay, f, s, n_sat, n_nf);
+        else if (nv) convert8<false>(a.grad + e, a.mem + e, nv, a.decay, f, s, n_sat, n_nf);
     }
-    // codewords of this thread's symbols, concatenated in two 64-bit halves
-    uint64_t wa = 0, wb = 0;
-    uint32_t la = 0, lb = 0;
-    bool missing = false;
+    // codewords of this thread's symbols, concatenated in two halves of at most 64 bits
+    uint32_t ent[8];
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
-        if ((uint32_t)j < nv) {
-            const uint32_t ent = s_enc[s[j]];
-            const uint32_t l = ent & 0xffu;
-            missing |= (l == 0);
-            if (j < 4) { wa = (wa << l) | (ent >> 8); la += l; }
-            else       { wb = (wb << l) | (ent >> 8); lb += l; }
-        }
-    }
+    for (int j = 0; j < 8; ++j) ent[j] = ((uint32_t)j < nv) ? s_enc[s[j]] : 0u;
+    const uint32_t any = ent[0] | ent[1] | ent[2] | ent[3] | ent[4] | ent[5] | ent[6] | ent[7];
+    const bool missing = (any & kEncMissing) != 0;
+    // the low byte of an entry is its length, at most 16: sums of four stay inside the byte
+    const uint32_t la = (ent[0] + ent[1] + ent[2] + ent[3]) & 0xffu;
+    const uint32_t lb = (ent[4] + ent[5] + ent[6] + ent[7]) & 0xffu;
+    const uint32_t c01 = ((ent[0] >> 8) << (ent[1] & 0xffu)) | (ent[1] >> 8);
+    const uint32_t c23 = ((ent[2] >> 8) << (ent[3] & 0xffu)) | (ent[3] >> 8);
+    const uint32_t c45 = ((ent[4] >> 8) << (ent[5] & 0xffu)) | (ent[5] >> 8);
+    const uint32_t c67 = ((ent[6] >> 8) << (ent[7] & 0xffu)) | (ent[7] >> 8);
+    const uint64_t wa = ((uint64_t)c01 << ((ent[2] + ent[3]) & 0xffu)) | c23;
+    const uint64_t wb = ((uint64_t)c45 << ((ent[6] + ent[7]) & 0xffu)) | c67;
     uint32_t total;
     const uint32_t off = block_exclusive_scan_256(la + lb, s_scan, &total);
-    put_bits(s_bits, off, wa, la);
-    put_bits(s_bits, off + la, wb, lb);
+    if (!missing) {
+        put_bits(s_bits, off + la, wa);
+        put_bits(s_bits, off + la + lb, wb);
+    }
     uint8_t* stream = a.streams + (size_t)u * a.stream_capacity;
     if ((tid & 15u) == 0)
         *reinterpret_cast<uint16_t*>(stream + ctrl->sub_off + 2ull * ((uint64_t)chunk * kSubs + (tid >> 4))) = (uint16_t)off;
@@ -546,6 +600,8 @@ struct DecArgs {
     float* out;        // average (or the single client's values); nullable when sym_out is given
     uint8_t* sym_out;  // nullable; only with n_clients == 1
     co3_result* res;
+    uint32_t B;        // clients decoded side by side in one block
+    uint32_t G;        // chunks per block (tile)
     Ws ws;
 };
 
@@ -593,15 +649,45 @@ __global__ void __launch_bounds__(kThreads) check_streams_kernel(DecArgs a) {
     }
 }
 
-// Sequential reader of one sub-chunk: a 64-bit window over the chunk's words, bounds-checked.
+constexpr int kMaxPairs = 16;                  // (chunk, client) pairs decoded side by side in one block
+constexpr int kPayWordsPerPair = 448;          // staging per pair: 7 bits/symbol; larger chunks are read in place
+constexpr int kPaySlack = 72;                  // words a reader may run past its chunk before the end check
+
+// Shared memory of one decode block; `pay` is sized for the pairs in use and followed by kPaySlack words.
+struct DecSmem {
+    uint16_t lut[kDecLut];
+    float val[256];
+    uint32_t sym[kMaxPairs][kC / 4];
+    const uint32_t* pair_base[kMaxPairs];  // where the pair's words are read from (shared or global)
+    const uint32_t* pair_src[kMaxPairs];   // global source of a staged pair
+    uint32_t pair_words[kMaxPairs];
+    uint32_t pair_staged[kMaxPairs];
+    uint32_t pair_cnt[kMaxPairs];
+    uint64_t chunk_elem0[kMaxPairs];       // first element of each chunk of the tile
+    uint32_t pay[1];
+};
+
+// Position of word j of sub-chunk s in the symbol buffer of pair p: rotated so that the 32 threads of a
+// warp (2 pairs x 16 sub-chunks, all at the same j) hit 32 different banks, and so do 32 consecutive j.
+__device__ __forceinline__ uint32_t sym_slot(uint32_t p, uint32_t s, uint32_t j) {
+    return s * 32u + ((j + s + 16u * (p & 1u)) & 31u);
+}
+
+// Sequential reader of one sub-chunk: a 64-bit window over the chunk's words.
+// kChecked: reads beyond the chunk return 0 (needed when the words are read in place from global memory);
+// otherwise the words sit in shared memory with kPaySlack readable words behind them.
+template <bool kChecked>
 struct BitReader {
-    const uint32_t* base;  // generic pointer: shared (staged) or global
+    const uint32_t* base;
     uint32_t nwords;
     uint32_t next;  // next word to fetch
     uint64_t buf;   // unread bits, left-aligned
     int have;       // number of valid bits in buf
 
-    __device__ __forceinline__ uint32_t word(uint32_t i) const { return i < nwords ? base[i] : 0u; }
+    __device__ __forceinline__ uint32_t word(uint32_t i) const {
+        if (kChecked) return i < nwords ? base[i] : 0u;
+        return base[i];
+    }
     __device__ __forceinline__ void init(const uint32_t* b, uint32_t n, uint32_t bit_off) {
         base = b;
         nwords = n;
@@ -620,165 +706,201 @@ struct BitReader {
     __device__ __forceinline__ uint32_t position() const { return next * 32u - (uint32_t)have; }
 };
 
-// Decodes one symbol.  Returns the symbol; sets err when the bits are no codeword.
-__device__ __forceinline__ uint32_t decode_one(BitReader& br, const uint16_t* __restrict__ s_lut,
-                                               const uint32_t* __restrict__ long_tab, bool& err) {
+// Decodes one symbol and returns its table entry (symbol in the low byte); `seen` collects the entries so
+// that the invalid flag can be tested once per sub-chunk.
+template <bool kChecked>
+__device__ __forceinline__ uint32_t decode_one(BitReader<kChecked>& br, const uint16_t* __restrict__ s_lut,
+                                               const uint16_t* __restrict__ sub_tab, uint32_t& seen) {
     const uint32_t top = (uint32_t)(br.buf >> 32);
-    const uint32_t ent = s_lut[top >> (32 - kDecBits)];
-    uint32_t len = ent >> 8, sym = ent & 0xffu;
-    if (len > (uint32_t)kDecBits) {  // codeword longer than the table index: search the short list
-        const uint32_t w16 = top >> 16, cnt = min(long_tab[0], 256u);
-        len = 0;
-        for (uint32_t i = 0; i < cnt; ++i) {
-            const uint32_t e = long_tab[1 + i];
-            const uint32_t l = (e >> 8) & 0xffu;
-            if ((w16 >> (16u - l)) == (e >> 16)) { len = l; sym = e & 0xffu; break; }
-        }
-    }
-    if (len == 0) { err = true; len = 1; sym = 0; }
+    uint32_t ent = s_lut[top >> (32 - kDecBits)];
+    if (ent & kDecLong)  // codeword longer than the table index: second level, by the next four bits
+        ent = __ldg(sub_tab + ((ent & 0xffu) << kSubBits) + ((top >> (32 - CO3_MAX_CODE_LEN)) & ((1u << kSubBits) - 1u)));
+    seen |= ent;
+    const uint32_t len = (ent >> 8) & 0x1fu;
     br.buf <<= len;
     br.have -= (int)len;
-    return sym;
+    return ent;
 }
 
-template <int B, int G>
-struct DecSmem {
-    static constexpr int kPairs = B * G;
-    static constexpr int kPayWords = kPairs * 384;  // staging for ~6 bits/symbol; larger chunks are read in place
-    uint16_t lut[kDecLut];
-    float val[256];
-    uint32_t sym[kPairs][kC / 4];
-    uint32_t pay[kPayWords];
-    const uint32_t* pair_base[kPairs];
-    uint32_t pair_words[kPairs];
-    uint32_t pair_chunk[kPairs];
-    uint32_t pair_cnt[kPairs];
-};
-
-// Position of word j of sub-chunk s in the symbol buffer of pair p: rotated so that the 32 threads of a
-// warp (2 pairs x 16 sub-chunks, all at the same j) hit 32 different banks, and so do 32 consecutive j.
-__device__ __forceinline__ uint32_t sym_slot(uint32_t p, uint32_t s, uint32_t j) {
-    return s * 32u + ((j + s + 16u * (p & 1u)) & 31u);
+// Decodes `my` (<= 128) symbols of one sub-chunk into the swizzled symbol buffer, four per word.
+// Returns the bit position (inside the chunk) behind the last symbol.
+template <bool kChecked, bool kWhole>
+__device__ __forceinline__ uint32_t decode_sub(const uint32_t* words, uint32_t nwords, uint32_t off, uint32_t my,
+                                               const uint16_t* __restrict__ s_lut, const uint16_t* __restrict__ sub_tab,
+                                               uint32_t* out, uint32_t p, uint32_t s, bool& err) {
+    BitReader<kChecked> br;
+    br.init(words, nwords, off);
+    uint32_t seen = 0;
+    const uint32_t rot = s + 16u * (p & 1u);
+    uint32_t* row = out + s * 32u;
+#pragma unroll 2
+    for (uint32_t j = 0; j < 32; ++j) {
+        uint32_t w = 0;
+        if (kWhole || j * 4 < my) {
+            br.refill();
+            const uint32_t e0 = decode_one(br, s_lut, sub_tab, seen);
+            const uint32_t e1 = (kWhole || j * 4 + 1 < my) ? decode_one(br, s_lut, sub_tab, seen) : 0u;
+            br.refill();
+            const uint32_t e2 = (kWhole || j * 4 + 2 < my) ? decode_one(br, s_lut, sub_tab, seen) : 0u;
+            const uint32_t e3 = (kWhole || j * 4 + 3 < my) ? decode_one(br, s_lut, sub_tab, seen) : 0u;
+            w = __byte_perm(__byte_perm(e0, e1, 0x0040), __byte_perm(e2, e3, 0x0040), 0x5410);
+        }
+        row[(j + rot) & 31u] = w;
+    }
+    if (seen & kDecErrBit) err = true;
+    return br.position();
 }
 
-template <int B, int G>
-__global__ void __launch_bounds__(16 * B * G) decode_kernel(DecArgs a) {
-    constexpr int kPairs = B * G;
-    constexpr int kT = 16 * kPairs;
-    constexpr int kWordsPerThread = (G * (kC / 4)) / kT;  // symbol words each thread sums per tile = 32 / B
+// Adds, in client order, the values of the four symbols of word w of the tile for the nb clients of the batch.
+// Returns the last client's symbol word.
+__device__ __forceinline__ uint32_t sum_word(const DecSmem& sm, uint32_t w, uint32_t B, uint32_t nb, float (&acc)[4]) {
+    const uint32_t cl = w / (kC / 4), wi = w % (kC / 4);
+    const uint32_t s = wi >> 5, j = wi & 31u;
+    uint32_t symw = 0;
+    for (uint32_t ul = 0; ul < nb; ++ul) {
+        const uint32_t p = cl * B + ul;
+        symw = sm.sym[p][sym_slot(p, s, j)];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) acc[q] = __fadd_rn(acc[q], sm.val[(symw >> (8 * q)) & 0xffu]);
+    }
+    return symw;
+}
+
+// Divides the sums by the number of clients and stores the (up to four) elements of word w of the tile.
+__device__ __forceinline__ void write_word(const DecArgs& a, const DecSmem& sm, const TileDesc& td, uint32_t w,
+                                           uint32_t B, const float (&acc)[4], uint32_t symw) {
+    const uint32_t cl = w / (kC / 4), wi = w % (kC / 4);
+    if (cl >= td.n_chunks) return;
+    const uint32_t cnt = sm.pair_cnt[cl * B];
+    const uint32_t i0 = wi * 4;
+    if (i0 >= cnt) return;
+    const uint32_t nv = min(4u, cnt - i0);
+    const uint64_t e = sm.chunk_elem0[cl] + i0;
+    if (a.out) {
+        const float U = (float)a.n_clients;
+        float* o = a.out + e;
+        if (nv == 4 && (reinterpret_cast<uintptr_t>(o) & 15u) == 0) {
+            *reinterpret_cast<float4*>(o) = make_float4(__fdiv_rn(acc[0], U), __fdiv_rn(acc[1], U),
+                                                        __fdiv_rn(acc[2], U), __fdiv_rn(acc[3], U));
+        } else {
+            for (uint32_t q = 0; q < nv; ++q) o[q] = __fdiv_rn(acc[q], U);
+        }
+    }
+    if (a.sym_out) {
+        uint8_t* o = a.sym_out + e;
+        if (nv == 4 && (reinterpret_cast<uintptr_t>(o) & 3u) == 0) {
+            *reinterpret_cast<uint32_t*>(o) = symw;
+        } else {
+            for (uint32_t q = 0; q < nv; ++q) o[q] = (uint8_t)(symw >> (8 * q));
+        }
+    }
+}
+
+// One block decodes a tile of G chunks for B clients at a time: 16 threads (sub-chunks) per (chunk, client)
+// pair write symbols to shared memory, then every thread sums its share of the tile over the clients in
+// client order.  kMulti: more clients than fit side by side (B = 16, G = 1): partial sums stay in registers.
+template <bool kMulti>
+__global__ void __launch_bounds__(kThreads) decode_kernel(DecArgs a) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    DecSmem<B, G>& sm = *reinterpret_cast<DecSmem<B, G>*>(smem_raw);
+    DecSmem& sm = *reinterpret_cast<DecSmem*>(smem_raw);
+    const uint32_t B = kMulti ? 16u : a.B, G = kMulti ? 1u : a.G;
+    const uint32_t n_pairs = B * G, n_thr = 16u * n_pairs;
+    const uint32_t pay_words = n_pairs * kPayWordsPerPair;
 
     const Ctrl* ctrl = a.ws.ctrl;
     if (ctrl->abort) return;
     const uint32_t tile = blockIdx.x, tid = threadIdx.x;
     if (tile >= ctrl->n_tiles) return;
-    const uint32_t seg = find_seg(a.ws.first_tile, a.n_seg, tile);
-    const uint32_t chunk0 = a.ws.first_chunk[seg] + (tile - a.ws.first_tile[seg]) * G;
-    const uint32_t n_chunks_tile = min((uint32_t)G, a.ws.first_chunk[seg + 1] - chunk0);
-    const co3_seg sg = a.segs[seg];
+    const TileDesc td = a.ws.tile_desc[tile];
     const uint64_t cap_words = (a.stream_bytes - ctrl->payload_off) / 4;
 
-    for (uint32_t i = tid; i < (uint32_t)kDecLut / 2; i += kT)
-        reinterpret_cast<uint32_t*>(sm.lut)[i] = reinterpret_cast<const uint32_t*>(a.ws.dec_lut + (size_t)seg * kDecLut)[i];
-    for (uint32_t i = tid; i < 256; i += kT) sm.val[i] = a.ws.val_lut[seg * 256 + i];
-    const uint32_t* long_tab = a.ws.dec_long + (size_t)seg * kLongStride;
+    for (uint32_t i = tid; i < (uint32_t)kDecLut / 8; i += n_thr)
+        reinterpret_cast<uint4*>(sm.lut)[i] = __ldg(reinterpret_cast<const uint4*>(a.ws.dec_lut + (size_t)td.seg * kDecLut) + i);
+    for (uint32_t i = tid; i < 256; i += n_thr) sm.val[i] = a.ws.val_lut[td.seg * 256 + i];
+    const uint16_t* sub_tab = a.ws.dec_sub + (size_t)td.seg * kSubLut;
 
-    float carry[kWordsPerThread][4];  // running sums across client batches (only when G == 1)
+    float carry[2][4];  // running sums across client batches (kMulti only)
     bool err = false;
 
     for (uint32_t u0 = 0; u0 < a.n_clients; u0 += B) {
-        const uint32_t nb = min((uint32_t)B, a.n_clients - u0);
-        __syncthreads();  // previous batch fully consumed; LUTs visible
+        const uint32_t nb = min(B, a.n_clients - u0);
+        __syncthreads();  // previous batch fully consumed; tables visible
         // ---- pair descriptors (pair = one chunk of one client) and staging plan
         if (tid < 32) {
-            uint32_t nw = 0, cnt = 0, chunk = 0;
-            const uint32_t* base = nullptr;
-            if (tid < (uint32_t)kPairs) {
+            uint32_t nw = 0, cnt = 0;
+            const uint32_t* src = nullptr;
+            if (tid < n_pairs) {
                 const uint32_t cl = tid / B, ul = tid % B;
-                if (cl < n_chunks_tile && ul < nb) {
-                    chunk = chunk0 + cl;
+                if (cl < td.n_chunks && ul < nb) {
+                    const uint32_t chunk = td.chunk0 + cl;
                     const uint8_t* stream = stream_of(a, u0 + ul);
                     const uint64_t* word_off = reinterpret_cast<const uint64_t*>(stream + ctrl->chunk_off);
                     const uint64_t w0 = word_off[chunk], w1 = word_off[chunk + 1];
-                    const uint64_t start = (uint64_t)(chunk - a.ws.first_chunk[seg]) * kC;
-                    cnt = (uint32_t)min((uint64_t)kC, sg.n_elem - start);
+                    const ChunkDesc cd = a.ws.chunk_desc[chunk];
+                    cnt = cd.cnt;
+                    if (ul == 0) sm.chunk_elem0[cl] = cd.elem0;
                     if (w0 > w1 || w1 > cap_words || w1 - w0 > (uint64_t)kSlotWords) {
                         err = true;
                         cnt = 0;
                     } else {
                         nw = (uint32_t)(w1 - w0);
-                        base = reinterpret_cast<const uint32_t*>(stream + ctrl->payload_off) + w0;
+                        src = reinterpret_cast<const uint32_t*>(stream + ctrl->payload_off) + w0;
                     }
                 }
             }
-            uint32_t inc = nw;  // inclusive prefix of the staged sizes over the pairs
+            uint32_t inc = nw;  // inclusive prefix of the sizes over the pairs
 #pragma unroll
             for (int d = 1; d < 32; d <<= 1) {
                 const uint32_t y = __shfl_up_sync(0xffffffffu, inc, d);
                 if (tid >= (uint32_t)d) inc += y;
             }
-            if (tid < (uint32_t)kPairs) {
-                const bool staged = inc <= (uint32_t)DecSmem<B, G>::kPayWords;
-                if (staged && nw) {
-                    uint32_t* dst = sm.pay + (inc - nw);
-                    sm.pair_base[tid] = dst;
-                } else {
-                    sm.pair_base[tid] = base;  // read in place
-                }
-                sm.pair_words[tid] = (staged ? 0x80000000u : 0u) | nw;
-                sm.pair_chunk[tid] = chunk;
+            if (tid < n_pairs) {
+                const bool staged = inc <= pay_words;
+                sm.pair_base[tid] = staged ? sm.pay + (inc - nw) : src;
+                sm.pair_src[tid] = src;
+                sm.pair_words[tid] = nw;
+                sm.pair_staged[tid] = staged ? 1u : 0u;
                 sm.pair_cnt[tid] = cnt;
-                // remember the source for the copy below
-                if (staged && nw) reinterpret_cast<const uint32_t**>(sm.sym[tid])[0] = base;
             }
         }
         __syncthreads();
         // ---- stage the payloads (coalesced)
-        for (uint32_t p = 0; p < (uint32_t)kPairs; ++p) {
-            const uint32_t pw = sm.pair_words[p];
-            if (!(pw & 0x80000000u) || !(pw & 0x7fffffffu)) continue;
-            const uint32_t* src = reinterpret_cast<const uint32_t* const*>(sm.sym[p])[0];
+        for (uint32_t p = 0; p < n_pairs; ++p) {
+            if (!sm.pair_staged[p]) continue;
+            const uint32_t nw = sm.pair_words[p];
+            const uint32_t* src = sm.pair_src[p];
             uint32_t* dst = const_cast<uint32_t*>(sm.pair_base[p]);
-            const uint32_t nw = pw & 0x7fffffffu;
-            for (uint32_t i = tid; i < nw; i += kT) dst[i] = __ldg(src + i);
+            for (uint32_t i = tid; i < nw; i += n_thr) dst[i] = __ldg(src + i);
         }
         __syncthreads();
         // ---- decode: thread = (pair, sub-chunk)
         {
             const uint32_t p = tid >> 4, s = tid & 15u;
             const uint32_t cnt = sm.pair_cnt[p];
-            const uint32_t nw = sm.pair_words[p] & 0x7fffffffu;
+            const uint32_t nw = sm.pair_words[p];
             const uint32_t my = cnt > s * kS ? min((uint32_t)kS, cnt - s * kS) : 0u;
             uint32_t* out = sm.sym[p];
             if (my) {
                 const uint32_t cl = p / B, ul = p % B;
                 const uint8_t* stream = stream_of(a, u0 + ul);
-                const uint16_t* sub = reinterpret_cast<const uint16_t*>(stream + ctrl->sub_off) + (uint64_t)(chunk0 + cl) * kSubs;
+                const uint16_t* sub = reinterpret_cast<const uint16_t*>(stream + ctrl->sub_off) + (uint64_t)(td.chunk0 + cl) * kSubs;
                 const uint32_t off = sub[s];
                 const bool last = cnt <= (s + 1) * kS;
+                const uint32_t expect = last ? 0u : sub[s + 1];
                 if (off > nw * 32u) {
                     err = true;
                     for (uint32_t j = 0; j < 32; ++j) out[sym_slot(p, s, j)] = 0;
                 } else {
-                    BitReader br;
-                    br.init(sm.pair_base[p], nw, off);
-                    for (uint32_t j = 0; j < 32; ++j) {  // four symbols per output word
-                        uint32_t w = 0;
-                        if (j * 4 < my) {
-                            br.refill();
-                            const uint32_t s0 = decode_one(br, sm.lut, long_tab, err);
-                            const uint32_t s1 = (j * 4 + 1 < my) ? decode_one(br, sm.lut, long_tab, err) : 0u;
-                            br.refill();
-                            const uint32_t s2 = (j * 4 + 2 < my) ? decode_one(br, sm.lut, long_tab, err) : 0u;
-                            const uint32_t s3 = (j * 4 + 3 < my) ? decode_one(br, sm.lut, long_tab, err) : 0u;
-                            w = s0 | (s1 << 8) | (s2 << 16) | (s3 << 24);
-                        }
-                        out[sym_slot(p, s, j)] = w;
+                    uint32_t end;
+                    const uint32_t* words = sm.pair_base[p];
+                    if (sm.pair_staged[p]) {
+                        if (my == (uint32_t)kS) end = decode_sub<false, true>(words, nw, off, my, sm.lut, sub_tab, out, p, s, err);
+                        else end = decode_sub<false, false>(words, nw, off, my, sm.lut, sub_tab, out, p, s, err);
+                    } else {
+                        end = decode_sub<true, false>(words, nw, off, my, sm.lut, sub_tab, out, p, s, err);
                     }
-                    const uint32_t end = br.position();
                     if (!last) {
-                        if (end != sub[s + 1]) err = true;
+                        if (end != expect) err = true;
                     } else if (((end + 31u) >> 5) != nw) {
                         err = true;
                     }
@@ -788,57 +910,35 @@ __global__ void __launch_bounds__(16 * B * G) decode_kernel(DecArgs a) {
             }
         }
         __syncthreads();
-        // ---- ordered sum over the clients of this batch; thread owns whole symbol words
+        // ---- ordered sum over the clients of this batch; a thread owns whole symbol words
         const bool first_batch = (u0 == 0), last_batch = (u0 + B >= a.n_clients);
+        if (kMulti) {
 #pragma unroll
-        for (int r = 0; r < kWordsPerThread; ++r) {
-            const uint32_t w = tid + r * kT;         // word index inside the tile
-            const uint32_t cl = w / (kC / 4), wi = w % (kC / 4);
-            const uint32_t s = wi >> 5, j = wi & 31u;
-            float acc[4];
+            for (int r = 0; r < 2; ++r) {
+                const uint32_t w = tid + r * kThreads;
+                float acc[4];
 #pragma unroll
-            for (int q = 0; q < 4; ++q) acc[q] = (G == 1 && !first_batch) ? carry[r][q] : 0.0f;
-            uint32_t symw = 0;
-            for (uint32_t ul = 0; ul < nb; ++ul) {
-                const uint32_t p = cl * B + ul;
-                symw = sm.sym[p][sym_slot(p, s, j)];
+                for (int q = 0; q < 4; ++q) acc[q] = first_batch ? 0.0f : carry[r][q];
+                const uint32_t symw = sum_word(sm, w, B, nb, acc);
+                if (!last_batch) {
 #pragma unroll
-                for (int q = 0; q < 4; ++q) acc[q] = __fadd_rn(acc[q], sm.val[(symw >> (8 * q)) & 0xffu]);
-            }
-            if (G == 1 && !last_batch) {
-#pragma unroll
-                for (int q = 0; q < 4; ++q) carry[r][q] = acc[q];
-                continue;
-            }
-            if (cl >= n_chunks_tile) continue;
-            const uint32_t cnt = sm.pair_cnt[cl * B];
-            const uint32_t i0 = wi * 4;
-            if (i0 >= cnt) continue;
-            const uint32_t nv = min(4u, cnt - i0);
-            const uint64_t e = sg.elem_off + (uint64_t)(chunk0 + cl - a.ws.first_chunk[seg]) * kC + i0;
-            if (a.out) {
-                const float U = (float)a.n_clients;
-                float* o = a.out + e;
-                if (nv == 4 && (reinterpret_cast<uintptr_t>(o) & 15u) == 0) {
-                    *reinterpret_cast<float4*>(o) = make_float4(__fdiv_rn(acc[0], U), __fdiv_rn(acc[1], U),
-                                                                __fdiv_rn(acc[2], U), __fdiv_rn(acc[3], U));
+                    for (int q = 0; q < 4; ++q) carry[r][q] = acc[q];
                 } else {
-                    for (uint32_t q = 0; q < nv; ++q) o[q] = __fdiv_rn(acc[q], U);
+                    write_word(a, sm, td, w, B, acc, symw);
                 }
             }
-            if (a.sym_out) {
-                uint8_t* o = a.sym_out + e;
-                if (nv == 4 && (reinterpret_cast<uintptr_t>(o) & 3u) == 0) {
-                    *reinterpret_cast<uint32_t*>(o) = symw;
-                } else {
-                    for (uint32_t q = 0; q < nv; ++q) o[q] = (uint8_t)(symw >> (8 * q));
-                }
+        } else {
+            const uint32_t tile_words = G * (kC / 4);
+            for (uint32_t w = tid; w < tile_words; w += n_thr) {
+                float acc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+                const uint32_t symw = sum_word(sm, w, B, nb, acc);
+                write_word(a, sm, td, w, B, acc, symw);
             }
         }
     }
     if (__syncthreads_or(err) && tid == 0) {
         set_status(a.res, CO3_ERR_CORRUPT);
-        atomicMin(&a.res->first_bad_chunk, chunk0);
+        atomicMin(&a.res->first_bad_chunk, td.chunk0);
     }
 }
 
@@ -852,7 +952,7 @@ using namespace co3;
 namespace {
 
 struct WsLayout {
-    size_t ctrl, first_chunk, first_tile, fmt, enc_lut, dec_lut, dec_long, val_lut, client_fail, chunk_bits,
+    size_t ctrl, first_chunk, chunk_desc, tile_desc, fmt, enc_lut, dec_lut, dec_sub, val_lut, client_fail, chunk_bits,
         bit_prefix, slots, total;
     uint32_t n_chunks_max;
 };
@@ -867,11 +967,12 @@ bool ws_layout(uint64_t n_elem, uint32_t n_seg, uint32_t n_clients, WsLayout* L)
     size_t o = 0;
     L->ctrl = o;        o += up256(sizeof(Ctrl));
     L->first_chunk = o; o += up256(4 * ((size_t)n_seg + 1));
-    L->first_tile = o;  o += up256(4 * ((size_t)n_seg + 1));
+    L->chunk_desc = o;  o += up256(sizeof(ChunkDesc) * (size_t)nc);
+    L->tile_desc = o;   o += up256(sizeof(TileDesc) * (size_t)nc);
     L->fmt = o;         o += up256(sizeof(FmtDev) * (size_t)n_seg);
     L->enc_lut = o;     o += up256(4 * 256 * (size_t)n_seg);
     L->dec_lut = o;     o += up256(2 * (size_t)kDecLut * n_seg);
-    L->dec_long = o;    o += up256(4 * (size_t)kLongStride * n_seg);
+    L->dec_sub = o;     o += up256(2 * (size_t)kSubLut * n_seg);
     L->val_lut = o;     o += up256(4 * 256 * (size_t)n_seg);
     L->client_fail = o; o += up256(4 * (size_t)(n_clients ? n_clients : 1));
     L->chunk_bits = o;  o += up256(4 * (size_t)n_clients * nc);
@@ -886,11 +987,12 @@ Ws ws_pointers(void* base, const WsLayout& L) {
     Ws w;
     w.ctrl = reinterpret_cast<Ctrl*>(b + L.ctrl);
     w.first_chunk = reinterpret_cast<uint32_t*>(b + L.first_chunk);
-    w.first_tile = reinterpret_cast<uint32_t*>(b + L.first_tile);
+    w.chunk_desc = reinterpret_cast<ChunkDesc*>(b + L.chunk_desc);
+    w.tile_desc = reinterpret_cast<TileDesc*>(b + L.tile_desc);
     w.fmt = reinterpret_cast<FmtDev*>(b + L.fmt);
     w.enc_lut = reinterpret_cast<uint32_t*>(b + L.enc_lut);
     w.dec_lut = reinterpret_cast<uint16_t*>(b + L.dec_lut);
-    w.dec_long = reinterpret_cast<uint32_t*>(b + L.dec_long);
+    w.dec_sub = reinterpret_cast<uint16_t*>(b + L.dec_sub);
     w.val_lut = reinterpret_cast<float*>(b + L.val_lut);
     w.client_fail = reinterpret_cast<uint32_t*>(b + L.client_fail);
     w.chunk_bits = reinterpret_cast<uint32_t*>(b + L.chunk_bits);
@@ -962,19 +1064,10 @@ int begin_call(const WsLayout& L, const Ws& ws, co3_result* res, uint32_t n_res,
     return CO3_OK;
 }
 
-template <int B, int G>
-int launch_decode(const DecArgs& da, uint32_t n_tiles_max, cudaStream_t st) {
-    const size_t smem = sizeof(DecSmem<B, G>);
-    CO3_CUDA(cudaFuncSetAttribute(decode_kernel<B, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    if (n_tiles_max == 0) return CO3_OK;
-    CO3_LAUNCH(CO3_KERNEL_DECODE, st, decode_kernel<B, G><<<n_tiles_max, 16 * B * G, smem, st>>>(da));
-    return CO3_OK;
-}
-
-int decode_common(const uint8_t* const* streams, const uint8_t* single, size_t stream_bytes, uint32_t n_clients, const co3_fmt* fmts,
-                  const co3_code* codes, const co3_seg* segs, uint32_t n_seg, uint64_t n_elem, uint32_t chunk_syms,
-                  float* out, uint8_t* sym_out, void* workspace, size_t workspace_bytes, co3_result* res,
-                  cudaStream_t st) {
+int decode_common(const uint8_t* const* streams, const uint8_t* single, size_t stream_bytes, uint32_t n_clients,
+                  const co3_fmt* fmts, const co3_code* codes, const co3_seg* segs, uint32_t n_seg, uint64_t n_elem,
+                  uint32_t chunk_syms, float* out, uint8_t* sym_out, void* workspace, size_t workspace_bytes,
+                  co3_result* res, cudaStream_t st) {
     if ((!streams && !single) || !fmts || !codes || !res || !workspace || n_clients == 0 || chunk_syms != (uint32_t)kC)
         return CO3_ERR_INVALID_ARG;
     if ((!segs && n_seg) || (!out && !sym_out) || (sym_out && n_clients != 1)) return CO3_ERR_INVALID_ARG;
@@ -984,23 +1077,32 @@ int decode_common(const uint8_t* const* streams, const uint8_t* single, size_t s
     if (workspace_bytes < L.total) return CO3_ERR_CAPACITY;
     const Ws ws = ws_pointers(workspace, L);
 
-    // clients decoded side by side per block (B) and chunks per block (G): 16 sub-chunk threads per pair
-    int B = 1;
-    while (B < 16 && (uint32_t)B < n_clients) B <<= 1;
-    int G = 16 / B;
-    const uint64_t chunks = L.n_chunks_max;
-    if (G > 1 && chunks / G < 2 * 148) G = (4 / B) > 0 ? 4 / B : 1;  // small inputs: more, smaller blocks
-    const int rc = begin_call(L, ws, res, 1, st, fmts, codes, segs, n_seg, n_elem, (uint32_t)G, 1);
+    // B clients side by side and G chunks per block, 16 sub-chunk threads per (chunk, client) pair, at most
+    // 16 pairs; small inputs take fewer chunks per block so that the grid still covers the GPU
+    const bool multi = n_clients > (uint32_t)kMaxPairs;
+    uint32_t B = multi ? (uint32_t)kMaxPairs : n_clients;
+    uint32_t G = multi ? 1u : (uint32_t)kMaxPairs / B;
+    const uint32_t g_min = (B == 1) ? 2u : 1u;  // a block needs at least one full warp
+    if (!multi && G > g_min) {
+        const uint64_t want = L.n_chunks_max / (2 * 148) + 1;  // chunks per block that still give two waves
+        if (want < G) G = (uint32_t)(want < g_min ? g_min : want);
+    }
+    const int rc = begin_call(L, ws, res, 1, st, fmts, codes, segs, n_seg, n_elem, G, 1);
     if (rc != CO3_OK) return rc;
-    DecArgs da{streams, single, stream_bytes, n_clients, segs, n_seg, n_elem, out, sym_out, res, ws};
+    DecArgs da{streams, single, stream_bytes, n_clients, segs, n_seg, n_elem, out, sym_out, res, B, G, ws};
     CO3_LAUNCH(CO3_KERNEL_CHECK, st, check_streams_kernel<<<n_clients, kThreads, 0, st>>>(da));
-    const uint32_t tiles = (uint32_t)(chunks / G + n_seg);  // upper bound; surplus blocks return at once
-#define CO3_DEC_CASE(b, g) \
-    if (B == b && G == g) return launch_decode<b, g>(da, tiles, st);
-    CO3_DEC_CASE(1, 16) CO3_DEC_CASE(1, 4) CO3_DEC_CASE(2, 8) CO3_DEC_CASE(2, 2) CO3_DEC_CASE(4, 4)
-    CO3_DEC_CASE(4, 1) CO3_DEC_CASE(8, 2) CO3_DEC_CASE(8, 1) CO3_DEC_CASE(16, 1)
-#undef CO3_DEC_CASE
-    return CO3_ERR_INVALID_ARG;
+    const uint32_t tiles = (uint32_t)(L.n_chunks_max / G + n_seg);  // upper bound; surplus blocks return at once
+    if (tiles == 0) return CO3_OK;
+    const uint32_t n_pairs = B * G;
+    const size_t smem = offsetof(DecSmem, pay) + 4 * ((size_t)n_pairs * kPayWordsPerPair + kPaySlack);
+    if (multi) {
+        CO3_CUDA(cudaFuncSetAttribute(decode_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        CO3_LAUNCH(CO3_KERNEL_DECODE, st, decode_kernel<true><<<tiles, kThreads, smem, st>>>(da));
+    } else {
+        CO3_CUDA(cudaFuncSetAttribute(decode_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        CO3_LAUNCH(CO3_KERNEL_DECODE, st, decode_kernel<false><<<tiles, 16 * n_pairs, smem, st>>>(da));
+    }
+    return CO3_OK;
 }
 
 int encode_common(const float* grad, float* mem, float decay, const uint8_t* sym, const co3_fmt* fmts,
@@ -1023,7 +1125,7 @@ int encode_common(const float* grad, float* mem, float decay, const uint8_t* sym
     const int rc = begin_call(L, ws, res, n_clients, st, sym ? nullptr : fmts, codes, segs, n_seg, n_elem, 1, n_clients);
     if (rc != CO3_OK) return rc;
     if (L.n_chunks_max) {
-        PackArgs pa{grad, mem, decay, sym, segs, n_seg, client_stride, streams_out, stream_capacity, res, ws};
+        PackArgs pa{grad, mem, decay, sym, client_stride, streams_out, stream_capacity, res, ws};
         const dim3 grid(L.n_chunks_max, n_clients);
         if (sym) CO3_LAUNCH(CO3_KERNEL_PACK, st, pack_kernel<true><<<grid, kThreads, 0, st>>>(pa));
         else CO3_LAUNCH(CO3_KERNEL_PACK, st, pack_kernel<false><<<grid, kThreads, 0, st>>>(pa));
@@ -1109,7 +1211,7 @@ int co3_convert(const float* grad, float* mem, float decay, const co3_fmt* fmts,
     const int rc = begin_call(L, ws, res, n_clients, st, fmts, nullptr, segs, n_seg, n_elem, 1, 1);
     if (rc != CO3_OK) return rc;
     if (L.n_chunks_max == 0) return CO3_OK;
-    ConvertArgs ca{grad, mem, decay, segs, n_seg, client_stride_elems, sym_out, hist_out, res, ws};
+    ConvertArgs ca{grad, mem, decay, client_stride_elems, sym_out, hist_out, res, ws};
     const dim3 grid(L.n_chunks_max, n_clients);
     if (sym_out && hist_out) CO3_LAUNCH(CO3_KERNEL_CONVERT, st, convert_kernel<true, true><<<grid, kThreads, 0, st>>>(ca));
     else if (sym_out) CO3_LAUNCH(CO3_KERNEL_CONVERT, st, convert_kernel<true, false><<<grid, kThreads, 0, st>>>(ca));
