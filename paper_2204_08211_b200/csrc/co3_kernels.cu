@@ -649,23 +649,26 @@ __global__ void __launch_bounds__(kThreads) check_streams_kernel(DecArgs a) {
     }
 }
 
-constexpr int kMaxPairs = 16;                  // (chunk, client) pairs decoded side by side in one block
-constexpr int kPayWordsPerPair = 448;          // staging per pair: 7 bits/symbol; larger chunks are read in place
-constexpr int kPaySlack = 72;                  // words a reader may run past its chunk before the end check
+constexpr int kMaxPairs = 16;          // (chunk, client) pairs decoded side by side in one block
+constexpr int kPaySlotWords = 456;     // staging per pair: 7 bits/symbol plus alignment; larger chunks are read in place
+constexpr int kPaySlack = 72;          // words a reader may run past its chunk before the end check
 
-// Shared memory of one decode block; `pay` is sized for the pairs in use and followed by kPaySlack words.
+// Fixed part of the shared memory of one decode block; behind it follow the symbol buffer
+// sym[n_pairs][kC / 4] and the payload staging area pay[n_pairs * kPaySlotWords + kPaySlack].
 struct DecSmem {
     uint16_t lut[kDecLut];
     float val[256];
-    uint32_t sym[kMaxPairs][kC / 4];
-    const uint32_t* pair_base[kMaxPairs];  // where the pair's words are read from (shared or global)
-    const uint32_t* pair_src[kMaxPairs];   // global source of a staged pair
+    uint64_t bar;                          // completion barrier of the bulk copies of one batch
+    uint64_t pad;
+    uint64_t chunk_elem0[kMaxPairs];       // first element of each chunk of the tile
+    const uint32_t* pair_src[kMaxPairs];   // the pair's first payload word in global memory
+    uint32_t pair_off[kMaxPairs];          // staged pairs: index of that word in pay[]
     uint32_t pair_words[kMaxPairs];
     uint32_t pair_staged[kMaxPairs];
     uint32_t pair_cnt[kMaxPairs];
-    uint64_t chunk_elem0[kMaxPairs];       // first element of each chunk of the tile
-    uint32_t pay[1];
+    uint16_t sub[kMaxPairs][kSubs];        // sub-chunk bit offsets of each pair
 };
+static_assert(sizeof(DecSmem) % 16 == 0 && offsetof(DecSmem, sub) % 16 == 0, "dynamic arrays behind DecSmem must stay 16-byte aligned");
 
 // Position of word j of sub-chunk s in the symbol buffer of pair p: rotated so that the 32 threads of a
 // warp (2 pairs x 16 sub-chunks, all at the same j) hit 32 different banks, and so do 32 consecutive j.
@@ -685,7 +688,7 @@ struct BitReader {
     int have;       // number of valid bits in buf
 
     __device__ __forceinline__ uint32_t word(uint32_t i) const {
-        if (kChecked) return i < nwords ? base[i] : 0u;
+        if (kChecked) return i < nwords ? __ldg(base + i) : 0u;
         return base[i];
     }
     __device__ __forceinline__ void init(const uint32_t* b, uint32_t n, uint32_t bit_off) {
@@ -722,17 +725,15 @@ __device__ __forceinline__ uint32_t decode_one(BitReader<kChecked>& br, const ui
     return ent;
 }
 
-// Decodes `my` (<= 128) symbols of one sub-chunk into the swizzled symbol buffer, four per word.
-// Returns the bit position (inside the chunk) behind the last symbol.
+// Decodes `my` (<= 128) symbols of one sub-chunk into its row of the swizzled symbol buffer, four per
+// word.  Returns the bit position (inside the chunk) behind the last symbol.
 template <bool kChecked, bool kWhole>
 __device__ __forceinline__ uint32_t decode_sub(const uint32_t* words, uint32_t nwords, uint32_t off, uint32_t my,
                                                const uint16_t* __restrict__ s_lut, const uint16_t* __restrict__ sub_tab,
-                                               uint32_t* out, uint32_t p, uint32_t s, bool& err) {
+                                               uint32_t* row, uint32_t rot, bool& err) {
     BitReader<kChecked> br;
     br.init(words, nwords, off);
     uint32_t seen = 0;
-    const uint32_t rot = s + 16u * (p & 1u);
-    uint32_t* row = out + s * 32u;
 #pragma unroll 2
     for (uint32_t j = 0; j < 32; ++j) {
         uint32_t w = 0;
@@ -753,15 +754,16 @@ __device__ __forceinline__ uint32_t decode_sub(const uint32_t* words, uint32_t n
 
 // Adds, in client order, the values of the four symbols of word w of the tile for the nb clients of the batch.
 // Returns the last client's symbol word.
-__device__ __forceinline__ uint32_t sum_word(const DecSmem& sm, uint32_t w, uint32_t B, uint32_t nb, float (&acc)[4]) {
+__device__ __forceinline__ uint32_t sum_word(const float* __restrict__ val, const uint32_t* __restrict__ sym, uint32_t w,
+                                             uint32_t B, uint32_t nb, float (&acc)[4]) {
     const uint32_t cl = w / (kC / 4), wi = w % (kC / 4);
     const uint32_t s = wi >> 5, j = wi & 31u;
     uint32_t symw = 0;
     for (uint32_t ul = 0; ul < nb; ++ul) {
         const uint32_t p = cl * B + ul;
-        symw = sm.sym[p][sym_slot(p, s, j)];
+        symw = sym[p * (kC / 4) + sym_slot(p, s, j)];
 #pragma unroll
-        for (int q = 0; q < 4; ++q) acc[q] = __fadd_rn(acc[q], sm.val[(symw >> (8 * q)) & 0xffu]);
+        for (int q = 0; q < 4; ++q) acc[q] = __fadd_rn(acc[q], val[(symw >> (8 * q)) & 0xffu]);
     }
     return symw;
 }
@@ -796,16 +798,20 @@ __device__ __forceinline__ void write_word(const DecArgs& a, const DecSmem& sm, 
     }
 }
 
-// One block decodes a tile of G chunks for B clients at a time: 16 threads (sub-chunks) per (chunk, client)
-// pair write symbols to shared memory, then every thread sums its share of the tile over the clients in
-// client order.  kMulti: more clients than fit side by side (B = 16, G = 1): partial sums stay in registers.
+// One block decodes a tile of G chunks for B clients at a time.  Warp 0 looks up where each (chunk, client)
+// pair's payload lies and starts one bulk copy per pair into shared memory (plus the segment's tables);
+// then 16 threads per pair (one per sub-chunk) decode into a symbol buffer, and finally every thread sums
+// its share of the tile over the clients in client order.  kMulti: more clients than fit side by side
+// (B = 16, G = 1): the partial sums stay in registers between batches.
 template <bool kMulti>
 __global__ void __launch_bounds__(kThreads) decode_kernel(DecArgs a) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     DecSmem& sm = *reinterpret_cast<DecSmem*>(smem_raw);
     const uint32_t B = kMulti ? 16u : a.B, G = kMulti ? 1u : a.G;
     const uint32_t n_pairs = B * G, n_thr = 16u * n_pairs;
-    const uint32_t pay_words = n_pairs * kPayWordsPerPair;
+    uint32_t* const sm_sym = reinterpret_cast<uint32_t*>(smem_raw + sizeof(DecSmem));
+    uint32_t* const sm_pay = sm_sym + n_pairs * (kC / 4);
+    const uint32_t pay_words = n_pairs * kPaySlotWords;
 
     const Ctrl* ctrl = a.ws.ctrl;
     if (ctrl->abort) return;
@@ -813,22 +819,23 @@ __global__ void __launch_bounds__(kThreads) decode_kernel(DecArgs a) {
     if (tile >= ctrl->n_tiles) return;
     const TileDesc td = a.ws.tile_desc[tile];
     const uint64_t cap_words = (a.stream_bytes - ctrl->payload_off) / 4;
-
-    for (uint32_t i = tid; i < (uint32_t)kDecLut / 8; i += n_thr)
-        reinterpret_cast<uint4*>(sm.lut)[i] = __ldg(reinterpret_cast<const uint4*>(a.ws.dec_lut + (size_t)td.seg * kDecLut) + i);
-    for (uint32_t i = tid; i < 256; i += n_thr) sm.val[i] = a.ws.val_lut[td.seg * 256 + i];
+    const uint64_t readable16 = a.stream_bytes & ~(size_t)15u;  // bulk copies move whole 16-byte units
     const uint16_t* sub_tab = a.ws.dec_sub + (size_t)td.seg * kSubLut;
 
+    if (tid == 0) mbar_init(&sm.bar, 1);
     float carry[2][4];  // running sums across client batches (kMulti only)
-    bool err = false;
+    bool err = false, hw_fail = false;
+    uint32_t phase = 0;
 
-    for (uint32_t u0 = 0; u0 < a.n_clients; u0 += B) {
+    for (uint32_t u0 = 0; u0 < a.n_clients; u0 += B, phase ^= 1u) {
         const uint32_t nb = min(B, a.n_clients - u0);
-        __syncthreads();  // previous batch fully consumed; tables visible
-        // ---- pair descriptors (pair = one chunk of one client) and staging plan
+        __syncthreads();  // barrier initialised; previous batch fully consumed
+        // ---- pair descriptors (pair = one chunk of one client), staging plan, bulk copies
         if (tid < 32) {
-            uint32_t nw = 0, cnt = 0;
+            uint32_t nw = 0, cnt = 0, lead = 0, span = 0;  // span: words of the 16-byte aligned copy
             const uint32_t* src = nullptr;
+            bool can_stage = false;
+            const uint16_t* sub_src = nullptr;
             if (tid < n_pairs) {
                 const uint32_t cl = tid / B, ul = tid % B;
                 if (cl < td.n_chunks && ul < nb) {
@@ -839,75 +846,89 @@ __global__ void __launch_bounds__(kThreads) decode_kernel(DecArgs a) {
                     const ChunkDesc cd = a.ws.chunk_desc[chunk];
                     cnt = cd.cnt;
                     if (ul == 0) sm.chunk_elem0[cl] = cd.elem0;
+                    sub_src = reinterpret_cast<const uint16_t*>(stream + ctrl->sub_off) + (uint64_t)chunk * kSubs;
                     if (w0 > w1 || w1 > cap_words || w1 - w0 > (uint64_t)kSlotWords) {
                         err = true;
                         cnt = 0;
                     } else {
                         nw = (uint32_t)(w1 - w0);
-                        src = reinterpret_cast<const uint32_t*>(stream + ctrl->payload_off) + w0;
+                        const uint64_t byte0 = ctrl->payload_off + 4ull * w0;
+                        src = reinterpret_cast<const uint32_t*>(stream + byte0);
+                        lead = (uint32_t)(byte0 & 15u) / 4u;
+                        span = (lead + nw + 3u) & ~3u;
+                        can_stage = nw != 0 && (byte0 & ~15ull) + 4ull * span <= readable16;
                     }
                 }
             }
-            uint32_t inc = nw;  // inclusive prefix of the sizes over the pairs
+            uint32_t inc = can_stage ? span : 0u;  // inclusive prefix of the staged spans over the pairs
 #pragma unroll
             for (int d = 1; d < 32; d <<= 1) {
                 const uint32_t y = __shfl_up_sync(0xffffffffu, inc, d);
                 if (tid >= (uint32_t)d) inc += y;
             }
+            const bool staged = can_stage && inc <= pay_words;
+            uint32_t bytes = (staged ? 4u * span : 0u) + (sub_src ? 2u * kSubs : 0u);
+            if (tid == 0 && u0 == 0) bytes += 2u * kDecLut + 4u * 256u;  // the segment's tables, once
+            const uint32_t total = __reduce_add_sync(0xffffffffu, bytes);
+            if (tid == 0) {
+                fence_async_smem();
+                mbar_arrive_expect_tx(&sm.bar, total);
+            }
+            __syncwarp();
+            if (tid == 0 && u0 == 0) {
+                bulk_copy_g2s(sm.lut, a.ws.dec_lut + (size_t)td.seg * kDecLut, 2u * kDecLut, &sm.bar);
+                bulk_copy_g2s(sm.val, a.ws.val_lut + (size_t)td.seg * 256, 4u * 256u, &sm.bar);
+            }
+            if (staged) bulk_copy_g2s(sm_pay + (inc - span), src - lead, 4u * span, &sm.bar);
+            if (sub_src) bulk_copy_g2s(sm.sub[tid], sub_src, 2u * kSubs, &sm.bar);
             if (tid < n_pairs) {
-                const bool staged = inc <= pay_words;
-                sm.pair_base[tid] = staged ? sm.pay + (inc - nw) : src;
                 sm.pair_src[tid] = src;
+                sm.pair_off[tid] = inc - span + lead;
                 sm.pair_words[tid] = nw;
                 sm.pair_staged[tid] = staged ? 1u : 0u;
                 sm.pair_cnt[tid] = cnt;
             }
         }
         __syncthreads();
-        // ---- stage the payloads (coalesced)
-        for (uint32_t p = 0; p < n_pairs; ++p) {
-            if (!sm.pair_staged[p]) continue;
-            const uint32_t nw = sm.pair_words[p];
-            const uint32_t* src = sm.pair_src[p];
-            uint32_t* dst = const_cast<uint32_t*>(sm.pair_base[p]);
-            for (uint32_t i = tid; i < nw; i += n_thr) dst[i] = __ldg(src + i);
+        if (!__syncthreads_and(mbar_wait(&sm.bar, phase))) {  // never expected: the copies are in bounds and aligned
+            hw_fail = true;
+            mbar_wait(&sm.bar, phase);
+            break;
         }
-        __syncthreads();
         // ---- decode: thread = (pair, sub-chunk)
         {
             const uint32_t p = tid >> 4, s = tid & 15u;
             const uint32_t cnt = sm.pair_cnt[p];
             const uint32_t nw = sm.pair_words[p];
             const uint32_t my = cnt > s * kS ? min((uint32_t)kS, cnt - s * kS) : 0u;
-            uint32_t* out = sm.sym[p];
+            uint32_t* row = sm_sym + p * (kC / 4) + s * 32u;
+            const uint32_t rot = s + 16u * (p & 1u);
+            bool zero = true;
             if (my) {
-                const uint32_t cl = p / B, ul = p % B;
-                const uint8_t* stream = stream_of(a, u0 + ul);
-                const uint16_t* sub = reinterpret_cast<const uint16_t*>(stream + ctrl->sub_off) + (uint64_t)(td.chunk0 + cl) * kSubs;
-                const uint32_t off = sub[s];
+                const uint32_t off = sm.sub[p][s];
                 const bool last = cnt <= (s + 1) * kS;
-                const uint32_t expect = last ? 0u : sub[s + 1];
+                const uint32_t expect = last ? 0u : sm.sub[p][s + 1];
                 if (off > nw * 32u) {
                     err = true;
-                    for (uint32_t j = 0; j < 32; ++j) out[sym_slot(p, s, j)] = 0;
                 } else {
                     uint32_t end;
-                    const uint32_t* words = sm.pair_base[p];
                     if (sm.pair_staged[p]) {
-                        if (my == (uint32_t)kS) end = decode_sub<false, true>(words, nw, off, my, sm.lut, sub_tab, out, p, s, err);
-                        else end = decode_sub<false, false>(words, nw, off, my, sm.lut, sub_tab, out, p, s, err);
+                        const uint32_t* words = sm_pay + sm.pair_off[p];
+                        if (my == (uint32_t)kS) end = decode_sub<false, true>(words, nw, off, my, sm.lut, sub_tab, row, rot, err);
+                        else end = decode_sub<false, false>(words, nw, off, my, sm.lut, sub_tab, row, rot, err);
                     } else {
-                        end = decode_sub<true, false>(words, nw, off, my, sm.lut, sub_tab, out, p, s, err);
+                        end = decode_sub<true, false>(sm.pair_src[p], nw, off, my, sm.lut, sub_tab, row, rot, err);
                     }
+                    zero = false;
                     if (!last) {
                         if (end != expect) err = true;
                     } else if (((end + 31u) >> 5) != nw) {
                         err = true;
                     }
                 }
-            } else {
-                for (uint32_t j = 0; j < 32; ++j) out[sym_slot(p, s, j)] = 0;
             }
+            if (zero)
+                for (uint32_t j = 0; j < 32; ++j) row[j] = 0;
         }
         __syncthreads();
         // ---- ordered sum over the clients of this batch; a thread owns whole symbol words
@@ -919,7 +940,7 @@ __global__ void __launch_bounds__(kThreads) decode_kernel(DecArgs a) {
                 float acc[4];
 #pragma unroll
                 for (int q = 0; q < 4; ++q) acc[q] = first_batch ? 0.0f : carry[r][q];
-                const uint32_t symw = sum_word(sm, w, B, nb, acc);
+                const uint32_t symw = sum_word(sm.val, sm_sym, w, B, nb, acc);
                 if (!last_batch) {
 #pragma unroll
                     for (int q = 0; q < 4; ++q) carry[r][q] = acc[q];
@@ -931,14 +952,17 @@ __global__ void __launch_bounds__(kThreads) decode_kernel(DecArgs a) {
             const uint32_t tile_words = G * (kC / 4);
             for (uint32_t w = tid; w < tile_words; w += n_thr) {
                 float acc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-                const uint32_t symw = sum_word(sm, w, B, nb, acc);
+                const uint32_t symw = sum_word(sm.val, sm_sym, w, B, nb, acc);
                 write_word(a, sm, td, w, B, acc, symw);
             }
         }
     }
-    if (__syncthreads_or(err) && tid == 0) {
-        set_status(a.res, CO3_ERR_CORRUPT);
-        atomicMin(&a.res->first_bad_chunk, td.chunk0);
+    const bool any_hw = __syncthreads_or(hw_fail);
+    const bool any_err = __syncthreads_or(err);
+    if (tid == 0) {
+        if (any_hw) set_status(a.res, CO3_ERR_CUDA);
+        if (any_err) set_status(a.res, CO3_ERR_CORRUPT);
+        if (any_hw || any_err) atomicMin(&a.res->first_bad_chunk, td.chunk0);
     }
 }
 
@@ -1094,7 +1118,7 @@ int decode_common(const uint8_t* const* streams, const uint8_t* single, size_t s
     const uint32_t tiles = (uint32_t)(L.n_chunks_max / G + n_seg);  // upper bound; surplus blocks return at once
     if (tiles == 0) return CO3_OK;
     const uint32_t n_pairs = B * G;
-    const size_t smem = offsetof(DecSmem, pay) + 4 * ((size_t)n_pairs * kPayWordsPerPair + kPaySlack);
+    const size_t smem = sizeof(DecSmem) + 4 * ((size_t)n_pairs * (kC / 4 + kPaySlotWords) + kPaySlack);
     if (multi) {
         CO3_CUDA(cudaFuncSetAttribute(decode_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         CO3_LAUNCH(CO3_KERNEL_DECODE, st, decode_kernel<true><<<tiles, kThreads, smem, st>>>(da));
