@@ -276,17 +276,15 @@ __device__ __forceinline__ void add_counts(co3_result* r, uint32_t n_sat, uint32
     }
 }
 
-// Correct + convert + memory update of this thread's 8 elements (Algorithm 1, client side).
-// kFull: the chunk is complete and 16-byte aligned, so the group is read and written as two float4.
-// Symbols land in s[]; the new memory is stored; counters accumulate in n_sat / n_nf.
-template <bool kFull>
-__device__ __forceinline__ void convert8(const float* __restrict__ gp, float* __restrict__ mp, uint32_t nv, float decay,
-                                         const FmtDev& f, uint32_t (&s)[8], uint32_t& n_sat, uint32_t& n_nf) {
-    float g[8], m[8], mo[8];
-    if (kFull) { load8_vec(gp, g); load8_vec(mp, m); }
-    else { load8_any(gp, nv, g); load8_any(mp, nv, m); }
+// Correct + convert + memory update of 8 elements held in registers (Algorithm 1, client side).
+// kWhole: all eight are valid, so the branch-free converter may be used.  Symbols land in s[], the new memory
+// in mo[]; counters accumulate in n_sat / n_nf.
+template <bool kWhole>
+__device__ __forceinline__ void convert8(const float (&g)[8], const float (&m)[8], uint32_t nv, float decay,
+                                         const FmtDev& f, float (&mo)[8], uint32_t (&s)[8], uint32_t& n_sat,
+                                         uint32_t& n_nf) {
     bool redo = true;
-    if (kFull && f.fast) {
+    if (kWhole && f.fast) {
         uint32_t a_max = 0;
         float nf_acc = 0.0f;
 #pragma unroll
@@ -301,18 +299,112 @@ __device__ __forceinline__ void convert8(const float* __restrict__ gp, float* __
             if ((uint32_t)j < nv) { n_sat += fl & 1u; n_nf += fl >> 1; }
         }
     }
-    if (kFull) store8_vec(mp, mo);
-    else store8_any(mp, nv, mo);
 }
 
 // ------------------------------------------------------------------------------------------------
-// convert: one block per (chunk, client)
+// Work feed of the persistent client kernels.  A work item is one chunk of one client; block b takes
+// items b, b + gridDim.x, ...  Thread 0 runs one item ahead: while the block works on item k it has
+// already started two bulk copies (gradient and memory of item k + 1, 8 KB each) into the other half
+// of a two-stage shared-memory ring, completed on that stage's mbarrier.  Chunks that are short or not
+// 16-byte aligned are not copied; their threads load from global memory directly.
+// ------------------------------------------------------------------------------------------------
+struct FeedItem {
+    ChunkDesc d;
+    uint64_t base;    // index of the chunk's first element from the batch base pointer
+    uint32_t client;
+    uint32_t tma;     // 1: gradient and memory arrive in the ring
+    uint32_t valid;   // 0: no more work
+    uint32_t chunk;   // chunk index inside the client
+};
+
+struct Feed {
+    float g[2][kC];
+    float m[2][kC];
+    uint64_t bar[2];
+    FeedItem item[2];
+    FmtDev fmt[2];    // converter constants of the item in each slot
+};
+
+struct FeedArgs {
+    const float* grad;
+    const float* mem;
+    uint64_t client_stride;
+    uint32_t n_clients;
+};
+
+// Thread 0 only: publishes item k in ring slot k & 1 and starts its copies.  `next` holds the chunk
+// descriptor fetched one call earlier for exactly this item; it is refilled for item k + 1.
+__device__ __forceinline__ void feed_issue(Feed& fd, const FeedArgs& fa, const Ws& ws, uint32_t n_chunks, uint64_t k,
+                                           ChunkDesc& next, bool use_tma) {
+    const uint64_t total = (uint64_t)n_chunks * fa.n_clients;
+    const uint64_t idx = blockIdx.x + k * gridDim.x;
+    FeedItem it;
+    it.valid = idx < total ? 1u : 0u;
+    it.d = next;
+    it.client = 0;
+    it.base = 0;
+    it.tma = 0;
+    it.chunk = 0;
+    if (it.valid) {
+        it.client = (uint32_t)(idx / n_chunks);
+        it.chunk = (uint32_t)(idx - (uint64_t)it.client * n_chunks);
+        it.base = (uint64_t)it.client * fa.client_stride + it.d.elem0;
+        const uintptr_t pg = reinterpret_cast<uintptr_t>(fa.grad + it.base), pm = reinterpret_cast<uintptr_t>(fa.mem + it.base);
+        it.tma = (use_tma && it.d.cnt == (uint32_t)kC && ((pg | pm) & 15u) == 0) ? 1u : 0u;
+    }
+    const uint32_t slot = (uint32_t)k & 1u;
+    fd.item[slot] = it;
+    if (it.tma) {
+        fence_async_smem();
+        mbar_arrive_expect_tx(&fd.bar[slot], 2u * kC * 4u);
+        bulk_copy_g2s(fd.g[slot], fa.grad + it.base, kC * 4u, &fd.bar[slot]);
+        bulk_copy_g2s(fd.m[slot], fa.mem + it.base, kC * 4u, &fd.bar[slot]);
+    }
+    const uint64_t idx_next = idx + gridDim.x;
+    if (idx_next < total) next = ws.chunk_desc[idx_next % n_chunks];
+}
+
+// The first threads of warp 0 copy the converter constants of the item in ring slot `slot` next to it; visible to the
+// block after its next barrier.
+__device__ __forceinline__ void feed_fetch_fmt(Feed& fd, const Ws& ws, uint32_t slot) {
+    static_assert(sizeof(FmtDev) % 4 == 0 && sizeof(FmtDev) / 4 <= 32, "FmtDev is copied word by word by one warp");
+    __syncwarp();  // the publishing thread 0 shares a warp with the copying threads
+    if (threadIdx.x < sizeof(FmtDev) / 4 && fd.item[slot].valid)
+        reinterpret_cast<uint32_t*>(&fd.fmt[slot])[threadIdx.x] =
+            reinterpret_cast<const uint32_t*>(&ws.fmt[fd.item[slot].d.seg])[threadIdx.x];
+}
+
+// All threads: this thread's 8 gradient and memory values of the current item.  Returns false if the
+// copies never arrived (never expected).
+// `parity` holds, per ring slot, the phase parity of the next copy to wait for.
+__device__ __forceinline__ bool feed_read(Feed& fd, const FeedArgs& fa, const FeedItem& it, uint64_t k, uint32_t i0,
+                                          uint32_t nv, uint32_t& parity, float (&g)[8], float (&m)[8]) {
+    if (it.tma) {
+        const uint32_t slot = (uint32_t)k & 1u;
+        const bool ok = mbar_wait(&fd.bar[slot], (parity >> slot) & 1u);
+        parity ^= 1u << slot;
+        if (!ok) return false;
+        const float4* gs = reinterpret_cast<const float4*>(&fd.g[slot][i0]);
+        const float4* ms = reinterpret_cast<const float4*>(&fd.m[slot][i0]);
+        const float4 a = gs[0], b = gs[1], c = ms[0], d = ms[1];
+        g[0] = a.x; g[1] = a.y; g[2] = a.z; g[3] = a.w; g[4] = b.x; g[5] = b.y; g[6] = b.z; g[7] = b.w;
+        m[0] = c.x; m[1] = c.y; m[2] = c.z; m[3] = c.w; m[4] = d.x; m[5] = d.y; m[6] = d.z; m[7] = d.w;
+    } else {
+        load8_any(fa.grad + it.base + i0, nv, g);
+        load8_any(fa.mem + it.base + i0, nv, m);
+    }
+    return true;
+}
+
+// ------------------------------------------------------------------------------------------------
+// convert: persistent blocks over (chunk, client) items
 // ------------------------------------------------------------------------------------------------
 struct ConvertArgs {
     const float* grad;
     float* mem;
     float decay;
     uint64_t client_stride;
+    uint32_t n_clients;
     uint8_t* sym_out;    // nullable
     uint64_t* hist_out;  // nullable
     co3_result* res;
@@ -323,55 +415,99 @@ constexpr int kHistCopies = 8;    // private histograms per block, spread over t
 constexpr int kHistStride = 260;  // words between copies: shifts each copy by four banks
 
 template <bool kSym, bool kHist>
-__global__ void __launch_bounds__(kThreads) convert_kernel(ConvertArgs a) {
-    __shared__ uint32_t s_hist[kHist ? kHistStride * kHistCopies : 1];
+__global__ void __launch_bounds__(kThreads, 4) convert_kernel(ConvertArgs a) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    Feed& fd = *reinterpret_cast<Feed*>(smem_raw);
+    uint32_t* s_hist = reinterpret_cast<uint32_t*>(smem_raw + sizeof(Feed));
     const Ctrl* ctrl = a.ws.ctrl;
     if (ctrl->abort) return;
-    const uint32_t chunk = blockIdx.x, u = blockIdx.y, tid = threadIdx.x;
-    if (chunk >= ctrl->n_chunks) return;
-    const ChunkDesc d = a.ws.chunk_desc[chunk];
-    const FmtDev f = a.ws.fmt[d.seg];
-    if (kHist) {
-        for (uint32_t i = tid; i < (uint32_t)(kHistStride * kHistCopies); i += kThreads) s_hist[i] = 0;
-        __syncthreads();
+    const uint32_t tid = threadIdx.x;
+    const uint32_t n_chunks = ctrl->n_chunks;
+    const FeedArgs fa{a.grad, a.mem, a.client_stride, a.n_clients};
+    if ((uint64_t)blockIdx.x >= (uint64_t)n_chunks * a.n_clients) return;
+
+    ChunkDesc next{};
+    if (tid == 0) {
+        mbar_init(&fd.bar[0], 1);
+        mbar_init(&fd.bar[1], 1);
+        next = a.ws.chunk_desc[blockIdx.x % n_chunks];
+        feed_issue(fd, fa, a.ws, n_chunks, 0, next, true);
     }
-    const uint64_t base = (uint64_t)u * a.client_stride + d.elem0;
-    const bool full = d.cnt == (uint32_t)kC && ((reinterpret_cast<uintptr_t>(a.grad + base) | reinterpret_cast<uintptr_t>(a.mem + base)) & 15u) == 0 &&
-                      (!kSym || (reinterpret_cast<uintptr_t>(a.sym_out + base) & 7u) == 0);
+    if (kHist)
+        for (uint32_t i = tid; i < (uint32_t)(kHistStride * kHistCopies); i += kThreads) s_hist[i] = 0;
+    __syncthreads();
+    feed_fetch_fmt(fd, a.ws, 0);
+    __syncthreads();
+
+    uint32_t n_sat = 0, n_nf = 0, hist_seg = 0xffffffffu, cur_client = 0, parity = 0;
+    bool hw_fail = false;
     const uint32_t i0 = tid * 8;
-    const uint32_t nv = d.cnt > i0 ? min(8u, d.cnt - i0) : 0u;
-    uint32_t n_sat = 0, n_nf = 0;
-    uint32_t s[8];
-    const uint64_t e = base + i0;
-    if (full) {
-        convert8<true>(a.grad + e, a.mem + e, 8, a.decay, f, s, n_sat, n_nf);
-        if (kSym) *reinterpret_cast<uint2*>(a.sym_out + e) = pack_sym8(s);
-    } else if (nv) {
-        convert8<false>(a.grad + e, a.mem + e, nv, a.decay, f, s, n_sat, n_nf);
-        if (kSym) {
+    for (uint64_t k = 0;; ++k) {
+        if (tid == 0) feed_issue(fd, fa, a.ws, n_chunks, k + 1, next, true);
+        const FeedItem it = fd.item[k & 1u];
+        if (!it.valid) break;
+        if (it.client != cur_client) {  // counters are per client
+            add_counts(&a.res[cur_client], n_sat, n_nf);
+            n_sat = n_nf = 0;
+            cur_client = it.client;
+        }
+        if (kHist && it.d.seg != hist_seg) {  // flush the private histograms when the segment changes
+            __syncthreads();
+            if (hist_seg != 0xffffffffu) {
+                uint32_t c = 0;
+#pragma unroll
+                for (int i = 0; i < kHistCopies; ++i) { c += s_hist[tid + i * kHistStride]; s_hist[tid + i * kHistStride] = 0; }
+                if (c) atomicAdd(reinterpret_cast<unsigned long long*>(&a.hist_out[(size_t)hist_seg * 256 + tid]), (unsigned long long)c);
+            }
+            hist_seg = it.d.seg;
+            __syncthreads();
+        }
+        const FmtDev f = fd.fmt[k & 1u];
+        const uint32_t nv = it.d.cnt > i0 ? min(8u, it.d.cnt - i0) : 0u;
+        float g[8], m[8], mo[8];
+        uint32_t s[8];
+        if (!feed_read(fd, fa, it, k, i0, nv, parity, g, m)) hw_fail = true;
+        const uint64_t e = it.base + i0;
+        if (it.tma) {
+            convert8<true>(g, m, 8, a.decay, f, mo, s, n_sat, n_nf);
+            store8_vec(a.mem + e, mo);
+        } else if (nv) {
+            convert8<false>(g, m, nv, a.decay, f, mo, s, n_sat, n_nf);
+            store8_any(a.mem + e, nv, mo);
+        }
+        if (kSym && nv) {
+            if (nv == 8 && (reinterpret_cast<uintptr_t>(a.sym_out + e) & 7u) == 0) {
+                *reinterpret_cast<uint2*>(a.sym_out + e) = pack_sym8(s);
+            } else {
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+                    if ((uint32_t)j < nv) a.sym_out[e + j] = (uint8_t)s[j];
+            }
+        }
+        if (kHist && nv) {
+            uint32_t* h = s_hist + (tid & (kHistCopies - 1)) * kHistStride;
 #pragma unroll
             for (int j = 0; j < 8; ++j)
-                if ((uint32_t)j < nv) a.sym_out[e + j] = (uint8_t)s[j];
+                if ((uint32_t)j < nv) atomicAdd(&h[s[j]], 1u);
         }
+        feed_fetch_fmt(fd, a.ws, (uint32_t)(k + 1) & 1u);  // item k + 1 was published before the previous barrier
+        __syncthreads();  // everyone has read ring slot k & 1 and item[k & 1] before thread 0 reuses them
     }
-    if (kHist && nv) {
-        uint32_t* h = s_hist + (tid & (kHistCopies - 1)) * kHistStride;
-#pragma unroll
-        for (int j = 0; j < 8; ++j)
-            if ((uint32_t)j < nv) atomicAdd(&h[s[j]], 1u);
-    }
-    add_counts(&a.res[u], n_sat, n_nf);
+    add_counts(&a.res[cur_client], n_sat, n_nf);
     if (kHist) {
         __syncthreads();
-        uint32_t c = 0;
+        if (hist_seg != 0xffffffffu) {
+            uint32_t c = 0;
 #pragma unroll
-        for (int i = 0; i < kHistCopies; ++i) c += s_hist[tid + i * kHistStride];
-        if (c) atomicAdd(reinterpret_cast<unsigned long long*>(&a.hist_out[(size_t)d.seg * 256 + tid]), (unsigned long long)c);
+            for (int i = 0; i < kHistCopies; ++i) c += s_hist[tid + i * kHistStride];
+            if (c) atomicAdd(reinterpret_cast<unsigned long long*>(&a.hist_out[(size_t)hist_seg * 256 + tid]), (unsigned long long)c);
+        }
     }
+    if (__syncthreads_or(hw_fail) && tid == 0) set_status(&a.res[cur_client], CO3_ERR_CUDA);
 }
 
 // ------------------------------------------------------------------------------------------------
-// pack: one block per (chunk, client).  Thread t owns symbols 8t .. 8t+7 of the chunk.
+// pack: persistent blocks over (chunk, client) items.  Thread t owns symbols 8t .. 8t+7 of the chunk.
 // ------------------------------------------------------------------------------------------------
 struct PackArgs {
     const float* grad;   // fused path
@@ -379,6 +515,7 @@ struct PackArgs {
     float decay;
     const uint8_t* sym;  // symbol path
     uint64_t client_stride;
+    uint32_t n_clients;
     uint8_t* streams;
     size_t stream_capacity;
     co3_result* res;
@@ -399,31 +536,52 @@ __device__ __forceinline__ void put_bits(uint32_t* buf, uint32_t end, uint64_t v
     if (w0) atomicOr(&buf[wl - 3], w0);
 }
 
-template <bool kFromSym>
-__global__ void __launch_bounds__(kThreads) pack_kernel(PackArgs a) {
-    __shared__ uint32_t s_enc[256];
-    __shared__ __align__(16) uint32_t s_bits[kSlotWords + 4];
-    __shared__ uint32_t s_scan[8];
-    const Ctrl* ctrl = a.ws.ctrl;
-    if (ctrl->abort) return;
-    const uint32_t chunk = blockIdx.x, u = blockIdx.y, tid = threadIdx.x;
-    if (chunk >= ctrl->n_chunks) return;
-    const ChunkDesc d = a.ws.chunk_desc[chunk];
-    s_enc[tid] = a.ws.enc_lut[d.seg * 256 + tid];
-    reinterpret_cast<uint4*>(s_bits)[tid] = make_uint4(0, 0, 0, 0);
-    if (tid == 0) reinterpret_cast<uint4*>(s_bits)[kThreads] = make_uint4(0, 0, 0, 0);
-    __syncthreads();
+constexpr int kBitWords = kSlotWords + 4;  // bit buffer of one chunk, multiple of four words
 
-    const uint64_t base = (uint64_t)u * a.client_stride + d.elem0;
-    const uint32_t i0 = tid * 8;
-    const uint32_t nv = d.cnt > i0 ? min(8u, d.cnt - i0) : 0u;
-    const uint64_t e = base + i0;
+// Exclusive prefix sum over the 256 threads of a block with one barrier; *total receives the block sum.
+// scratch: 8 words that no thread writes again before the block's next barrier after this call.
+__device__ __forceinline__ uint32_t block_exclusive_scan_once(uint32_t x, uint32_t* scratch, uint32_t* total) {
+    const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+    uint32_t inc = x;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const uint32_t y = __shfl_up_sync(0xffffffffu, inc, d);
+        if (lane >= (uint32_t)d) inc += y;
+    }
+    if (lane == 31u) scratch[warp] = inc;
+    __syncthreads();
+    uint32_t base = 0, sum = 0;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) {
+        const uint32_t s = scratch[w];
+        if ((uint32_t)w < warp) base += s;
+        sum += s;
+    }
+    *total = sum;
+    return base + inc - x;
+}
+
+struct PackSmem {
+    Feed feed;
+    uint32_t bits[2][kBitWords];
+    uint32_t enc[256];
+    uint32_t scan[2][8];
+};
+
+// One work item of the pack kernel for one thread: symbols of its 8 elements (converted here unless
+// kFromSym), their codewords, the block-wide scan of the lengths, and the bits ORed into the chunk's buffer.
+// kWhole: the chunk is complete (and, on the fused path, was delivered through the ring).
+// Returns the chunk's total bit count; `missing` reports a symbol without codeword.
+template <bool kFromSym, bool kWhole>
+__device__ __forceinline__ uint32_t pack_item(const PackArgs& a, PackSmem& sm, const FeedArgs& fa, const FeedItem& it,
+                                              uint64_t k, uint32_t& parity, uint32_t& enc_seg, uint32_t& n_sat,
+                                              uint32_t& n_nf, bool& hw_fail, bool& missing, uint32_t& off_out) {
+    const uint32_t tid = threadIdx.x, i0 = tid * 8;
+    const uint32_t nv = kWhole ? 8u : (it.d.cnt > i0 ? min(8u, it.d.cnt - i0) : 0u);
+    const uint64_t e = it.base + i0;
     uint32_t s[8];
-    uint32_t n_sat = 0, n_nf = 0;
-    bool full;
     if (kFromSym) {
-        full = d.cnt == (uint32_t)kC && (reinterpret_cast<uintptr_t>(a.sym + base) & 7u) == 0;
-        if (full) {
+        if (kWhole && (reinterpret_cast<uintptr_t>(a.sym + e) & 7u) == 0) {
             const uint2 w = __ldg(reinterpret_cast<const uint2*>(a.sym + e));
 #pragma unroll
             for (int j = 0; j < 4; ++j) { s[j] = (w.x >> (8 * j)) & 0xffu; s[4 + j] = (w.y >> (8 * j)) & 0xffu; }
@@ -432,18 +590,23 @@ __global__ void __launch_bounds__(kThreads) pack_kernel(PackArgs a) {
             for (int j = 0; j < 8; ++j) s[j] = (uint32_t)j < nv ? a.sym[e + j] : 0u;
         }
     } else {
-        const FmtDev f = a.ws.fmt[d.seg];
-        full = d.cnt == (uint32_t)kC &&
-               ((reinterpret_cast<uintptr_t>(a.grad + base) | reinterpret_cast<uintptr_t>(a.mem + base)) & 15u) == 0;
-        if (full) convert8<true>(a.grad + e, a.mem + e, 8, a.decay, f, s, n_sat, n_nf);
-        else if (nv) convert8<false>(a.grad + e, a.mem + e, nv, a.decay, f, s, n_sat, n_nf);
+        const FmtDev f = sm.feed.fmt[k & 1u];
+        float g[8], m[8], mo[8];
+        if (!feed_read(sm.feed, fa, it, k, i0, nv, parity, g, m)) hw_fail = true;
+        if (kWhole) {
+            convert8<true>(g, m, 8, a.decay, f, mo, s, n_sat, n_nf);
+            store8_vec(a.mem + e, mo);
+        } else if (nv) {
+            convert8<false>(g, m, nv, a.decay, f, mo, s, n_sat, n_nf);
+            store8_any(a.mem + e, nv, mo);
+        }
     }
     // codewords of this thread's symbols, concatenated in two halves of at most 64 bits
     uint32_t ent[8];
 #pragma unroll
-    for (int j = 0; j < 8; ++j) ent[j] = ((uint32_t)j < nv) ? s_enc[s[j]] : 0u;
+    for (int j = 0; j < 8; ++j) ent[j] = (kWhole || (uint32_t)j < nv) ? sm.enc[s[j]] : 0u;
     const uint32_t any = ent[0] | ent[1] | ent[2] | ent[3] | ent[4] | ent[5] | ent[6] | ent[7];
-    const bool missing = (any & kEncMissing) != 0;
+    missing = (any & kEncMissing) != 0;
     // the low byte of an entry is its length, at most 16: sums of four stay inside the byte
     const uint32_t la = (ent[0] + ent[1] + ent[2] + ent[3]) & 0xffu;
     const uint32_t lb = (ent[4] + ent[5] + ent[6] + ent[7]) & 0xffu;
@@ -454,27 +617,90 @@ __global__ void __launch_bounds__(kThreads) pack_kernel(PackArgs a) {
     const uint64_t wa = ((uint64_t)c01 << ((ent[2] + ent[3]) & 0xffu)) | c23;
     const uint64_t wb = ((uint64_t)c45 << ((ent[6] + ent[7]) & 0xffu)) | c67;
     uint32_t total;
-    const uint32_t off = block_exclusive_scan_256(la + lb, s_scan, &total);
+    const uint32_t off = block_exclusive_scan_once(la + lb, sm.scan[k & 1u], &total);
+    // Behind the scan's barrier every thread has finished the previous item's copy-out and this item's table
+    // look-ups: clear the other bit buffer and fetch the next item's tables.
+    for (uint32_t i = tid; i < (uint32_t)kBitWords / 4; i += kThreads)
+        reinterpret_cast<uint4*>(sm.bits[(k + 1) & 1u])[i] = make_uint4(0, 0, 0, 0);
+    const FeedItem& nx = sm.feed.item[(k + 1) & 1u];
+    if (nx.valid && nx.d.seg != enc_seg) {
+        enc_seg = nx.d.seg;
+        sm.enc[tid] = a.ws.enc_lut[enc_seg * 256 + tid];
+    }
+    if (!kFromSym) feed_fetch_fmt(sm.feed, a.ws, (uint32_t)(k + 1) & 1u);
     if (!missing) {
-        put_bits(s_bits, off + la, wa);
-        put_bits(s_bits, off + la + lb, wb);
+        uint32_t* bits = sm.bits[k & 1u];
+        put_bits(bits, off + la, wa);
+        put_bits(bits, off + la + lb, wb);
     }
-    uint8_t* stream = a.streams + (size_t)u * a.stream_capacity;
-    if ((tid & 15u) == 0)
-        *reinterpret_cast<uint16_t*>(stream + ctrl->sub_off + 2ull * ((uint64_t)chunk * kSubs + (tid >> 4))) = (uint16_t)off;
-    if (!kFromSym) add_counts(&a.res[u], n_sat, n_nf);
-    if (__syncthreads_or(missing)) {
-        if (tid == 0) {
-            set_status(&a.res[u], CO3_ERR_NO_CODEWORD);
-            atomicMin(&a.res[u].first_bad_chunk, chunk);
-            a.ws.client_fail[u] = 1u;
+    off_out = off;
+    return total;
+}
+
+template <bool kFromSym>
+__global__ void __launch_bounds__(kThreads, 4) pack_kernel(PackArgs a) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    PackSmem& sm = *reinterpret_cast<PackSmem*>(smem_raw);
+    const Ctrl* ctrl = a.ws.ctrl;
+    if (ctrl->abort) return;
+    const uint32_t tid = threadIdx.x;
+    const uint32_t n_chunks = ctrl->n_chunks;
+    const FeedArgs fa{a.grad, a.mem, a.client_stride, a.n_clients};
+    if ((uint64_t)blockIdx.x >= (uint64_t)n_chunks * a.n_clients) return;
+
+    ChunkDesc next{};
+    if (tid == 0) {
+        mbar_init(&sm.feed.bar[0], 1);
+        mbar_init(&sm.feed.bar[1], 1);
+        next = a.ws.chunk_desc[blockIdx.x % n_chunks];
+        feed_issue(sm.feed, fa, a.ws, n_chunks, 0, next, !kFromSym);
+    }
+    for (uint32_t i = tid; i < (uint32_t)kBitWords / 4; i += kThreads) reinterpret_cast<uint4*>(sm.bits[0])[i] = make_uint4(0, 0, 0, 0);
+    __syncthreads();
+    uint32_t enc_seg = sm.feed.item[0].valid ? sm.feed.item[0].d.seg : 0u;
+    sm.enc[tid] = a.ws.enc_lut[enc_seg * 256 + tid];
+    feed_fetch_fmt(sm.feed, a.ws, 0);
+    const uint64_t sub_off = ctrl->sub_off;
+    __syncthreads();
+
+    uint32_t n_sat = 0, n_nf = 0, cur_client = 0, parity = 0;
+    bool hw_fail = false;
+    for (uint64_t k = 0;; ++k) {
+        // item k + 1 goes into the ring slot and descriptor that item k - 1 used; every thread is past the
+        // last barrier of item k - 1 and read them before it
+        if (tid == 0) feed_issue(sm.feed, fa, a.ws, n_chunks, k + 1, next, !kFromSym);
+        const FeedItem it = sm.feed.item[k & 1u];
+        if (!it.valid) break;
+        if (!kFromSym && it.client != cur_client) {
+            add_counts(&a.res[cur_client], n_sat, n_nf);
+            n_sat = n_nf = 0;
+            cur_client = it.client;
         }
+        bool missing;
+        uint32_t off, total;
+        const bool whole = kFromSym ? it.d.cnt == (uint32_t)kC : it.tma != 0;
+        if (whole) total = pack_item<kFromSym, true>(a, sm, fa, it, k, parity, enc_seg, n_sat, n_nf, hw_fail, missing, off);
+        else total = pack_item<kFromSym, false>(a, sm, fa, it, k, parity, enc_seg, n_sat, n_nf, hw_fail, missing, off);
+        uint8_t* stream = a.streams + (size_t)it.client * a.stream_capacity;
+        const uint32_t chunk = it.chunk;
+        if ((tid & 15u) == 0)
+            *reinterpret_cast<uint16_t*>(stream + sub_off + 2ull * ((uint64_t)chunk * kSubs + (tid >> 4))) = (uint16_t)off;
+        if (__syncthreads_or(missing)) {  // bit buffer complete
+            if (tid == 0) {
+                set_status(&a.res[it.client], CO3_ERR_NO_CODEWORD);
+                atomicMin(&a.res[it.client].first_bad_chunk, chunk);
+                a.ws.client_fail[it.client] = 1u;
+            }
+        }
+        const size_t ci = (size_t)it.client * a.ws.n_chunks_max + chunk;
+        if (tid == 0) a.ws.chunk_bits[ci] = total;
+        const uint32_t words = (total + 31u) >> 5;
+        uint32_t* slot = a.ws.slots + ci * kSlotWords;
+        const uint32_t* bits = sm.bits[k & 1u];
+        for (uint32_t i = tid; i < words; i += kThreads) slot[i] = bits[i];
     }
-    const size_t ci = (size_t)u * a.ws.n_chunks_max + chunk;
-    if (tid == 0) a.ws.chunk_bits[ci] = total;
-    const uint32_t words = (total + 31u) >> 5;
-    uint32_t* slot = a.ws.slots + ci * kSlotWords;
-    for (uint32_t i = tid; i < words; i += kThreads) slot[i] = s_bits[i];
+    if (!kFromSym) add_counts(&a.res[cur_client], n_sat, n_nf);
+    if (__syncthreads_or(hw_fail) && tid == 0) set_status(&a.res[cur_client], CO3_ERR_CUDA);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -1039,6 +1265,20 @@ uint64_t fixed_part_bound(uint32_t n_seg, uint64_t n_chunks_max) {
         if ((call) != cudaSuccess) return CO3_ERR_CUDA; \
     } while (0)
 
+// Blocks of a persistent kernel: enough to fill every SM at the kernel's occupancy, never more than the work.
+template <typename Kernel>
+int persistent_grid(Kernel kernel, size_t smem, uint64_t items, uint32_t* grid) {
+    int dev = 0, sms = 0, per_sm = 0;
+    CO3_CUDA(cudaGetDevice(&dev));
+    CO3_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    CO3_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    CO3_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kThreads, smem));
+    if (per_sm < 1) return CO3_ERR_CUDA;
+    const uint64_t want = (uint64_t)sms * (uint64_t)per_sm;
+    *grid = (uint32_t)(items < want ? items : want);
+    return CO3_OK;
+}
+
 bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
 
 // Optional per-kernel timing (off by default): an event pair around every launch, read back by
@@ -1149,10 +1389,18 @@ int encode_common(const float* grad, float* mem, float decay, const uint8_t* sym
     const int rc = begin_call(L, ws, res, n_clients, st, sym ? nullptr : fmts, codes, segs, n_seg, n_elem, 1, n_clients);
     if (rc != CO3_OK) return rc;
     if (L.n_chunks_max) {
-        PackArgs pa{grad, mem, decay, sym, client_stride, streams_out, stream_capacity, res, ws};
-        const dim3 grid(L.n_chunks_max, n_clients);
-        if (sym) CO3_LAUNCH(CO3_KERNEL_PACK, st, pack_kernel<true><<<grid, kThreads, 0, st>>>(pa));
-        else CO3_LAUNCH(CO3_KERNEL_PACK, st, pack_kernel<false><<<grid, kThreads, 0, st>>>(pa));
+        PackArgs pa{grad, mem, decay, sym, client_stride, n_clients, streams_out, stream_capacity, res, ws};
+        const uint64_t items = (uint64_t)L.n_chunks_max * n_clients;
+        uint32_t grid = 0;
+        if (sym) {
+            const int g = persistent_grid(pack_kernel<true>, sizeof(PackSmem), items, &grid);
+            if (g != CO3_OK) return g;
+            CO3_LAUNCH(CO3_KERNEL_PACK, st, pack_kernel<true><<<grid, kThreads, sizeof(PackSmem), st>>>(pa));
+        } else {
+            const int g = persistent_grid(pack_kernel<false>, sizeof(PackSmem), items, &grid);
+            if (g != CO3_OK) return g;
+            CO3_LAUNCH(CO3_KERNEL_PACK, st, pack_kernel<false><<<grid, kThreads, sizeof(PackSmem), st>>>(pa));
+        }
     }
     ScanArgs sa{segs, n_seg, n_elem, streams_out, stream_capacity, res, ws};
     CO3_LAUNCH(CO3_KERNEL_SCAN, st, scan_kernel<<<n_clients, kScanThreads, 0, st>>>(sa));
@@ -1235,12 +1483,21 @@ int co3_convert(const float* grad, float* mem, float decay, const co3_fmt* fmts,
     const int rc = begin_call(L, ws, res, n_clients, st, fmts, nullptr, segs, n_seg, n_elem, 1, 1);
     if (rc != CO3_OK) return rc;
     if (L.n_chunks_max == 0) return CO3_OK;
-    ConvertArgs ca{grad, mem, decay, client_stride_elems, sym_out, hist_out, res, ws};
-    const dim3 grid(L.n_chunks_max, n_clients);
-    if (sym_out && hist_out) CO3_LAUNCH(CO3_KERNEL_CONVERT, st, convert_kernel<true, true><<<grid, kThreads, 0, st>>>(ca));
-    else if (sym_out) CO3_LAUNCH(CO3_KERNEL_CONVERT, st, convert_kernel<true, false><<<grid, kThreads, 0, st>>>(ca));
-    else if (hist_out) CO3_LAUNCH(CO3_KERNEL_CONVERT, st, convert_kernel<false, true><<<grid, kThreads, 0, st>>>(ca));
-    else CO3_LAUNCH(CO3_KERNEL_CONVERT, st, convert_kernel<false, false><<<grid, kThreads, 0, st>>>(ca));
+    ConvertArgs ca{grad, mem, decay, client_stride_elems, n_clients, sym_out, hist_out, res, ws};
+    const uint64_t items = (uint64_t)L.n_chunks_max * n_clients;
+    const size_t smem = sizeof(Feed) + (hist_out ? 4 * (size_t)kHistStride * kHistCopies : 0);
+    uint32_t grid = 0;
+#define CO3_CONVERT_CASE(S, H)                                                                                       \
+    {                                                                                                                \
+        const int g = persistent_grid(convert_kernel<S, H>, smem, items, &grid);                                     \
+        if (g != CO3_OK) return g;                                                                                   \
+        CO3_LAUNCH(CO3_KERNEL_CONVERT, st, convert_kernel<S, H><<<grid, kThreads, smem, st>>>(ca));                  \
+    }
+    if (sym_out && hist_out) CO3_CONVERT_CASE(true, true)
+    else if (sym_out) CO3_CONVERT_CASE(true, false)
+    else if (hist_out) CO3_CONVERT_CASE(false, true)
+    else CO3_CONVERT_CASE(false, false)
+#undef CO3_CONVERT_CASE
     return CO3_OK;
 }
 
