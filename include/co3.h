@@ -130,6 +130,31 @@ int co3_convert(const float* grad, float* mem, float decay,
                 void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * co3_convert without a workspace argument (the paper has no counterpart; this exists for the host
+ * program's sake).  Some callers are not allowed to obtain device memory at the point where they run
+ * the conversion: a plug-in inside a server that handed all device memory to its own pool at start-up,
+ * or a latency-bound loop that must never enter the CUDA allocator because an allocation can stall the
+ * whole device.  For them the scratch space is a fixed array of CO3_STATIC_SCRATCH_BYTES inside the
+ * library image (each GPU that loads the library carries one copy until the process ends).  This call,
+ * and everything it calls, performs no cudaMalloc / cudaFree and no other allocating routine; inputs,
+ * outputs and `res` are still the caller's, with the same meaning as in co3_convert.
+ *   - Layouts whose workspace need (co3_workspace_bytes(n_elem, n_seg, 0, ...)) exceeds
+ *     CO3_STATIC_SCRATCH_BYTES are refused with CO3_ERR_CAPACITY before anything is enqueued; the
+ *     18-layer residual network layout (62 segments, 11.2 M elements) fits.
+ *   - The first call on each device looks the array's device address up (with that device current) and
+ *     keeps it; make that first call outside any stream capture.
+ *   - All calls on a device share the one array, which still holds the previous call's tables; whatever
+ *     must start from zero is cleared at the start of each call.  Two calls whose kernels can overlap on
+ *     the GPU (different streams without an ordering between them) race on it: order them.
+ *   - Leave profiling (co3_profile_enable) off if event creation counts as allocation for you.
+ */
+#define CO3_STATIC_SCRATCH_BYTES (2u << 20)
+int co3_convert_static(const float* grad, float* mem, float decay,
+                       const co3_fmt* fmts /* [device] n_seg */, const co3_seg* segs /* [device] n_seg */,
+                       uint32_t n_seg, uint64_t n_elem, uint32_t n_clients, uint64_t client_stride_elems,
+                       uint8_t* sym_out, uint64_t* hist_out, co3_result* res, void* stream);
+
+/*
  * Huffman code for one layer from 256 integer weights (Sec. IV-A (ii)); host function, all
  * pointers [host].  Every symbol fmt can produce takes part with weight max(w, 1); other symbols
  * get length 0.  Ties: a leaf before a merged node, leaves by symbol, merged nodes by age.

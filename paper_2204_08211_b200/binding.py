@@ -43,6 +43,7 @@ def _load():
     L.co3_workspace_bytes.argtypes = [u64, u32, u32, u32, C.POINTER(sz)]
     L.co3_stream_capacity_bytes.argtypes = [u64, u32, u32, C.POINTER(sz)]
     L.co3_convert.argtypes = [vp, vp, f32, vp, vp, u32, u64, u32, u64, vp, vp, vp, vp, sz, vp]
+    L.co3_convert_static.argtypes = [vp, vp, f32, vp, vp, u32, u64, u32, u64, vp, vp, vp, vp]
     L.co3_code_build.argtypes = [vp, vp, vp]
     L.co3_encode.argtypes = [vp, vp, f32, vp, vp, vp, u32, u64, u32, u64, vp, sz, u32, vp, sz, vp, vp]
     L.co3_encode_symbols.argtypes = [vp, vp, vp, u32, u64, u32, u64, vp, sz, u32, vp, sz, vp, vp]
@@ -50,7 +51,7 @@ def _load():
     L.co3_decode.argtypes = [vp, sz, vp, vp, vp, u32, u64, u32, vp, vp, vp, sz, vp, vp]
     L.co3_profile_enable.argtypes = [C.c_int]
     L.co3_profile_read.argtypes = [vp, vp]
-    for name in ("co3_profile_enable", "co3_profile_read", "co3_workspace_bytes", "co3_stream_capacity_bytes", "co3_convert", "co3_code_build", "co3_encode",
+    for name in ("co3_profile_enable", "co3_profile_read", "co3_convert_static", "co3_workspace_bytes", "co3_stream_capacity_bytes", "co3_convert", "co3_code_build", "co3_encode",
                  "co3_encode_symbols", "co3_decode_aggregate", "co3_decode"):
         getattr(L, name).restype = C.c_int
     _lib = L
@@ -144,6 +145,19 @@ def co3_convert(grad, mem, decay, fmts, segs, n_seg, n_elem, n_clients, client_s
                                n_clients, client_stride_elems, _dev(sym_out, True), _dev(hist_out, True),
                                _dev(res), _dev(workspace), workspace.numel() * workspace.element_size(),
                                _stream(stream))
+
+
+STATIC_SCRATCH_BYTES = 2 << 20
+
+
+def co3_convert_static(grad, mem, decay, fmts, segs, n_seg, n_elem, n_clients, client_stride_elems, sym_out, hist_out,
+                       res, stream=None) -> int:
+    """co3_convert on the library's built-in scratch array: no workspace tensor, nothing is allocated.
+    For hosts that may not allocate device memory where they call this; layouts needing more than
+    STATIC_SCRATCH_BYTES of workspace return ERR_CAPACITY.  Calls on one device share the array: order them."""
+    return _load().co3_convert_static(_dev(grad), _dev(mem), float(decay), _dev(fmts), _dev(segs), n_seg, n_elem,
+                                      n_clients, client_stride_elems, _dev(sym_out, True), _dev(hist_out, True),
+                                      _dev(res), _stream(stream))
 
 
 def co3_encode(grad, mem, decay, fmts, codes, segs, n_seg, n_elem, n_clients, client_stride_elems, streams_out,

@@ -1501,6 +1501,47 @@ int co3_convert(const float* grad, float* mem, float decay, const co3_fmt* fmts,
     return CO3_OK;
 }
 
+// ------------------------------------------------------------------------------------------------
+// co3_convert_static: the convert entry point for callers that must not allocate device memory.
+// Its scratch space is the file-scope array below, part of the library image: every device that loads
+// the library holds one copy until the process exits.
+// ------------------------------------------------------------------------------------------------
+static __device__ __align__(256) unsigned char g_static_scratch[CO3_STATIC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+// Device address of g_static_scratch on each device, null until that device's first call.  In host code the
+// array's name is only a handle for cudaGetSymbolAddress, never an address a kernel may use.
+void* g_static_scratch_addr[kMaxDevices];
+
+int static_scratch_address(void** out) {
+    int dev = -1;
+    CO3_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return CO3_ERR_INVALID_ARG;
+    if (g_static_scratch_addr[dev] == nullptr) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || p == nullptr) return CO3_ERR_CUDA;
+        g_static_scratch_addr[dev] = p;
+    }
+    *out = g_static_scratch_addr[dev];
+    return CO3_OK;
+}
+}  // namespace
+
+int co3_convert_static(const float* grad, float* mem, float decay, const co3_fmt* fmts, const co3_seg* segs,
+                       uint32_t n_seg, uint64_t n_elem, uint32_t n_clients, uint64_t client_stride_elems,
+                       uint8_t* sym_out, uint64_t* hist_out, co3_result* res, void* stream) {
+    size_t need = 0;
+    const int rc = co3_workspace_bytes(n_elem, n_seg, 0, CO3_CHUNK_SYMS, &need);
+    if (rc != CO3_OK) return rc;
+    if (need > (size_t)CO3_STATIC_SCRATCH_BYTES) return CO3_ERR_CAPACITY;  // layout too large for the built-in scratch
+    void* scratch = nullptr;
+    const int ra = static_scratch_address(&scratch);
+    if (ra != CO3_OK) return ra;
+    return co3_convert(grad, mem, decay, fmts, segs, n_seg, n_elem, n_clients, client_stride_elems, sym_out, hist_out,
+                       res, scratch, (size_t)CO3_STATIC_SCRATCH_BYTES, stream);
+}
+
 int co3_encode(const float* grad, float* mem, float decay, const co3_fmt* fmts, const co3_code* codes,
                const co3_seg* segs, uint32_t n_seg, uint64_t n_elem, uint32_t n_clients, uint64_t client_stride_elems,
                uint8_t* streams_out, size_t stream_capacity, uint32_t chunk_syms, void* workspace,
