@@ -15,6 +15,14 @@
  *
  * Where the paper is silent the reading taken is stated next to the code (zero and gradual
  * underflow, tie-breaks, length limit, container layout).
+ *
+ * Pins (tests/test_oracle_*.py): library casts to the standard 8/16-bit layouts, the closed forms
+ * of Sec. V-B, exact-rational brute force over the printed level form, the printed bias
+ * polynomials of Sec. IV-B, Kraft equality / entropy bounds / brute-force optimality for the
+ * code, a hand-worked container example.  Parity unpinned (the paper prints nothing to check
+ * them against; only this oracle and the CUDA library agreeing): the order among equal Huffman
+ * weights and the 16-bit length limit, the container layout, the NaN/Inf reading, and the tie
+ * between zero and the smallest normal level when sub-normal levels are flushed.
  */
 #include <math.h>
 #include <stdint.h>

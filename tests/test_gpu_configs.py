@@ -1,0 +1,227 @@
+"""The five workload configurations through the C ABI against the oracle (needs a B200).
+
+Small-scale versions are compared element by element; the full-size launch that bench.py times (config 2:
+10 clients x 11,181,642 elements) is compared on sampled chunks, which the oracle can compute one by one
+because chunks are coded independently, plus properties that hold at any size.
+"""
+import numpy as np
+import pytest
+import torch
+
+import co3_inputs as ci
+import oracle
+import paper_2204_08211_b200 as co3
+from harness import Case, Gpu, oracle_codes, oracle_convert, oracle_encode, oracle_hist, same_bits
+from paper_2204_08211_b200.session import Co3Session
+
+pytestmark = pytest.mark.gpu
+
+
+def _fmts(cfg, sizes, fmt=None):
+    E, M = fmt or cfg["fmt"]
+    return [(E, M, 0) + ci.scale_for(E, M, cfg["beta"][k % len(cfg["beta"])], cfg["alpha"][k % len(cfg["alpha"])])
+            for k in range(len(sizes))]
+
+
+def _grads(cfg, sizes, n_clients, rnd, outliers=False):
+    g = np.zeros((n_clients, sum(sizes)), dtype=np.float32)
+    offs = np.concatenate([[0], np.cumsum(sizes)])
+    for u in range(n_clients):
+        seed = ci.client_round_seed(cfg["seed"], u, rnd)
+        for k, n in enumerate(sizes):
+            g[u, offs[k]:offs[k + 1]] = ci.gennorm(
+                n, cfg["beta"][k % len(cfg["beta"])], cfg["alpha"][k % len(cfg["alpha"])], seed * 1_000_003 + k, "cpu",
+                cfg.get("outlier_frac", 0.0) if outliers else 0.0, cfg.get("outlier_mult", 1.0)).numpy()
+    return g
+
+
+def test_config1_code_fitted_every_round():
+    """1 client, 1e6 elements, [1,4,3], decay 0.9, 4 of the 10 rounds: convert + histogram -> code -> encode symbols."""
+    cfg = ci.config(1)
+    sizes = list(cfg["sizes"])
+    case = Case(sizes, _fmts(cfg, sizes), n_clients=1, decay=cfg["decay"])
+    gpu = Gpu(case)
+    mem_o = np.zeros((1, case.n_elem), dtype=np.float32)
+    mem_g = mem_o.copy()
+    for rnd in range(4):
+        g = _grads(cfg, sizes, 1, rnd)
+        syms, ghats, _, _ = oracle_convert(case, g, mem_o)
+        hist = oracle_hist(case, syms)
+        conv = gpu.convert(g, mem_g)
+        mem_g = conv["mem"]
+        assert np.array_equal(conv["sym"], syms) and same_bits(mem_g, mem_o) and np.array_equal(conv["hist"], hist)
+        st, code = co3.co3_code_build(conv["hist"][0], co3.make_fmts(case.fmts))          # the library's builder
+        ocode = oracle.code_build(hist[0], case.ofmt(0))
+        ln, bits = oracle.code_arrays(ocode)
+        assert st == co3.OK and np.array_equal(code["len"][0], ln) and np.array_equal(code["bits"][0], bits)
+        want = oracle_encode(case, syms, [ocode])[0][1]
+        out = gpu.encode(None, None, [ocode], from_sym=syms)
+        assert np.array_equal(out["streams"][0], want)
+        dec = gpu.decode(out["streams"][0], [ocode])
+        assert dec["res"][0]["status"] == co3.OK
+        assert np.array_equal(dec["sym"][:case.n_elem], syms[0]) and same_bits(dec["ghat"][:case.n_elem], ghats[0])
+
+
+def test_config2_layout_two_clients_three_rounds():
+    """The 62-layer layout at full length with 2 of the 10 clients: everything compared element by element."""
+    cfg = ci.config(2)
+    sizes = list(cfg["sizes"])
+    case = Case(sizes, _fmts(cfg, sizes), n_clients=2, decay=cfg["decay"])
+    gpu = Gpu(case)
+    mem_o = np.zeros((2, case.n_elem), dtype=np.float32)
+    mem_g = mem_o.copy()
+    codes = None
+    for rnd in range(3):
+        g = _grads(cfg, sizes, 2, rnd)
+        syms, _, nsat, _ = oracle_convert(case, g, mem_o)
+        if codes is None:
+            codes = oracle_codes(case, oracle_hist(case, syms))
+        want = oracle_encode(case, syms, codes)
+        out = gpu.encode(g, mem_g, codes)
+        mem_g = out["mem"]
+        assert same_bits(mem_g, mem_o) and np.array_equal(out["res"]["n_saturated"], nsat)
+        for u in range(2):
+            assert np.array_equal(out["streams"][u], want[u][1])
+        agg = gpu.decode_aggregate(out["streams"], codes)
+        st, avg = oracle.decode_aggregate([w[1] for w in want], sizes, [case.ofmt(k) for k in range(case.n_seg)], codes)
+        assert agg["res"][0]["status"] == co3.OK and same_bits(agg["avg"][:case.n_elem], avg)
+
+
+def test_config3_many_clients_batched():
+    """100 clients in one batched encode and one decode-aggregate (layer layout scaled down 64x)."""
+    cfg = ci.config(3)
+    sizes = [max(1, n // 64) for n in cfg["sizes"]]
+    case = Case(sizes, _fmts(cfg, sizes), n_clients=100, decay=cfg["decay"])
+    g = _grads(cfg, sizes, 100, 0)
+    mem_o = np.zeros_like(g)
+    syms, _, _, _ = oracle_convert(case, g, mem_o)
+    codes = oracle_codes(case, oracle_hist(case, syms))
+    want = oracle_encode(case, syms, codes)
+    gpu = Gpu(case)
+    out = gpu.encode(g, np.zeros_like(g), codes)
+    assert same_bits(out["mem"], mem_o)
+    for u in range(100):
+        assert np.array_equal(out["streams"][u], want[u][1])
+    agg = gpu.decode_aggregate(out["streams"], codes)
+    st, avg = oracle.decode_aggregate([w[1] for w in want], sizes, [case.ofmt(k) for k in range(case.n_seg)], codes)
+    assert agg["res"][0]["status"] == co3.OK and same_bits(agg["avg"][:case.n_elem], avg)
+
+
+def test_config4_format_shape_decay_sweep():
+    """All 36 cells of the sweep at 200k elements, 2 rounds each."""
+    cfg = ci.config(4)
+    n = 200_000
+    for cell in cfg["cells"]:
+        E, M = cell["fmt"]
+        c = dict(cfg, beta=(cell["beta"],))
+        case = Case([n], _fmts(c, [n], (E, M)), n_clients=1, decay=cell["decay"])
+        gpu = Gpu(case)
+        mem_o = np.zeros((1, n), dtype=np.float32)
+        mem_g = mem_o.copy()
+        codes = None
+        for rnd in range(2):
+            g = _grads(c, [n], 1, rnd)
+            syms, ghats, nsat, _ = oracle_convert(case, g, mem_o)
+            if codes is None:
+                codes = oracle_codes(case, oracle_hist(case, syms))
+            out = gpu.encode(g, mem_g, codes)
+            mem_g = out["mem"]
+            assert same_bits(mem_g, mem_o), cell
+            assert np.array_equal(out["streams"][0], oracle_encode(case, syms, codes)[0][1]), cell
+            assert out["res"][0]["n_saturated"] == nsat[0]
+            dec = gpu.decode(out["streams"][0], codes, want_sym=False)
+            assert same_bits(dec["ghat"][:n], ghats[0]), cell
+
+
+def test_config5_outliers_and_eight_clients():
+    """GenNorm(0.8) with 0.01 % outliers at 100x scale: 3M elements x 1 client and 400k x 8 clients, 3 rounds."""
+    cfg = ci.config(5)
+    for n, clients in ((3_000_000, 1), (400_000, 8)):
+        case = Case([n], _fmts(cfg, [n]), n_clients=clients, decay=cfg["decay"])
+        gpu = Gpu(case)
+        mem_o = np.zeros((clients, n), dtype=np.float32)
+        mem_g = mem_o.copy()
+        codes = None
+        for rnd in range(3):
+            g = _grads(cfg, [n], clients, rnd, outliers=True)
+            syms, _, nsat, _ = oracle_convert(case, g, mem_o)
+            if codes is None:
+                codes = oracle_codes(case, oracle_hist(case, syms))
+            want = oracle_encode(case, syms, codes)
+            out = gpu.encode(g, mem_g, codes)
+            mem_g = out["mem"]
+            assert same_bits(mem_g, mem_o) and np.array_equal(out["res"]["n_saturated"], nsat)
+            for u in range(clients):
+                assert np.array_equal(out["streams"][u], want[u][1])
+            agg = gpu.decode_aggregate(out["streams"], codes)
+            st, avg = oracle.decode_aggregate([w[1] for w in want], [n], [case.ofmt(0)], codes)
+            assert same_bits(agg["avg"][:n], avg)
+
+
+def test_config2_full_size_sampled_chunks():
+    """The launch bench.py times (10 clients x 11,181,642 elements, second round so that memory is live):
+    sampled chunks against the oracle, and size-independent properties of the streams."""
+    import bench
+    cfg, sizes, fmts, clients = bench.workload(2)
+    sess = Co3Session(sizes, fmts, clients, cfg["decay"], "cuda")
+    g0 = bench.make_grads(cfg, sizes, clients, sess.stride, 0, "cuda")
+    g1 = bench.make_grads(cfg, sizes, clients, sess.stride, 1, "cuda")
+    mems = sess.new_client_buffer()
+    hist = sess.histogram(g0, sess.new_client_buffer())
+    assert int(hist.sum()) == sess.n_elem * clients
+    sess.set_codes_from_weights(hist)
+    sess.encode(g0, mems)
+    mem_before = mems.clone()
+    sess.encode(g1, mems)
+    avg = sess.decode_aggregate().clone()
+    torch.cuda.synchronize()
+    res = sess.encode_results()
+    assert (res["status"] == co3.OK).all() and sess.decode_result()["status"][0] == co3.OK
+
+    C = co3.CHUNK_SYMS
+    ofmts = [oracle.Fmt(E, M, 0, s, inv) for (E, M, _, s, inv) in fmts]
+    ocodes = [oracle.make_code(sess.codes_host[k]["len"], sess.codes_host[k]["bits"]) for k in range(len(sizes))]
+    seg_first = np.concatenate([[0], np.cumsum([(n + C - 1) // C for n in sizes])])
+    seg_off = np.concatenate([[0], np.cumsum(sizes)])
+    n_chunks = int(seg_first[-1])
+    al = lambda x: (x + 15) & ~15
+    chunk_off = al(64 + 24 * len(sizes))
+    sub_off = al(chunk_off + 8 * (n_chunks + 1))
+    pay_off = al(sub_off + 32 * n_chunks)
+    rng = np.random.default_rng(0)
+    picks = sorted(set(int(c) for c in rng.integers(0, n_chunks, size=24)) | {0, n_chunks - 1, int(seg_first[1]) - 1})
+    streams = [sess.stream_bytes(u) for u in range(clients)]
+    for u in range(clients):
+        s = streams[u]
+        assert int(s[40:48].view(np.uint64)[0]) * 4 + pay_off <= s.size == res[u]["container_bytes"]
+        wo = s[chunk_off:chunk_off + 8 * (n_chunks + 1)].view(np.uint64)
+        assert wo[0] == 0 and (np.diff(wo.astype(np.int64)) >= 0).all() and wo[-1] == s[40:48].view(np.uint64)[0]
+        segbits = s[64:64 + 24 * len(sizes)].view(np.uint64).reshape(-1, 3)
+        assert np.array_equal(segbits[:, 0], np.array(sizes, dtype=np.uint64))
+        assert int(segbits[:, 2].sum()) == res[u]["payload_bits"] == int(s[48:56].view(np.uint64)[0])
+    for c in picks:
+        k = int(np.searchsorted(seg_first, c, side="right") - 1)
+        start = (c - int(seg_first[k])) * C
+        cnt = min(C, sizes[k] - start)
+        lo = int(seg_off[k]) + start
+        ghat_sum = None
+        for u in range(clients):
+            base = u * sess.stride + lo
+            g = g1[base:base + cnt].cpu().numpy()
+            m = mem_before[base:base + cnt].cpu().numpy().copy()
+            r = oracle.convert(g, m, cfg["decay"], ofmts[k])
+            assert same_bits(mems[base:base + cnt].cpu().numpy(), m)
+            st, want = oracle.encode(r["sym"], [cnt], [ocodes[k]])
+            assert st == oracle.OK
+            # the oracle's one-chunk stream: its payload and sub-chunk offsets are this chunk's
+            w_pay = al(al(al(64 + 24) + 16) + 32)
+            s = streams[u]
+            wo = s[chunk_off + 8 * c:chunk_off + 8 * c + 16].view(np.uint64)
+            nwords = int(want[40:48].view(np.uint64)[0])
+            assert int(wo[1] - wo[0]) == nwords
+            assert np.array_equal(s[pay_off + 4 * int(wo[0]):pay_off + 4 * int(wo[1])], want[w_pay:w_pay + 4 * nwords])
+            assert np.array_equal(s[sub_off + 32 * c:sub_off + 32 * c + 32], want[al(al(64 + 24) + 16):al(al(64 + 24) + 16) + 32])
+            gh = r["ghat"]
+            ghat_sum = gh.copy() if ghat_sum is None else (ghat_sum + gh).astype(np.float32)
+        want_avg = (ghat_sum / np.float32(clients)).astype(np.float32)
+        assert same_bits(avg[lo:lo + cnt].cpu().numpy(), want_avg)
