@@ -26,6 +26,23 @@ if ROOT not in sys.path:
 
 METRIC = "co3_encode_decode_aggregate_throughput"
 UNIT = "gradient elements/s"
+RANK_SEED_STRIDE = 100_000   # ranks draw their synthetic clients from disjoint seed ranges
+
+
+def max_over_ranks(ms: float, world: int, device) -> float:
+    """Step time of the job: the slowest rank's."""
+    if world <= 1:
+        return ms
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def elements_per_step(n_elem: int, clients_per_rank: int, world: int) -> int:
+    """Whole-job work of one step: every rank encodes and aggregates its own clients (weak scaling)."""
+    return n_elem * clients_per_rank * world
 
 
 def load_peaks():
@@ -59,7 +76,7 @@ def make_grads(cfg, sizes, n_clients, stride, rnd, device, rank=0):
     import co3_inputs as ci
     out = torch.zeros(n_clients * stride, dtype=torch.float32, device=device)
     for u in range(n_clients):
-        seed = ci.client_round_seed(cfg["seed"] + 100_000 * rank, u, rnd)
+        seed = ci.client_round_seed(cfg["seed"] + RANK_SEED_STRIDE * rank, u, rnd)
         off = u * stride
         for k, n in enumerate(sizes):
             out[off:off + n] = ci.gennorm(int(n), float(cfg["beta"][k]), float(cfg["alpha"][k]),
@@ -161,22 +178,32 @@ def oracle_step(cfg, sizes, fmts, n_clients, codes=None):
 
 
 def run_reference(args):
+    """The CPU oracle as the reference arm: each step pushes a bounded sample of the workload (one client, the
+    leading layers) through convert + encode + decode-aggregate on one host core."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
     cfg, sizes, fmts, clients = workload(args.config)
-    sample_clients = 1
-    codes = None
-    _, _, codes = oracle_step(cfg, sizes, fmts, sample_clients, None)
+    # size the sample so that the whole run stays near two minutes: the oracle does about 6e6 elements/s
+    budget_s = 100.0 / max(1, args.steps + args.warmup)
+    target = max(200_000, int(6.0e6 * budget_s))
+    n_layers, acc = 0, 0
+    while n_layers < len(sizes) and (n_layers == 0 or acc + sizes[n_layers] <= target):
+        acc += sizes[n_layers]
+        n_layers += 1
+    sub_sizes, sub_fmts = list(sizes[:n_layers]), fmts[:n_layers]
+    sub_cfg = dict(cfg, beta=cfg["beta"][:n_layers], alpha=cfg["alpha"][:n_layers])
+    _, _, codes = oracle_step(sub_cfg, sub_sizes, sub_fmts, 1, None)
     for _ in range(max(0, args.warmup - 1)):
-        oracle_step(cfg, sizes, fmts, sample_clients, codes)
+        oracle_step(sub_cfg, sub_sizes, sub_fmts, 1, codes)
     elems, secs = 0, 0.0
     for _ in range(args.steps):
-        e, dt, _ = oracle_step(cfg, sizes, fmts, sample_clients, codes)
+        e, dt, _ = oracle_step(sub_cfg, sub_sizes, sub_fmts, 1, codes)
         elems += e
         secs += dt
     value = elems / secs
-    sample = "%d of %d clients per step, full layer layout (%d elements each)" % (sample_clients, clients, sum(sizes))
+    sample = "1 of %d clients, first %d of %d layers (%d of %d elements) per step" % (
+        clients, n_layers, len(sizes), sum(sub_sizes), sum(sizes))
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * secs / args.steps,
@@ -251,11 +278,8 @@ def run_ours(args):
     ms = e0.elapsed_time(e1)
     clocks = sampler.stop() if rank == 0 else None
     er, dr = check()
-    if world > 1:
-        t = torch.tensor([ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
-    elems_per_step = sess.n_elem * clients * world
+    ms = max_over_ranks(ms, world, dev)
+    elems_per_step = elements_per_step(sess.n_elem, clients, world)
     value = elems_per_step * args.steps / (ms * 1e-3)
 
     # ---- per-kernel times: a second pass of the same steps with an event pair around every launch
@@ -266,6 +290,27 @@ def run_ours(args):
     prof = co3.co3_profile_read()
     co3.co3_profile_enable(False)
     launches_per_step = sum(n for n, _ in prof.values()) // args.steps
+
+    # ---- the stand-alone correct + convert + memory kernel (the flow that fits the code between conversion and
+    # coding), timed the same way outside the step: with symbols out, and with symbols and histogram out
+    sym_buf = sess.new_client_buffer(torch.uint8)
+    mems_k1 = sess.new_client_buffer()
+    k1 = {}
+    for name, hist_buf in (("convert", None), ("convert_hist", sess.hist)):
+        for i in range(args.warmup + args.steps):
+            if i == args.warmup:
+                torch.cuda.synchronize()
+                co3.co3_profile_enable(True)
+            st = co3.co3_convert(grads[i % n_rounds], mems_k1, sess.decay, sess.fmts, sess.segs, sess.n_seg, sess.n_elem,
+                                 clients, sess.stride, sym_buf, hist_buf, sess.res_enc, sess.workspace, stream)
+            if st != co3.OK:
+                raise RuntimeError("co3_convert: " + co3.co3_status_string(st))
+        torch.cuda.synchronize()
+        k1[name] = co3.co3_profile_read()["convert"]
+        co3.co3_profile_enable(False)
+    check_enc = sess.encode_results()
+    if (check_enc["status"] != co3.OK).any():
+        raise RuntimeError("device status after co3_convert: %s" % check_enc["status"])
 
     # ---- end to end: pinned host gradients in, averaged gradient out, every step
     host_g = [torch.empty(clients * sess.stride, dtype=torch.float32).pin_memory() for _ in range(n_rounds)]
@@ -288,10 +333,7 @@ def run_ours(args):
     e1.record(stream)
     barrier()
     e2e_ms = e0.elapsed_time(e1)
-    if world > 1:
-        t = torch.tensor([e2e_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
+    e2e_ms = max_over_ranks(e2e_ms, world, dev)
     check()
     e2e_value = elems_per_step * e2e_steps / (e2e_ms * 1e-3)
 
@@ -320,7 +362,13 @@ def run_ours(args):
             k["achieved_gbs"] = alg_bytes[name] / 1e9 / (avg_ms * 1e-3)
             k["frac_of_peak"] = k["achieved_gbs"] / peak
         kernels[name] = k
-    dom = max((k for k in kernels if k in alg_bytes), key=lambda k: kernels[k]["avg_ms"] * kernels[k]["launches_per_step"])
+    for name, (n, tot) in k1.items():
+        avg_ms = tot / n
+        gb = alg_bytes["convert"] / 1e9
+        kernels[name] = {"launches_per_step": 0, "avg_ms": avg_ms, "algorithmic_gb_per_launch": gb,
+                         "achieved_gbs": gb / (avg_ms * 1e-3), "frac_of_peak": gb / (avg_ms * 1e-3) / peak,
+                         "note": "stand-alone co3_convert over the same batch, outside the timed step"}
+    dom = max((k for k in ("pack", "decode")), key=lambda k: kernels[k]["avg_ms"] * kernels[k]["launches_per_step"])
     roofline = {"kernel": dom + "_kernel", "bound": "hbm", "achieved": kernels[dom]["achieved_gbs"], "peak": peak,
                 "unit": "GB/s", "frac": kernels[dom]["frac_of_peak"], "traffic": None, "peak_source": peak_src,
                 "timed": "second pass of the same steps with CUDA events around every launch"}
@@ -329,9 +377,11 @@ def run_ours(args):
     # ---- CPU baseline: the oracle on a bounded sample (one client, full layer layout)
     cpu = None
     if not args.no_cpu_baseline:
-        elems, secs, _ = oracle_step(cfg, sizes, fmts, 1, None)
+        n_cpu = min(2, clients)
+        elems, secs, _ = oracle_step(cfg, sizes, fmts, n_cpu, None)
         cpu = {"value": elems / secs, "unit": UNIT, "cores": 1, "kind": "oracle",
-               "sample": "1 of %d clients, full layer layout (%d elements): convert + encode + decode" % (clients, sess.n_elem)}
+               "sample": "%d of %d clients, full layer layout (%d elements each): convert + encode + decode-aggregate, "
+                         "%.1f s" % (n_cpu, clients, sess.n_elem, secs)}
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
@@ -357,8 +407,8 @@ def run_ours(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
-    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=2)
     ap.add_argument("--clients", type=int, default=None, help="override the clients per GPU (profiling small cases)")
