@@ -797,19 +797,29 @@ __global__ void __launch_bounds__(kScanThreads) scan_kernel(ScanArgs a) {
     }
 }
 
-// compact: one block per (chunk, client) moves the chunk's words to their final position.
+// compact: moves the chunks' words from their slots to their final positions; one warp per chunk, eight
+// chunks of one client per block, loads batched eight deep.
 __global__ void __launch_bounds__(kThreads) compact_kernel(ScanArgs a) {
     const Ctrl* ctrl = a.ws.ctrl;
     if (ctrl->abort) return;
-    const uint32_t chunk = blockIdx.x, u = blockIdx.y, tid = threadIdx.x;
+    const uint32_t u = blockIdx.y, lane = threadIdx.x & 31u;
+    const uint32_t chunk = blockIdx.x * (kThreads / 32) + (threadIdx.x >> 5);
     if (chunk >= ctrl->n_chunks || a.ws.client_fail[u]) return;
     uint8_t* stream = a.streams + (size_t)u * a.stream_capacity;
     const uint64_t w0 = reinterpret_cast<const uint64_t*>(stream + ctrl->chunk_off)[chunk];
     const size_t ci = (size_t)u * a.ws.n_chunks_max + chunk;
     const uint32_t words = (a.ws.chunk_bits[ci] + 31u) >> 5;
-    const uint32_t* slot = a.ws.slots + ci * kSlotWords;
-    uint32_t* dst = reinterpret_cast<uint32_t*>(stream + ctrl->payload_off) + w0;
-    for (uint32_t i = tid; i < words; i += kThreads) dst[i] = slot[i];
+    const uint32_t* __restrict__ slot = a.ws.slots + ci * kSlotWords;
+    uint32_t* __restrict__ dst = reinterpret_cast<uint32_t*>(stream + ctrl->payload_off) + w0;
+    uint32_t i = lane;
+    for (; i + 7 * 32 < words; i += 8 * 32) {
+        uint32_t v[8];
+#pragma unroll
+        for (int r = 0; r < 8; ++r) v[r] = __ldg(slot + i + r * 32);
+#pragma unroll
+        for (int r = 0; r < 8; ++r) dst[i + r * 32] = v[r];
+    }
+    for (; i < words; i += 32) dst[i] = __ldg(slot + i);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -1405,7 +1415,7 @@ int encode_common(const float* grad, float* mem, float decay, const uint8_t* sym
     ScanArgs sa{segs, n_seg, n_elem, streams_out, stream_capacity, res, ws};
     CO3_LAUNCH(CO3_KERNEL_SCAN, st, scan_kernel<<<n_clients, kScanThreads, 0, st>>>(sa));
     if (L.n_chunks_max) {
-        CO3_LAUNCH(CO3_KERNEL_COMPACT, st, compact_kernel<<<dim3(L.n_chunks_max, n_clients), kThreads, 0, st>>>(sa));
+        CO3_LAUNCH(CO3_KERNEL_COMPACT, st, compact_kernel<<<dim3((L.n_chunks_max + kThreads / 32 - 1) / (kThreads / 32), n_clients), kThreads, 0, st>>>(sa));
     }
     return CO3_OK;
 }
