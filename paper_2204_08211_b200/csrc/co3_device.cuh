@@ -19,8 +19,8 @@ constexpr int kSubBits = CO3_MAX_CODE_LEN - kDecBits;        // second-level tab
 constexpr int kSubLut = 256 << kSubBits;                     // at most 256 second-level tables per segment
 constexpr uint32_t kEncMissing = 0x80000000u;                // encode table entry of a symbol without codeword
 constexpr uint32_t kDecLong = 0x8000u;                       // decode table entry: look in a second-level table
-constexpr uint32_t kDecInvalid = 0x4100u;                    // decode table entry: no codeword (consumes one bit)
-constexpr uint32_t kDecErrBit = 0x4000u;
+constexpr uint32_t kDecInvalid = 0x01ffu;                    // decode table entry: no codeword; consumes one bit and
+                                                             // yields 0xff, which is a symbol of no format
 constexpr uint32_t kMagic = 0x53334F43u;                     // 'C','O','3','S'
 constexpr uint32_t kHeaderBytes = 64;
 constexpr int kThreads = 256;

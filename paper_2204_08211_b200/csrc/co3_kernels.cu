@@ -182,6 +182,7 @@ __global__ void __launch_bounds__(kThreads) prepare_kernel(PrepArgs a) {
         if (tid == 0) s_kraft = 0;
         __syncthreads();
         if (len > CO3_MAX_CODE_LEN || (len && (bits >> len))) code_ok = false;
+        if (tid == 255 && len) code_ok = false;  // 0xff is a symbol of no format: the decoder uses it as its error mark
         if (code_ok && len) atomicAdd(&s_kraft, 1u << (CO3_MAX_CODE_LEN - len));
         a.ws.enc_lut[k * 256 + tid] = (code_ok && len) ? ((bits << 8) | len) : kEncMissing;
         uint16_t* lut = a.ws.dec_lut + (size_t)k * kDecLut;
@@ -945,17 +946,20 @@ struct BitReader {
     __device__ __forceinline__ uint32_t position() const { return next * 32u - (uint32_t)have; }
 };
 
-// Decodes one symbol and returns its table entry (symbol in the low byte); `seen` collects the entries so
-// that the invalid flag can be tested once per sub-chunk.
+// Second-level look-up for a codeword longer than the first table's index; rare, kept out of line so that
+// the common path carries none of its instructions.
+__device__ __noinline__ uint32_t decode_long(const uint16_t* __restrict__ sub_tab, uint32_t ent, uint32_t top) {
+    return __ldg(sub_tab + ((ent & 0xffu) << kSubBits) + ((top >> (32 - CO3_MAX_CODE_LEN)) & ((1u << kSubBits) - 1u)));
+}
+
+// Decodes one symbol and returns its table entry: symbol in the low byte (0xff = no codeword matched).
 template <bool kChecked>
 __device__ __forceinline__ uint32_t decode_one(BitReader<kChecked>& br, const uint16_t* __restrict__ s_lut,
-                                               const uint16_t* __restrict__ sub_tab, uint32_t& seen) {
+                                               const uint16_t* __restrict__ sub_tab) {
     const uint32_t top = (uint32_t)(br.buf >> 32);
     uint32_t ent = s_lut[top >> (32 - kDecBits)];
-    if (ent & kDecLong)  // codeword longer than the table index: second level, by the next four bits
-        ent = __ldg(sub_tab + ((ent & 0xffu) << kSubBits) + ((top >> (32 - CO3_MAX_CODE_LEN)) & ((1u << kSubBits) - 1u)));
-    seen |= ent;
-    const uint32_t len = (ent >> 8) & 0x1fu;
+    if (ent >= kDecLong) ent = decode_long(sub_tab, ent, top);
+    const uint32_t len = ent >> 8;
     br.buf <<= len;
     br.have -= (int)len;
     return ent;
@@ -969,22 +973,23 @@ __device__ __forceinline__ uint32_t decode_sub(const uint32_t* words, uint32_t n
                                                uint32_t* row, uint32_t rot, bool& err) {
     BitReader<kChecked> br;
     br.init(words, nwords, off);
-    uint32_t seen = 0;
+    uint32_t marks = 0;  // collects, per byte lane, whether some symbol byte was 0xff
 #pragma unroll 2
     for (uint32_t j = 0; j < 32; ++j) {
         uint32_t w = 0;
         if (kWhole || j * 4 < my) {
             br.refill();
-            const uint32_t e0 = decode_one(br, s_lut, sub_tab, seen);
-            const uint32_t e1 = (kWhole || j * 4 + 1 < my) ? decode_one(br, s_lut, sub_tab, seen) : 0u;
+            const uint32_t e0 = decode_one(br, s_lut, sub_tab);
+            const uint32_t e1 = (kWhole || j * 4 + 1 < my) ? decode_one(br, s_lut, sub_tab) : 0u;
             br.refill();
-            const uint32_t e2 = (kWhole || j * 4 + 2 < my) ? decode_one(br, s_lut, sub_tab, seen) : 0u;
-            const uint32_t e3 = (kWhole || j * 4 + 3 < my) ? decode_one(br, s_lut, sub_tab, seen) : 0u;
+            const uint32_t e2 = (kWhole || j * 4 + 2 < my) ? decode_one(br, s_lut, sub_tab) : 0u;
+            const uint32_t e3 = (kWhole || j * 4 + 3 < my) ? decode_one(br, s_lut, sub_tab) : 0u;
             w = __byte_perm(__byte_perm(e0, e1, 0x0040), __byte_perm(e2, e3, 0x0040), 0x5410);
+            marks |= (~w - 0x01010101u) & w;  // bit 7 of a byte survives iff that byte of ~w is zero
         }
         row[(j + rot) & 31u] = w;
     }
-    if (seen & kDecErrBit) err = true;
+    if (marks & 0x80808080u) err = true;
     return br.position();
 }
 
