@@ -26,6 +26,9 @@ if ROOT not in sys.path:
 
 METRIC = "co3_encode_decode_aggregate_throughput"
 UNIT = "gradient elements/s"
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch, from the ncu captures summarised under profiles/
+# (config 2, 10 clients).  Only meaningful for that workload and for the kernels as they were captured.
+NCU_TRAFFIC_BYTES = {"pack": 1403.7e6, "decode": 117.0e6, "convert": 1406.1e6}
 RANK_SEED_STRIDE = 100_000   # ranks draw their synthetic clients from disjoint seed ranges
 
 
@@ -389,7 +392,10 @@ def run_ours(args):
                          "note": "stand-alone call over the same data, outside the timed step"}
     dom = max((k for k in ("pack", "decode")), key=lambda k: kernels[k]["avg_ms"] * kernels[k]["launches_per_step"])
     roofline = {"kernel": dom + "_kernel", "bound": "hbm", "achieved": kernels[dom]["achieved_gbs"], "peak": peak,
-                "unit": "GB/s", "frac": kernels[dom]["frac_of_peak"], "traffic": None, "peak_source": peak_src,
+                "unit": "GB/s", "frac": kernels[dom]["frac_of_peak"],
+                "traffic": NCU_TRAFFIC_BYTES.get(dom) if (args.config == 2 and clients == 10) else None,
+                "traffic_unit": "bytes per launch (ncu dram__bytes_read.sum + dram__bytes_write.sum)",
+                "algorithmic_bytes_per_launch": alg_bytes[dom], "peak_source": peak_src,
                 "timed": "second pass of the same steps with CUDA events around every launch"}
     bits = float(er["payload_bits"].astype(np.float64).sum())
 
