@@ -913,56 +913,48 @@ __device__ __forceinline__ uint32_t sym_slot(uint32_t p, uint32_t s, uint32_t j)
     return s * 32u + ((j + s + 16u * (p & 1u)) & 31u);
 }
 
-// Sequential reader of one sub-chunk: a 64-bit window over the chunk's words.
-// kChecked: reads beyond the chunk return 0 (needed when the words are read in place from global memory);
-// otherwise the words sit in shared memory with kPaySlack readable words behind them.
-template <bool kChecked>
-struct BitReader {
-    const uint32_t* base;
-    uint32_t nwords;
-    uint32_t next;  // next word to fetch
-    uint64_t buf;   // unread bits, left-aligned
-    int have;       // number of valid bits in buf
-
-    __device__ __forceinline__ uint32_t word(uint32_t i) const {
-        if (kChecked) return i < nwords ? __ldg(base + i) : 0u;
-        return base[i];
-    }
-    __device__ __forceinline__ void init(const uint32_t* b, uint32_t n, uint32_t bit_off) {
-        base = b;
-        nwords = n;
-        const uint32_t w = bit_off >> 5, sh = bit_off & 31u;
-        buf = (((uint64_t)word(w) << 32) | word(w + 1)) << sh;
-        have = 64 - (int)sh;
-        next = w + 2;
-    }
-    __device__ __forceinline__ void refill() {  // keeps at least 32 valid bits
-        if (have <= 32) {
-            buf |= (uint64_t)word(next) << (32 - have);
-            ++next;
-            have += 32;
-        }
-    }
-    __device__ __forceinline__ uint32_t position() const { return next * 32u - (uint32_t)have; }
-};
-
 // Second-level look-up for a codeword longer than the first table's index; rare, kept out of line so that
-// the common path carries none of its instructions.
-__device__ __noinline__ uint32_t decode_long(const uint16_t* __restrict__ sub_tab, uint32_t ent, uint32_t top) {
-    return __ldg(sub_tab + ((ent & 0xffu) << kSubBits) + ((top >> (32 - CO3_MAX_CODE_LEN)) & ((1u << kSubBits) - 1u)));
+// the common path carries none of its instructions.  `win` holds the stream bits from the codeword's start.
+__device__ __noinline__ uint32_t decode_long(const uint16_t* __restrict__ sub_tab, uint32_t ent, uint32_t win) {
+    return __ldg(sub_tab + ((ent & 0xffu) << kSubBits) + ((win >> (32 - CO3_MAX_CODE_LEN)) & ((1u << kSubBits) - 1u)));
 }
 
-// Decodes one symbol and returns its table entry: symbol in the low byte (0xff = no codeword matched).
+// The 32 stream bits that start at bit `pos` of the chunk.
+// kChecked: words beyond the chunk read as 0 (needed when the words are read in place from global memory);
+// otherwise the words sit in shared memory with kPaySlack readable words behind them.
 template <bool kChecked>
-__device__ __forceinline__ uint32_t decode_one(BitReader<kChecked>& br, const uint16_t* __restrict__ s_lut,
-                                               const uint16_t* __restrict__ sub_tab) {
-    const uint32_t top = (uint32_t)(br.buf >> 32);
-    uint32_t ent = s_lut[top >> (32 - kDecBits)];
-    if (ent >= kDecLong) ent = decode_long(sub_tab, ent, top);
-    const uint32_t len = ent >> 8;
-    br.buf <<= len;
-    br.have -= (int)len;
-    return ent;
+__device__ __forceinline__ uint32_t window_at(const uint32_t* words, uint32_t nwords, uint32_t pos) {
+    const uint32_t i = pos >> 5;
+    uint32_t hi, lo;
+    if (kChecked) {
+        hi = i < nwords ? __ldg(words + i) : 0u;
+        lo = i + 1 < nwords ? __ldg(words + i + 1) : 0u;
+    } else {
+        hi = words[i];
+        lo = words[i + 1];
+    }
+    return __funnelshift_l(lo, hi, pos);  // shift count taken modulo 32
+}
+
+// Decodes two symbols from the position `pos` on (a codeword has at most 16 bits, so one 32-bit window holds
+// both) and advances it.  Returns the two table entries: symbol in the low byte, 0xff = no codeword matched.
+template <bool kChecked, bool kSecond>
+__device__ __forceinline__ void decode_two(const uint32_t* words, uint32_t nwords, uint32_t& pos,
+                                           const uint16_t* __restrict__ s_lut, const uint16_t* __restrict__ sub_tab,
+                                           uint32_t& e0, uint32_t& e1) {
+    uint32_t win = window_at<kChecked>(words, nwords, pos);
+    e0 = s_lut[win >> (32 - kDecBits)];
+    if (e0 >= kDecLong) e0 = decode_long(sub_tab, e0, win);
+    const uint32_t l0 = e0 >> 8;
+    e1 = 0;
+    uint32_t l1 = 0;
+    if (kSecond) {
+        win <<= l0;
+        e1 = s_lut[win >> (32 - kDecBits)];
+        if (e1 >= kDecLong) e1 = decode_long(sub_tab, e1, win);
+        l1 = e1 >> 8;
+    }
+    pos += l0 + l1;
 }
 
 // Decodes `my` (<= 128) symbols of one sub-chunk into its row of the swizzled symbol buffer, four per
@@ -971,26 +963,24 @@ template <bool kChecked, bool kWhole>
 __device__ __forceinline__ uint32_t decode_sub(const uint32_t* words, uint32_t nwords, uint32_t off, uint32_t my,
                                                const uint16_t* __restrict__ s_lut, const uint16_t* __restrict__ sub_tab,
                                                uint32_t* row, uint32_t rot, bool& err) {
-    BitReader<kChecked> br;
-    br.init(words, nwords, off);
+    uint32_t pos = off;
     uint32_t marks = 0;  // collects, per byte lane, whether some symbol byte was 0xff
 #pragma unroll 2
     for (uint32_t j = 0; j < 32; ++j) {
         uint32_t w = 0;
         if (kWhole || j * 4 < my) {
-            br.refill();
-            const uint32_t e0 = decode_one(br, s_lut, sub_tab);
-            const uint32_t e1 = (kWhole || j * 4 + 1 < my) ? decode_one(br, s_lut, sub_tab) : 0u;
-            br.refill();
-            const uint32_t e2 = (kWhole || j * 4 + 2 < my) ? decode_one(br, s_lut, sub_tab) : 0u;
-            const uint32_t e3 = (kWhole || j * 4 + 3 < my) ? decode_one(br, s_lut, sub_tab) : 0u;
+            uint32_t e0, e1, e2 = 0, e3 = 0;
+            if (kWhole || j * 4 + 1 < my) decode_two<kChecked, true>(words, nwords, pos, s_lut, sub_tab, e0, e1);
+            else decode_two<kChecked, false>(words, nwords, pos, s_lut, sub_tab, e0, e1);
+            if (kWhole || j * 4 + 3 < my) decode_two<kChecked, true>(words, nwords, pos, s_lut, sub_tab, e2, e3);
+            else if (j * 4 + 2 < my) decode_two<kChecked, false>(words, nwords, pos, s_lut, sub_tab, e2, e3);
             w = __byte_perm(__byte_perm(e0, e1, 0x0040), __byte_perm(e2, e3, 0x0040), 0x5410);
             marks |= (~w - 0x01010101u) & w;  // bit 7 of a byte survives iff that byte of ~w is zero
         }
         row[(j + rot) & 31u] = w;
     }
     if (marks & 0x80808080u) err = true;
-    return br.position();
+    return pos;
 }
 
 // Adds, in client order, the values of the four symbols of word w of the tile for the nb clients of the batch.
