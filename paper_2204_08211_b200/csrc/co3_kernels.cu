@@ -891,7 +891,7 @@ constexpr int kPaySlotWords = 456;     // staging per pair: 7 bits/symbol plus a
 constexpr int kPaySlack = 72;          // words a reader may run past its chunk before the end check
 
 // Fixed part of the shared memory of one decode block; behind it follow the symbol buffer
-// sym[n_pairs][kC / 4] and the payload staging area pay[n_pairs * kPaySlotWords + kPaySlack].
+// sym[n_pairs][128] of one decode phase and the payload staging area pay[n_pairs * kPaySlotWords + kPaySlack].
 struct DecSmem {
     uint16_t lut[kDecLut];
     float val[256];
@@ -907,10 +907,18 @@ struct DecSmem {
 };
 static_assert(sizeof(DecSmem) % 16 == 0 && offsetof(DecSmem, sub) % 16 == 0, "dynamic arrays behind DecSmem must stay 16-byte aligned");
 
-// Position of word j of sub-chunk s in the symbol buffer of pair p: rotated so that the 32 threads of a
-// warp (2 pairs x 16 sub-chunks, all at the same j) hit 32 different banks, and so do 32 consecutive j.
+// A tile is decoded in kPhases rounds of kPhaseSyms symbols per sub-chunk: the symbol buffer between the
+// decoding threads and the summing threads then holds a quarter of a chunk per pair.
+constexpr int kPhases = 4;
+constexpr int kPhaseSyms = kS / kPhases;            // 32 symbols of every sub-chunk per phase
+constexpr int kPhaseWords = kPhaseSyms / 4;         // 8 symbol words per sub-chunk and phase
+constexpr int kPairPhaseWords = kSubs * kPhaseWords;  // 128 symbol words per pair and phase
+
+// Position of word j (0..7) of sub-chunk s in the phase's symbol buffer of pair p: rotated so that the 32
+// threads of a warp (2 pairs x 16 sub-chunks, all at the same j) hit 32 different banks, and so do 32
+// consecutive words read by the summing threads.
 __device__ __forceinline__ uint32_t sym_slot(uint32_t p, uint32_t s, uint32_t j) {
-    return s * 32u + ((j + s + 16u * (p & 1u)) & 31u);
+    return s * kPhaseWords + ((j + (s >> 2) + 4u * (p & 1u)) & (kPhaseWords - 1));
 }
 
 // Second-level look-up for a codeword longer than the first table's index; rare, kept out of line so that
@@ -957,16 +965,15 @@ __device__ __forceinline__ void decode_two(const uint32_t* words, uint32_t nword
     pos += l0 + l1;
 }
 
-// Decodes `my` (<= 128) symbols of one sub-chunk into its row of the swizzled symbol buffer, four per
-// word.  Returns the bit position (inside the chunk) behind the last symbol.
+// One phase of one sub-chunk: decodes symbols [4 * j0, 4 * j0 + 32) of the sub-chunk (those below `my`) from bit
+// position `pos` on into the pair's phase buffer, four per word, and advances `pos`.
 template <bool kChecked, bool kWhole>
-__device__ __forceinline__ uint32_t decode_sub(const uint32_t* words, uint32_t nwords, uint32_t off, uint32_t my,
-                                               const uint16_t* __restrict__ s_lut, const uint16_t* __restrict__ sub_tab,
-                                               uint32_t* row, uint32_t rot, bool& err) {
-    uint32_t pos = off;
-    uint32_t marks = 0;  // collects, per byte lane, whether some symbol byte was 0xff
+__device__ __forceinline__ void decode_part(const uint32_t* words, uint32_t nwords, uint32_t& pos, uint32_t j0, uint32_t my,
+                                            const uint16_t* __restrict__ s_lut, const uint16_t* __restrict__ sub_tab,
+                                            uint32_t* pair_buf, uint32_t p, uint32_t s, uint32_t& marks) {
 #pragma unroll 2
-    for (uint32_t j = 0; j < 32; ++j) {
+    for (uint32_t jj = 0; jj < (uint32_t)kPhaseWords; ++jj) {
+        const uint32_t j = j0 + jj;
         uint32_t w = 0;
         if (kWhole || j * 4 < my) {
             uint32_t e0, e1, e2 = 0, e3 = 0;
@@ -975,37 +982,35 @@ __device__ __forceinline__ uint32_t decode_sub(const uint32_t* words, uint32_t n
             if (kWhole || j * 4 + 3 < my) decode_two<kChecked, true>(words, nwords, pos, s_lut, sub_tab, e2, e3);
             else if (j * 4 + 2 < my) decode_two<kChecked, false>(words, nwords, pos, s_lut, sub_tab, e2, e3);
             w = __byte_perm(__byte_perm(e0, e1, 0x0040), __byte_perm(e2, e3, 0x0040), 0x5410);
-            marks |= (~w - 0x01010101u) & w;  // bit 7 of a byte survives iff that byte of ~w is zero
+            marks |= (~w - 0x01010101u) & w;  // bit 7 of a byte survives iff that byte of ~w is zero (symbol 0xff)
         }
-        row[(j + rot) & 31u] = w;
+        pair_buf[sym_slot(p, s, jj)] = w;
     }
-    if (marks & 0x80808080u) err = true;
-    return pos;
 }
 
-// Adds, in client order, the values of the four symbols of word w of the tile for the nb clients of the batch.
-// Returns the last client's symbol word.
+// Adds, in client order, the values of the four symbols of word w of the tile's current phase for the nb clients
+// of the batch.  Returns the last client's symbol word.
 __device__ __forceinline__ uint32_t sum_word(const float* __restrict__ val, const uint32_t* __restrict__ sym, uint32_t w,
                                              uint32_t B, uint32_t nb, float (&acc)[4]) {
-    const uint32_t cl = w / (kC / 4), wi = w % (kC / 4);
-    const uint32_t s = wi >> 5, j = wi & 31u;
+    const uint32_t cl = w / kPairPhaseWords, wi = w % kPairPhaseWords;
+    const uint32_t s = wi / kPhaseWords, j = wi % kPhaseWords;
     uint32_t symw = 0;
     for (uint32_t ul = 0; ul < nb; ++ul) {
         const uint32_t p = cl * B + ul;
-        symw = sym[p * (kC / 4) + sym_slot(p, s, j)];
+        symw = sym[p * kPairPhaseWords + sym_slot(p, s, j)];
 #pragma unroll
         for (int q = 0; q < 4; ++q) acc[q] = __fadd_rn(acc[q], val[(symw >> (8 * q)) & 0xffu]);
     }
     return symw;
 }
 
-// Divides the sums by the number of clients and stores the (up to four) elements of word w of the tile.
+// Divides the sums by the number of clients and stores the (up to four) elements of word w of the tile's phase.
 __device__ __forceinline__ void write_word(const DecArgs& a, const DecSmem& sm, const TileDesc& td, uint32_t w,
-                                           uint32_t B, const float (&acc)[4], uint32_t symw) {
-    const uint32_t cl = w / (kC / 4), wi = w % (kC / 4);
+                                           uint32_t phase, uint32_t B, const float (&acc)[4], uint32_t symw) {
+    const uint32_t cl = w / kPairPhaseWords, wi = w % kPairPhaseWords;
     if (cl >= td.n_chunks) return;
     const uint32_t cnt = sm.pair_cnt[cl * B];
-    const uint32_t i0 = wi * 4;
+    const uint32_t i0 = (wi / kPhaseWords) * kS + phase * kPhaseSyms + (wi % kPhaseWords) * 4;  // element inside the chunk
     if (i0 >= cnt) return;
     const uint32_t nv = min(4u, cnt - i0);
     const uint64_t e = sm.chunk_elem0[cl] + i0;
@@ -1041,7 +1046,7 @@ __global__ void __launch_bounds__(kThreads) decode_kernel(DecArgs a) {
     const uint32_t B = kMulti ? 16u : a.B, G = kMulti ? 1u : a.G;
     const uint32_t n_pairs = B * G, n_thr = 16u * n_pairs;
     uint32_t* const sm_sym = reinterpret_cast<uint32_t*>(smem_raw + sizeof(DecSmem));
-    uint32_t* const sm_pay = sm_sym + n_pairs * (kC / 4);
+    uint32_t* const sm_pay = sm_sym + n_pairs * kPairPhaseWords;
     const uint32_t pay_words = n_pairs * kPaySlotWords;
 
     const Ctrl* ctrl = a.ws.ctrl;
@@ -1054,7 +1059,7 @@ __global__ void __launch_bounds__(kThreads) decode_kernel(DecArgs a) {
     const uint16_t* sub_tab = a.ws.dec_sub + (size_t)td.seg * kSubLut;
 
     if (tid == 0) mbar_init(&sm.bar, 1);
-    float carry[2][4];  // running sums across client batches (kMulti only)
+    float carry[kPhases][4];  // running sums across client batches (kMulti only)
     bool err = false, hw_fail = false;
     uint32_t phase = 0;
 
@@ -1126,65 +1131,66 @@ __global__ void __launch_bounds__(kThreads) decode_kernel(DecArgs a) {
             mbar_wait(&sm.bar, phase);
             break;
         }
-        // ---- decode: thread = (pair, sub-chunk)
-        {
-            const uint32_t p = tid >> 4, s = tid & 15u;
-            const uint32_t cnt = sm.pair_cnt[p];
-            const uint32_t nw = sm.pair_words[p];
-            const uint32_t my = cnt > s * kS ? min((uint32_t)kS, cnt - s * kS) : 0u;
-            uint32_t* row = sm_sym + p * (kC / 4) + s * 32u;
-            const uint32_t rot = s + 16u * (p & 1u);
-            bool zero = true;
-            if (my) {
-                const uint32_t off = sm.sub[p][s];
-                const bool last = cnt <= (s + 1) * kS;
-                const uint32_t expect = last ? 0u : sm.sub[p][s + 1];
-                if (off > nw * 32u) {
-                    err = true;
-                } else {
-                    uint32_t end;
-                    if (sm.pair_staged[p]) {
-                        const uint32_t* words = sm_pay + sm.pair_off[p];
-                        if (my == (uint32_t)kS) end = decode_sub<false, true>(words, nw, off, my, sm.lut, sub_tab, row, rot, err);
-                        else end = decode_sub<false, false>(words, nw, off, my, sm.lut, sub_tab, row, rot, err);
-                    } else {
-                        end = decode_sub<true, false>(sm.pair_src[p], nw, off, my, sm.lut, sub_tab, row, rot, err);
-                    }
-                    zero = false;
-                    if (!last) {
-                        if (end != expect) err = true;
-                    } else if (((end + 31u) >> 5) != nw) {
-                        err = true;
-                    }
-                }
-            }
-            if (zero)
-                for (uint32_t j = 0; j < 32; ++j) row[j] = 0;
+        // ---- thread = (pair, sub-chunk): where its bits start and how many symbols it has
+        const uint32_t p = tid >> 4, sc = tid & 15u;
+        const uint32_t cnt = sm.pair_cnt[p];
+        const uint32_t nw = sm.pair_words[p];
+        uint32_t my = cnt > sc * kS ? min((uint32_t)kS, cnt - sc * kS) : 0u;
+        const bool staged = sm.pair_staged[p] != 0;
+        const uint32_t* const swords = sm_pay + sm.pair_off[p];  // staged copy in shared memory
+        const uint32_t* const gwords = sm.pair_src[p];           // the words in place, in global memory
+        uint32_t* pair_buf = sm_sym + p * kPairPhaseWords;
+        uint32_t pos = my ? sm.sub[p][sc] : 0u, marks = 0;
+        const bool last = cnt <= (sc + 1) * kS;
+        const uint32_t expect = (my && !last) ? sm.sub[p][sc + 1] : 0u;
+        if (my && pos > nw * 32u) {
+            err = true;
+            my = 0;
         }
-        __syncthreads();
-        // ---- ordered sum over the clients of this batch; a thread owns whole symbol words
+        const bool had_symbols = my != 0;
         const bool first_batch = (u0 == 0), last_batch = (u0 + B >= a.n_clients);
-        if (kMulti) {
 #pragma unroll
-            for (int r = 0; r < 2; ++r) {
-                const uint32_t w = tid + r * kThreads;
-                float acc[4];
+        for (int ph = 0; ph < kPhases; ++ph) {
+            // ---- decode this phase's 32 symbols of the sub-chunk
+            const uint32_t j0 = ph * kPhaseWords;
+            if (my > j0 * 4) {
+                if (!staged) decode_part<true, false>(gwords, nw, pos, j0, my, sm.lut, sub_tab, pair_buf, p, sc, marks);
+                else if (my == (uint32_t)kS) decode_part<false, true>(swords, nw, pos, j0, my, sm.lut, sub_tab, pair_buf, p, sc, marks);
+                else decode_part<false, false>(swords, nw, pos, j0, my, sm.lut, sub_tab, pair_buf, p, sc, marks);
+            } else {
+                for (uint32_t jj = 0; jj < (uint32_t)kPhaseWords; ++jj) pair_buf[sym_slot(p, sc, jj)] = 0;
+            }
+            __syncthreads();
+            // ---- ordered sum over the clients of this batch; a thread owns whole symbol words
+            if (kMulti) {
+                if (tid < (uint32_t)kPairPhaseWords) {
+                    float acc[4];
 #pragma unroll
-                for (int q = 0; q < 4; ++q) acc[q] = first_batch ? 0.0f : carry[r][q];
-                const uint32_t symw = sum_word(sm.val, sm_sym, w, B, nb, acc);
-                if (!last_batch) {
+                    for (int q = 0; q < 4; ++q) acc[q] = first_batch ? 0.0f : carry[ph][q];
+                    const uint32_t symw = sum_word(sm.val, sm_sym, tid, B, nb, acc);
+                    if (!last_batch) {
 #pragma unroll
-                    for (int q = 0; q < 4; ++q) carry[r][q] = acc[q];
-                } else {
-                    write_word(a, sm, td, w, B, acc, symw);
+                        for (int q = 0; q < 4; ++q) carry[ph][q] = acc[q];
+                    } else {
+                        write_word(a, sm, td, tid, ph, B, acc, symw);
+                    }
+                }
+            } else {
+                const uint32_t tile_words = G * kPairPhaseWords;
+                for (uint32_t w = tid; w < tile_words; w += n_thr) {
+                    float acc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+                    const uint32_t symw = sum_word(sm.val, sm_sym, w, B, nb, acc);
+                    write_word(a, sm, td, w, ph, B, acc, symw);
                 }
             }
-        } else {
-            const uint32_t tile_words = G * (kC / 4);
-            for (uint32_t w = tid; w < tile_words; w += n_thr) {
-                float acc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-                const uint32_t symw = sum_word(sm.val, sm_sym, w, B, nb, acc);
-                write_word(a, sm, td, w, B, acc, symw);
+            __syncthreads();  // the phase buffer is free again
+        }
+        if (marks & 0x80808080u) err = true;
+        if (had_symbols) {  // the sub-chunk must end where the next one starts, the last one inside the chunk's last word
+            if (!last) {
+                if (pos != expect) err = true;
+            } else if (((pos + 31u) >> 5) != nw) {
+                err = true;
             }
         }
     }
@@ -1363,7 +1369,7 @@ int decode_common(const uint8_t* const* streams, const uint8_t* single, size_t s
     const uint32_t tiles = (uint32_t)(L.n_chunks_max / G + n_seg);  // upper bound; surplus blocks return at once
     if (tiles == 0) return CO3_OK;
     const uint32_t n_pairs = B * G;
-    const size_t smem = sizeof(DecSmem) + 4 * ((size_t)n_pairs * (kC / 4 + kPaySlotWords) + kPaySlack);
+    const size_t smem = sizeof(DecSmem) + 4 * ((size_t)n_pairs * (kPairPhaseWords + kPaySlotWords) + kPaySlack);
     if (multi) {
         CO3_CUDA(cudaFuncSetAttribute(decode_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         CO3_LAUNCH(CO3_KERNEL_DECODE, st, decode_kernel<true><<<tiles, kThreads, smem, st>>>(da));
