@@ -21,6 +21,7 @@ constexpr uint32_t kEncMissing = 0x80000000u;                // encode table ent
 constexpr uint32_t kDecLong = 0x8000u;                       // decode table entry: look in a second-level table
 constexpr uint32_t kDecInvalid = 0x01ffu;                    // decode table entry: no codeword; consumes one bit and
                                                              // yields 0xff, which is a symbol of no format
+constexpr int kRangeChunks = 4096;                            // chunks summed by one block in the two-level scan
 constexpr uint32_t kMagic = 0x53334F43u;                     // 'C','O','3','S'
 constexpr uint32_t kHeaderBytes = 64;
 constexpr int kThreads = 256;
@@ -81,6 +82,9 @@ struct Ws {
     uint32_t* client_fail;  // [n_clients]
     uint32_t* chunk_bits;   // [n_clients][n_chunks_max]
     uint64_t* bit_prefix;   // [n_clients][n_chunks_max + 1]
+    uint64_t* range_tot;    // [n_clients][n_ranges_max][2]  words and bits of each range of kRangeChunks chunks
+                            //                               (long inputs only), then their exclusive prefixes
+    uint64_t* totals;       // [n_clients][2]                payload words and bits of the client (long inputs)
     uint32_t* slots;        // [n_clients][n_chunks_max][kSlotWords]
     uint32_t n_chunks_max;
 };

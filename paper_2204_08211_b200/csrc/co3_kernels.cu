@@ -9,6 +9,8 @@
 //   decode_kernel         chunk-indexed prefix-code decoder fused with the ordered cross-client sum
 #include <cuda_runtime.h>
 #include <stddef.h>
+
+#include <algorithm>
 #include <stdint.h>
 
 #include "co3.h"
@@ -57,7 +59,7 @@ __global__ void __launch_bounds__(kThreads) prepare_kernel(PrepArgs a) {
     const uint32_t k = blockIdx.x;
     const uint32_t G = a.tile_chunks;
 
-    if (k == 0)
+    if (k == 0 && blockIdx.y == 0)
         for (uint32_t u = tid; u < a.n_res; u += kThreads) a.res[u].first_bad_chunk = 0xffffffffu;
 
     // ---- layout: elements, chunks and tiles of the segments before this one
@@ -97,7 +99,7 @@ __global__ void __launch_bounds__(kThreads) prepare_kernel(PrepArgs a) {
         if (tid == 0) fail_all(a, CO3_ERR_INVALID_ARG);
         return;
     }
-    if (tid == 0) {
+    if (tid == 0 && blockIdx.y == 0) {
         a.ws.first_chunk[k] = (uint32_t)c_before;
         if (k == a.n_seg - 1) {
             const uint64_t nc = c_before + my_chunks;
@@ -110,14 +112,15 @@ __global__ void __launch_bounds__(kThreads) prepare_kernel(PrepArgs a) {
             c->payload_off = align16(c->sub_off + 2ull * nc * kSubs);
         }
     }
-    for (uint64_t c = tid; c < my_chunks; c += kThreads) {
+    // descriptors: blockIdx.y strides over them, so that one long segment is laid out by many blocks
+    for (uint64_t c = (uint64_t)blockIdx.y * kThreads + tid; c < my_chunks; c += (uint64_t)gridDim.y * kThreads) {
         ChunkDesc d;
         d.seg = k;
         d.cnt = (uint32_t)min((uint64_t)kC, sg.n_elem - c * kC);
         d.elem0 = sg.elem_off + c * kC;
         a.ws.chunk_desc[c_before + c] = d;
     }
-    for (uint64_t t = tid; t < my_tiles; t += kThreads) {
+    for (uint64_t t = (uint64_t)blockIdx.y * kThreads + tid; t < my_tiles; t += (uint64_t)gridDim.y * kThreads) {
         TileDesc d;
         d.seg = k;
         d.chunk0 = (uint32_t)(c_before + t * G);
@@ -125,6 +128,7 @@ __global__ void __launch_bounds__(kThreads) prepare_kernel(PrepArgs a) {
         d.pad = 0;
         a.ws.tile_desc[t_before + t] = d;
     }
+    if (blockIdx.y != 0) return;  // helper blocks only lay out descriptors
 
     // ---- format constants and value table
     bool fmt_ok = true;
@@ -715,56 +719,170 @@ struct ScanArgs {
     uint8_t* streams;
     size_t stream_capacity;
     co3_result* res;
+    uint32_t two_level;    // 1: chunk offsets come from the range kernels below, scan_kernel only finishes
+    uint32_t n_ranges_max;
     Ws ws;
 };
 
 constexpr int kScanThreads = 1024;
+static_assert(kRangeChunks == 4 * kScanThreads, "one range is one tile of four chunks per thread");
+
+// Exclusive prefix of 32-bit per-thread sums over the 1024 threads of a block (two quantities at once);
+// *tot_w / *tot_b receive the block totals.  Contains two __syncthreads().
+__device__ __forceinline__ void block_scan_1024x2(uint32_t w, uint32_t b, uint64_t* s_w, uint64_t* s_b, uint64_t& ex_w,
+                                                  uint64_t& ex_b, uint64_t& tot_w, uint64_t& tot_b) {
+    const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+    uint32_t iw = w, ib = b;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const uint32_t yw = __shfl_up_sync(0xffffffffu, iw, d), yb = __shfl_up_sync(0xffffffffu, ib, d);
+        if (lane >= (uint32_t)d) { iw += yw; ib += yb; }
+    }
+    __syncthreads();  // earlier readers of s_w / s_b are done
+    if (lane == 31u) { s_w[warp] = iw; s_b[warp] = ib; }
+    __syncthreads();
+    uint64_t bw = 0, bb = 0;
+    tot_w = 0;
+    tot_b = 0;
+    for (uint32_t x = 0; x < 32; ++x) {
+        if (x < warp) { bw += s_w[x]; bb += s_b[x]; }
+        tot_w += s_w[x];
+        tot_b += s_b[x];
+    }
+    ex_w = bw + iw - w;
+    ex_b = bb + ib - b;
+}
+
+// Two-level scan for long inputs, step 1: words and bits of each range of kRangeChunks chunks.
+__global__ void __launch_bounds__(kScanThreads) range_totals_kernel(ScanArgs a) {
+    __shared__ uint64_t s_w[32], s_b[32];
+    const Ctrl* ctrl = a.ws.ctrl;
+    if (ctrl->abort) return;
+    const uint32_t y = blockIdx.x, u = blockIdx.y, tid = threadIdx.x;
+    const uint32_t n = ctrl->n_chunks;
+    if ((uint64_t)y * kRangeChunks >= n) return;
+    const uint32_t* bits = a.ws.chunk_bits + (size_t)u * a.ws.n_chunks_max;
+    const uint32_t c0 = y * kRangeChunks + 4 * tid;
+    uint32_t w = 0, b = 0;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const uint32_t x = (c0 + i < n) ? bits[c0 + i] : 0u;
+        b += x;
+        w += (x + 31u) >> 5;
+    }
+    uint64_t ew, eb, tw, tb;
+    block_scan_1024x2(w, b, s_w, s_b, ew, eb, tw, tb);
+    if (tid == 0) {
+        uint64_t* r = a.ws.range_tot + ((size_t)u * a.n_ranges_max + y) * 2;
+        r[0] = tw;
+        r[1] = tb;
+    }
+}
+
+// Step 2: one block per client turns the range totals into exclusive prefixes and the client's totals.
+__global__ void __launch_bounds__(kScanThreads) range_scan_kernel(ScanArgs a) {
+    const Ctrl* ctrl = a.ws.ctrl;
+    if (ctrl->abort) return;
+    const uint32_t u = blockIdx.x, tid = threadIdx.x;
+    const uint32_t n_ranges = (ctrl->n_chunks + kRangeChunks - 1) / kRangeChunks;
+    uint64_t* r = a.ws.range_tot + (size_t)u * a.n_ranges_max * 2;
+    // few ranges (one per 8 M elements): one thread walks them
+    if (tid == 0) {
+        uint64_t w = 0, b = 0;
+        for (uint32_t y = 0; y < n_ranges; ++y) {
+            const uint64_t tw = r[2 * y], tb = r[2 * y + 1];
+            r[2 * y] = w;
+            r[2 * y + 1] = b;
+            w += tw;
+            b += tb;
+        }
+        a.ws.totals[2 * u] = w;
+        a.ws.totals[2 * u + 1] = b;
+    }
+}
+
+// Step 3: every range scans its own chunks from its exclusive prefix and writes the chunk offsets.
+__global__ void __launch_bounds__(kScanThreads) range_apply_kernel(ScanArgs a) {
+    __shared__ uint64_t s_w[32], s_b[32];
+    const Ctrl* ctrl = a.ws.ctrl;
+    if (ctrl->abort) return;
+    const uint32_t y = blockIdx.x, u = blockIdx.y, tid = threadIdx.x;
+    const uint32_t n = ctrl->n_chunks;
+    if ((uint64_t)y * kRangeChunks >= n) return;
+    const uint32_t* bits = a.ws.chunk_bits + (size_t)u * a.ws.n_chunks_max;
+    uint64_t* bit_prefix = a.ws.bit_prefix + (size_t)u * (a.ws.n_chunks_max + 1ull);
+    uint8_t* stream = a.streams + (size_t)u * a.stream_capacity;
+    uint64_t* word_off = reinterpret_cast<uint64_t*>(stream + ctrl->chunk_off);
+    const uint64_t* r = a.ws.range_tot + ((size_t)u * a.n_ranges_max + y) * 2;
+    const uint32_t c0 = y * kRangeChunks + 4 * tid;
+    uint32_t bv[4], wv[4], w = 0, b = 0;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        bv[i] = (c0 + i < n) ? bits[c0 + i] : 0u;
+        wv[i] = (bv[i] + 31u) >> 5;
+        b += bv[i];
+        w += wv[i];
+    }
+    uint64_t ew, eb, tw, tb;
+    block_scan_1024x2(w, b, s_w, s_b, ew, eb, tw, tb);
+    uint64_t pw = r[0] + ew, pb = r[1] + eb;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        if (c0 + i < n) {
+            word_off[c0 + i] = pw;
+            bit_prefix[c0 + i] = pb;
+        }
+        pw += wv[i];
+        pb += bv[i];
+    }
+}
 
 __global__ void __launch_bounds__(kScanThreads) scan_kernel(ScanArgs a) {
     __shared__ uint64_t s_w[32], s_b[32];
     const Ctrl* ctrl = a.ws.ctrl;
     if (ctrl->abort) return;
-    const uint32_t u = blockIdx.x, tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
+    const uint32_t u = blockIdx.x, tid = threadIdx.x;
     const uint32_t n = ctrl->n_chunks;
     const uint32_t* bits = a.ws.chunk_bits + (size_t)u * a.ws.n_chunks_max;
     uint64_t* bit_prefix = a.ws.bit_prefix + (size_t)u * (a.ws.n_chunks_max + 1ull);
     uint8_t* stream = a.streams + (size_t)u * a.stream_capacity;
     uint64_t* word_off = reinterpret_cast<uint64_t*>(stream + ctrl->chunk_off);
 
-    const uint32_t per = (n + kScanThreads - 1) / kScanThreads;
-    const uint32_t lo = min(tid * per, n), hi = min(lo + per, n);
-    uint64_t sw = 0, sb = 0;
-    for (uint32_t c = lo; c < hi; ++c) {
-        const uint32_t b = bits[c];
-        sb += b;
-        sw += (b + 31u) >> 5;
-    }
-    uint64_t iw = sw, ib = sb;
+    // tiles of 4 * 1024 chunks: four consecutive chunks per thread, warp scan, one exchange through shared memory
+    uint64_t carry_w = 0, carry_b = 0;  // totals of the tiles already done (same in every thread)
+    if (a.two_level) {  // the range kernels have written the chunk offsets already
+        carry_w = a.ws.totals[2 * u];
+        carry_b = a.ws.totals[2 * u + 1];
+    } else {
+        for (uint32_t base = 0; base < n; base += 4 * kScanThreads) {
+            const uint32_t c0 = base + 4 * tid;
+            uint32_t b[4], w[4];
 #pragma unroll
-    for (int d = 1; d < 32; d <<= 1) {
-        const uint64_t yw = __shfl_up_sync(0xffffffffu, iw, d), yb = __shfl_up_sync(0xffffffffu, ib, d);
-        if (lane >= (uint32_t)d) { iw += yw; ib += yb; }
+            for (int i = 0; i < 4; ++i) {
+                b[i] = (c0 + i < n) ? bits[c0 + i] : 0u;
+                w[i] = (b[i] + 31u) >> 5;
+            }
+            const uint32_t tw4 = w[0] + w[1] + w[2] + w[3], tb4 = b[0] + b[1] + b[2] + b[3];
+            uint64_t ew, eb, tile_w, tile_b;
+            block_scan_1024x2(tw4, tb4, s_w, s_b, ew, eb, tile_w, tile_b);
+            uint64_t pw = carry_w + ew, pb = carry_b + eb;  // exclusive prefix of chunk c0
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                if (c0 + i < n) {
+                    word_off[c0 + i] = pw;
+                    bit_prefix[c0 + i] = pb;
+                }
+                pw += w[i];
+                pb += b[i];
+            }
+            carry_w += tile_w;
+            carry_b += tile_b;
+        }
     }
-    if (lane == 31u) { s_w[warp] = iw; s_b[warp] = ib; }
-    __syncthreads();
-    uint64_t bw = 0, bb = 0, tw = 0, tb = 0;
-    for (uint32_t w = 0; w < 32; ++w) {
-        if (w < warp) { bw += s_w[w]; bb += s_b[w]; }
-        tw += s_w[w];
-        tb += s_b[w];
-    }
-    uint64_t pw = bw + iw - sw, pb = bb + ib - sb;  // exclusive prefix of this thread's range
-
+    const uint64_t tw = carry_w, tb = carry_b;
     const uint64_t total_bytes = align16(ctrl->payload_off + 4ull * tw);
     const bool fits = total_bytes <= a.stream_capacity;
     const bool failed = a.ws.client_fail[u] != 0;
-    for (uint32_t c = lo; c < hi; ++c) {
-        word_off[c] = pw;
-        bit_prefix[c] = pb;
-        const uint32_t b = bits[c];
-        pb += b;
-        pw += (b + 31u) >> 5;
-    }
     if (tid == 0) {
         word_off[n] = tw;
         bit_prefix[n] = tb;
@@ -1214,7 +1332,8 @@ namespace {
 
 struct WsLayout {
     size_t ctrl, first_chunk, chunk_desc, tile_desc, fmt, enc_lut, dec_lut, dec_sub, val_lut, client_fail, chunk_bits,
-        bit_prefix, slots, total;
+        bit_prefix, range_tot, totals, slots, total;
+    uint32_t n_ranges_max;
     uint32_t n_chunks_max;
 };
 
@@ -1238,6 +1357,9 @@ bool ws_layout(uint64_t n_elem, uint32_t n_seg, uint32_t n_clients, WsLayout* L)
     L->client_fail = o; o += up256(4 * (size_t)(n_clients ? n_clients : 1));
     L->chunk_bits = o;  o += up256(4 * (size_t)n_clients * nc);
     L->bit_prefix = o;  o += up256(8 * (size_t)n_clients * (nc + 1));
+    L->n_ranges_max = (uint32_t)(nc / kRangeChunks + 1);
+    L->range_tot = o;   o += up256(16 * (size_t)n_clients * L->n_ranges_max);
+    L->totals = o;      o += up256(16 * (size_t)(n_clients ? n_clients : 1));
     L->slots = o;       o += up256(4 * (size_t)kSlotWords * n_clients * nc);
     L->total = o;
     return true;
@@ -1258,6 +1380,8 @@ Ws ws_pointers(void* base, const WsLayout& L) {
     w.client_fail = reinterpret_cast<uint32_t*>(b + L.client_fail);
     w.chunk_bits = reinterpret_cast<uint32_t*>(b + L.chunk_bits);
     w.bit_prefix = reinterpret_cast<uint64_t*>(b + L.bit_prefix);
+    w.range_tot = reinterpret_cast<uint64_t*>(b + L.range_tot);
+    w.totals = reinterpret_cast<uint64_t*>(b + L.totals);
     w.slots = reinterpret_cast<uint32_t*>(b + L.slots);
     w.n_chunks_max = L.n_chunks_max;
     return w;
@@ -1334,7 +1458,10 @@ int begin_call(const WsLayout& L, const Ws& ws, co3_result* res, uint32_t n_res,
     CO3_CUDA(cudaMemsetAsync(res, 0, sizeof(co3_result) * (size_t)n_res, st));
     CO3_CUDA(cudaMemsetAsync(ws.client_fail, 0, 4 * (size_t)(n_fail ? n_fail : 1), st));
     PrepArgs pa{fmts, codes, segs, n_seg, n_elem, tile_chunks, res, n_res, ws};
-    CO3_LAUNCH(CO3_KERNEL_PREPARE, st, prepare_kernel<<<n_seg ? n_seg : 1, kThreads, 0, st>>>(pa));
+    // extra blocks per segment when segments are long (their chunk descriptors are written in parallel)
+    const uint64_t per_seg = L.n_chunks_max / (n_seg ? n_seg : 1);
+    const uint32_t helpers = (uint32_t)std::min<uint64_t>(128, per_seg / (8 * kThreads) + 1);
+    CO3_LAUNCH(CO3_KERNEL_PREPARE, st, prepare_kernel<<<dim3(n_seg ? n_seg : 1, helpers), kThreads, 0, st>>>(pa));
     (void)L;
     return CO3_OK;
 }
@@ -1413,7 +1540,15 @@ int encode_common(const float* grad, float* mem, float decay, const uint8_t* sym
             CO3_LAUNCH(CO3_KERNEL_PACK, st, pack_kernel<false><<<grid, kThreads, sizeof(PackSmem), st>>>(pa));
         }
     }
-    ScanArgs sa{segs, n_seg, n_elem, streams_out, stream_capacity, res, ws};
+    // inputs beyond a few tiles of chunks per client: offsets by a two-level scan over many blocks
+    const uint32_t two_level = L.n_chunks_max > 4u * kRangeChunks ? 1u : 0u;
+    ScanArgs sa{segs, n_seg, n_elem, streams_out, stream_capacity, res, two_level, L.n_ranges_max, ws};
+    if (two_level) {
+        const dim3 rgrid(L.n_ranges_max, n_clients);
+        CO3_LAUNCH(CO3_KERNEL_SCAN, st, range_totals_kernel<<<rgrid, kScanThreads, 0, st>>>(sa));
+        CO3_LAUNCH(CO3_KERNEL_SCAN, st, range_scan_kernel<<<n_clients, kScanThreads, 0, st>>>(sa));
+        CO3_LAUNCH(CO3_KERNEL_SCAN, st, range_apply_kernel<<<rgrid, kScanThreads, 0, st>>>(sa));
+    }
     CO3_LAUNCH(CO3_KERNEL_SCAN, st, scan_kernel<<<n_clients, kScanThreads, 0, st>>>(sa));
     if (L.n_chunks_max) {
         CO3_LAUNCH(CO3_KERNEL_COMPACT, st, compact_kernel<<<dim3((L.n_chunks_max + kThreads / 32 - 1) / (kThreads / 32), n_clients), kThreads, 0, st>>>(sa));

@@ -46,10 +46,11 @@ class Co3Session:
         return buf[u * self.stride:u * self.stride + self.n_elem]
 
     # -- code fitting -------------------------------------------------------------------------
-    def histogram(self, grads: torch.Tensor, mems: torch.Tensor, stream=None) -> np.ndarray:
-        """Symbol counts per layer summed over clients for this round; `mems` is updated like a real round."""
+    def histogram(self, grads: torch.Tensor, mems: torch.Tensor, stream=None, sym_out=None) -> np.ndarray:
+        """Symbol counts per layer summed over clients for this round; `mems` is updated like a real round
+        and, if `sym_out` is given, the symbols are kept for co3_encode_symbols."""
         st = B.co3_convert(grads, mems, self.decay, self.fmts, self.segs, self.n_seg, self.n_elem, self.n_clients,
-                           self.stride, None, self.hist, self.res_enc, self.workspace, stream)
+                           self.stride, sym_out, self.hist, self.res_enc, self.workspace, stream)
         self._check(st, "co3_convert")
         return self.hist.cpu().numpy().astype(np.uint64).reshape(-1, 256)[:self.n_seg]
 

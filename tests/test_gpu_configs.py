@@ -158,6 +158,26 @@ def test_config5_outliers_and_eight_clients():
             assert same_bits(agg["avg"][:n], avg)
 
 
+def test_long_input_two_level_offsets():
+    """35.7 M elements in one layer (beyond 16384 chunks the chunk offsets come from the multi-block scan):
+    the whole stream and the decoded values against the oracle."""
+    cfg = ci.config(5)
+    n = 35_700_003
+    case = Case([n], _fmts(cfg, [n]), n_clients=1, decay=cfg["decay"])
+    g = _grads(cfg, [n], 1, 0, outliers=True)
+    mem_o = np.zeros((1, n), dtype=np.float32)
+    syms, ghats, nsat, _ = oracle_convert(case, g, mem_o)
+    codes = oracle_codes(case, oracle_hist(case, syms))
+    want = oracle_encode(case, syms, codes)[0][1]
+    gpu = Gpu(case)
+    out = gpu.encode(g, np.zeros_like(g), codes)
+    assert out["status"] == co3.OK and out["res"][0]["status"] == co3.OK and out["guard_ok"]
+    assert same_bits(out["mem"], mem_o) and out["res"][0]["n_saturated"] == nsat[0]
+    assert np.array_equal(out["streams"][0], want)
+    dec = gpu.decode(out["streams"][0], codes, want_sym=False)
+    assert dec["res"][0]["status"] == co3.OK and same_bits(dec["ghat"][:n], ghats[0])
+
+
 def test_config2_full_size_sampled_chunks():
     """The launch bench.py times (10 clients x 11,181,642 elements, second round so that memory is live):
     sampled chunks against the oracle, and size-independent properties of the streams."""
