@@ -1133,13 +1133,22 @@ __device__ __forceinline__ void write_word(const DecArgs& a, const DecSmem& sm, 
     const uint32_t nv = min(4u, cnt - i0);
     const uint64_t e = sm.chunk_elem0[cl] + i0;
     if (a.out) {
+        // acc / U; for a power of two the product with the exact reciprocal rounds the same real number
         const float U = (float)a.n_clients;
+        float r[4];
+        if ((a.n_clients & (a.n_clients - 1u)) == 0) {
+            const float inv = __fdiv_rn(1.0f, U);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) r[q] = __fmul_rn(acc[q], inv);
+        } else {
+#pragma unroll
+            for (int q = 0; q < 4; ++q) r[q] = __fdiv_rn(acc[q], U);
+        }
         float* o = a.out + e;
         if (nv == 4 && (reinterpret_cast<uintptr_t>(o) & 15u) == 0) {
-            *reinterpret_cast<float4*>(o) = make_float4(__fdiv_rn(acc[0], U), __fdiv_rn(acc[1], U),
-                                                        __fdiv_rn(acc[2], U), __fdiv_rn(acc[3], U));
+            *reinterpret_cast<float4*>(o) = make_float4(r[0], r[1], r[2], r[3]);
         } else {
-            for (uint32_t q = 0; q < nv; ++q) o[q] = __fdiv_rn(acc[q], U);
+            for (uint32_t q = 0; q < nv; ++q) o[q] = r[q];
         }
     }
     if (a.sym_out) {
