@@ -57,9 +57,11 @@ def load_peaks():
     return 6650.0, "fallback (6.65 TB/s, earlier measurement on this pool)"
 
 
-def workload(cfg_idx: int, clients_override=None):
+def workload(cfg_idx: int, clients_override=None, elements_override=None):
     import co3_inputs as ci
     cfg = ci.config(cfg_idx)
+    if elements_override is not None and len(cfg["sizes"]) == 1:
+        cfg = dict(cfg, sizes=(int(elements_override),))
     if "cells" in cfg:      # the sweep config: one representative cell
         cell = cfg["cells"][0]
         cfg = dict(cfg, fmt=cell["fmt"], beta=(cell["beta"],), decay=cell["decay"])
@@ -235,7 +237,7 @@ def run_ours(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
 
-    cfg, sizes, fmts, clients = workload(args.config, args.clients)
+    cfg, sizes, fmts, clients = workload(args.config, args.clients, args.elements)
     sess = Co3Session(sizes, fmts, clients, cfg["decay"], dev)
     n_rounds = 2
     grads = [make_grads(cfg, sizes, clients, sess.stride, r, dev, rank) for r in range(n_rounds)]
@@ -446,6 +448,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=2)
     ap.add_argument("--clients", type=int, default=None, help="override the clients per GPU (profiling small cases)")
+    ap.add_argument("--elements", type=int, default=None, help="override the length of a single-layer config (profiling)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     if args.impl == "reference":

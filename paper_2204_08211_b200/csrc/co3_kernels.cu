@@ -1106,12 +1106,18 @@ __device__ __forceinline__ void decode_part(const uint32_t* words, uint32_t nwor
     }
 }
 
-// Adds, in client order, the values of the four symbols of word w of the tile's current phase for the nb clients
-// of the batch.  Returns the last client's symbol word.
-__device__ __forceinline__ uint32_t sum_word(const float* __restrict__ val, const uint32_t* __restrict__ sym, uint32_t w,
-                                             uint32_t B, uint32_t nb, float (&acc)[4]) {
-    const uint32_t cl = w / kPairPhaseWords, wi = w % kPairPhaseWords;
-    const uint32_t s = wi / kPhaseWords, j = wi % kPhaseWords;
+// How the block's averages are formed: acc / U, or acc * (1 / U) when U is a power of two (the product with
+// the exact reciprocal rounds the same real number as the division).
+struct Averager {
+    float u, inv;
+    bool pow2;
+    __device__ __forceinline__ float operator()(float acc) const { return pow2 ? __fmul_rn(acc, inv) : __fdiv_rn(acc, u); }
+};
+
+// Adds, in client order, the values of the four symbols of word (s, j) of chunk cl of the tile's current phase
+// for the nb clients of the batch.  Returns the last client's symbol word.
+__device__ __forceinline__ uint32_t sum_word(const float* __restrict__ val, const uint32_t* __restrict__ sym, uint32_t cl,
+                                             uint32_t s, uint32_t j, uint32_t B, uint32_t nb, float (&acc)[4]) {
     uint32_t symw = 0;
     for (uint32_t ul = 0; ul < nb; ++ul) {
         const uint32_t p = cl * B + ul;
@@ -1122,33 +1128,20 @@ __device__ __forceinline__ uint32_t sum_word(const float* __restrict__ val, cons
     return symw;
 }
 
-// Divides the sums by the number of clients and stores the (up to four) elements of word w of the tile's phase.
-__device__ __forceinline__ void write_word(const DecArgs& a, const DecSmem& sm, const TileDesc& td, uint32_t w,
-                                           uint32_t phase, uint32_t B, const float (&acc)[4], uint32_t symw) {
-    const uint32_t cl = w / kPairPhaseWords, wi = w % kPairPhaseWords;
+// Averages the sums and stores the (up to four) elements that start at element i0 of chunk cl of the tile.
+__device__ __forceinline__ void write_word(const DecArgs& a, const DecSmem& sm, const TileDesc& td, uint32_t cl, uint32_t i0,
+                                           uint32_t B, const Averager& avg, const float (&acc)[4], uint32_t symw) {
     if (cl >= td.n_chunks) return;
     const uint32_t cnt = sm.pair_cnt[cl * B];
-    const uint32_t i0 = (wi / kPhaseWords) * kS + phase * kPhaseSyms + (wi % kPhaseWords) * 4;  // element inside the chunk
     if (i0 >= cnt) return;
     const uint32_t nv = min(4u, cnt - i0);
     const uint64_t e = sm.chunk_elem0[cl] + i0;
     if (a.out) {
-        // acc / U; for a power of two the product with the exact reciprocal rounds the same real number
-        const float U = (float)a.n_clients;
-        float r[4];
-        if ((a.n_clients & (a.n_clients - 1u)) == 0) {
-            const float inv = __fdiv_rn(1.0f, U);
-#pragma unroll
-            for (int q = 0; q < 4; ++q) r[q] = __fmul_rn(acc[q], inv);
-        } else {
-#pragma unroll
-            for (int q = 0; q < 4; ++q) r[q] = __fdiv_rn(acc[q], U);
-        }
         float* o = a.out + e;
         if (nv == 4 && (reinterpret_cast<uintptr_t>(o) & 15u) == 0) {
-            *reinterpret_cast<float4*>(o) = make_float4(r[0], r[1], r[2], r[3]);
+            *reinterpret_cast<float4*>(o) = make_float4(avg(acc[0]), avg(acc[1]), avg(acc[2]), avg(acc[3]));
         } else {
-            for (uint32_t q = 0; q < nv; ++q) o[q] = r[q];
+            for (uint32_t q = 0; q < nv; ++q) o[q] = avg(acc[q]);
         }
     }
     if (a.sym_out) {
@@ -1187,6 +1180,10 @@ __global__ void __launch_bounds__(kThreads) decode_kernel(DecArgs a) {
 
     if (tid == 0) mbar_init(&sm.bar, 1);
     float carry[kPhases][4];  // running sums across client batches (kMulti only)
+    Averager avg;
+    avg.u = (float)a.n_clients;
+    avg.pow2 = (a.n_clients & (a.n_clients - 1u)) == 0;
+    avg.inv = __fdiv_rn(1.0f, avg.u);
     bool err = false, hw_fail = false;
     uint32_t phase = 0;
 
@@ -1276,7 +1273,7 @@ __global__ void __launch_bounds__(kThreads) decode_kernel(DecArgs a) {
         }
         const bool had_symbols = my != 0;
         const bool first_batch = (u0 == 0), last_batch = (u0 + B >= a.n_clients);
-#pragma unroll
+#pragma unroll(kMulti ? kPhases : 1)
         for (int ph = 0; ph < kPhases; ++ph) {
             // ---- decode this phase's 32 symbols of the sub-chunk
             const uint32_t j0 = ph * kPhaseWords;
@@ -1291,23 +1288,35 @@ __global__ void __launch_bounds__(kThreads) decode_kernel(DecArgs a) {
             // ---- ordered sum over the clients of this batch; a thread owns whole symbol words
             if (kMulti) {
                 if (tid < (uint32_t)kPairPhaseWords) {
+                    const uint32_t s = tid / kPhaseWords, j = tid % kPhaseWords;
                     float acc[4];
 #pragma unroll
                     for (int q = 0; q < 4; ++q) acc[q] = first_batch ? 0.0f : carry[ph][q];
-                    const uint32_t symw = sum_word(sm.val, sm_sym, tid, B, nb, acc);
+                    const uint32_t symw = sum_word(sm.val, sm_sym, 0, s, j, B, nb, acc);
                     if (!last_batch) {
 #pragma unroll
                         for (int q = 0; q < 4; ++q) carry[ph][q] = acc[q];
                     } else {
-                        write_word(a, sm, td, tid, ph, B, acc, symw);
+                        write_word(a, sm, td, 0, s * kS + ph * kPhaseSyms + j * 4, B, avg, acc, symw);
                     }
+                }
+            } else if ((n_thr % kPairPhaseWords) == 0) {
+                // the thread keeps its place inside the chunk and steps over the tile's chunks
+                const uint32_t wi = tid % kPairPhaseWords, s = wi / kPhaseWords, j = wi % kPhaseWords;
+                const uint32_t i0 = s * kS + ph * kPhaseSyms + j * 4;
+                for (uint32_t cl = tid / kPairPhaseWords; cl < G; cl += n_thr / kPairPhaseWords) {
+                    float acc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+                    const uint32_t symw = sum_word(sm.val, sm_sym, cl, s, j, B, nb, acc);
+                    write_word(a, sm, td, cl, i0, B, avg, acc, symw);
                 }
             } else {
                 const uint32_t tile_words = G * kPairPhaseWords;
                 for (uint32_t w = tid; w < tile_words; w += n_thr) {
+                    const uint32_t cl = w / kPairPhaseWords, wi = w % kPairPhaseWords;
+                    const uint32_t s = wi / kPhaseWords, j = wi % kPhaseWords;
                     float acc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-                    const uint32_t symw = sum_word(sm.val, sm_sym, w, B, nb, acc);
-                    write_word(a, sm, td, w, ph, B, acc, symw);
+                    const uint32_t symw = sum_word(sm.val, sm_sym, cl, s, j, B, nb, acc);
+                    write_word(a, sm, td, cl, s * kS + ph * kPhaseSyms + j * 4, B, avg, acc, symw);
                 }
             }
             __syncthreads();  // the phase buffer is free again
