@@ -1064,23 +1064,31 @@ __device__ __forceinline__ uint32_t window_at(const uint32_t* words, uint32_t nw
 
 // Decodes two symbols from the position `pos` on (a codeword has at most 16 bits, so one 32-bit window holds
 // both) and advances it.  Returns the two table entries: symbol in the low byte, 0xff = no codeword matched.
+// Both look-ups are done assuming short codewords and tested together; if either hit a second-level marker
+// the pair is redone step by step.
 template <bool kChecked, bool kSecond>
 __device__ __forceinline__ void decode_two(const uint32_t* words, uint32_t nwords, uint32_t& pos,
                                            const uint16_t* __restrict__ s_lut, const uint16_t* __restrict__ sub_tab,
                                            uint32_t& e0, uint32_t& e1) {
-    uint32_t win = window_at<kChecked>(words, nwords, pos);
+    const uint32_t win = window_at<kChecked>(words, nwords, pos);
     e0 = s_lut[win >> (32 - kDecBits)];
-    if (e0 >= kDecLong) e0 = decode_long(sub_tab, e0, win);
-    const uint32_t l0 = e0 >> 8;
-    e1 = 0;
-    uint32_t l1 = 0;
-    if (kSecond) {
-        win <<= l0;
-        e1 = s_lut[win >> (32 - kDecBits)];
-        if (e1 >= kDecLong) e1 = decode_long(sub_tab, e1, win);
-        l1 = e1 >> 8;
+    if (!kSecond) {
+        if (e0 >= kDecLong) e0 = decode_long(sub_tab, e0, win);
+        e1 = 0;
+        pos += e0 >> 8;
+        return;
     }
-    pos += l0 + l1;
+    uint32_t l0 = e0 >> 8;
+    uint32_t win1 = win << (l0 & 31u);  // a marker's "length" is meaningless: keep the shift defined
+    e1 = s_lut[win1 >> (32 - kDecBits)];
+    if ((e0 | e1) >= kDecLong) {
+        if (e0 >= kDecLong) e0 = decode_long(sub_tab, e0, win);
+        l0 = e0 >> 8;
+        win1 = win << l0;
+        e1 = s_lut[win1 >> (32 - kDecBits)];
+        if (e1 >= kDecLong) e1 = decode_long(sub_tab, e1, win1);
+    }
+    pos += l0 + (e1 >> 8);
 }
 
 // One phase of one sub-chunk: decodes symbols [4 * j0, 4 * j0 + 32) of the sub-chunk (those below `my`) from bit
@@ -1119,9 +1127,12 @@ struct Averager {
 __device__ __forceinline__ uint32_t sum_word(const float* __restrict__ val, const uint32_t* __restrict__ sym, uint32_t cl,
                                              uint32_t s, uint32_t j, uint32_t B, uint32_t nb, float (&acc)[4]) {
     uint32_t symw = 0;
-    for (uint32_t ul = 0; ul < nb; ++ul) {
-        const uint32_t p = cl * B + ul;
-        symw = sym[p * kPairPhaseWords + sym_slot(p, s, j)];
+    uint32_t p = cl * B;
+    const uint32_t* row = sym + p * kPairPhaseWords + s * kPhaseWords;
+    const uint32_t rot = j + (s >> 2);
+#pragma unroll 2
+    for (uint32_t ul = 0; ul < nb; ++ul, ++p, row += kPairPhaseWords) {
+        symw = row[(rot + 4u * (p & 1u)) & (kPhaseWords - 1)];
 #pragma unroll
         for (int q = 0; q < 4; ++q) acc[q] = __fadd_rn(acc[q], val[(symw >> (8 * q)) & 0xffu]);
     }
