@@ -529,16 +529,24 @@ struct PackArgs {
 
 // ORs an n-bit value (v, right-aligned, n <= 64, bits above n clear) into the bit buffer so that its last
 // bit lands on stream bit end-1 (most significant bit first).  Words that receive only zeros are skipped.
+__device__ __forceinline__ void or_if_nonzero(uint32_t* word, uint32_t v) {
+    // a predicated shared-memory reduction: no branch around it
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.u32 p, %1, 0;\n\t"
+        "@p red.shared.or.b32 [%0], %1;\n\t}"
+        :
+        : "r"(smem_addr(word)), "r"(v)
+        : "memory");
+}
+
 __device__ __forceinline__ void put_bits(uint32_t* buf, uint32_t end, uint64_t v) {
     const uint32_t lo = (uint32_t)v, hi = (uint32_t)(v >> 32);
     const uint32_t q = (0u - end) & 31u;  // free bits behind the value in its last word
-    const uint32_t wl = (end + 31u) >> 5;  // one past the last word touched
-    const uint32_t w2 = lo << q;
-    const uint32_t w1 = __funnelshift_l(lo, hi, q);
-    const uint32_t w0 = __funnelshift_l(hi, 0u, q);
-    if (w2) atomicOr(&buf[wl - 1], w2);
-    if (w1) atomicOr(&buf[wl - 2], w1);
-    if (w0) atomicOr(&buf[wl - 3], w0);
+    uint32_t* last = buf + ((end + 31u) >> 5);  // one past the last word touched
+    or_if_nonzero(last - 1, lo << q);
+    or_if_nonzero(last - 2, __funnelshift_l(lo, hi, q));
+    or_if_nonzero(last - 3, __funnelshift_l(hi, 0u, q));
 }
 
 constexpr int kBitWords = kSlotWords + 4;  // bit buffer of one chunk, multiple of four words
