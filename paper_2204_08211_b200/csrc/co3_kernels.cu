@@ -382,7 +382,7 @@ __device__ __forceinline__ void feed_fetch_fmt(Feed& fd, const Ws& ws, uint32_t 
 // All threads: this thread's 8 gradient and memory values of the current item.  Returns false if the
 // copies never arrived (never expected).
 // `parity` holds, per ring slot, the phase parity of the next copy to wait for.
-__device__ __forceinline__ bool feed_read(Feed& fd, const FeedArgs& fa, const FeedItem& it, uint64_t k, uint32_t i0,
+__device__ __forceinline__ bool feed_read(Feed& fd, const FeedArgs& fa, const FeedItem& it, uint32_t k, uint32_t i0,
                                           uint32_t nv, uint32_t& parity, float (&g)[8], float (&m)[8]) {
     if (it.tma) {
         const uint32_t slot = (uint32_t)k & 1u;
@@ -527,29 +527,30 @@ struct PackArgs {
     Ws ws;
 };
 
-// ORs an n-bit value (v, right-aligned, n <= 64, bits above n clear) into the bit buffer so that its last
-// bit lands on stream bit end-1 (most significant bit first).  Words that receive only zeros are skipped.
-__device__ __forceinline__ void or_if_nonzero(uint32_t* word, uint32_t v) {
-    // a predicated shared-memory reduction: no branch around it
+// ORs an n-bit value (v, right-aligned, n <= 64, bits above n clear) into the chunk's bit buffer so that its
+// last bit lands on stream bit end-1 (most significant bit first).  Words that receive only zeros are skipped.
+__device__ __forceinline__ void or_if_nonzero(uint32_t word_addr, uint32_t v) {
+    // a predicated shared-memory reduction: no branch around it; word_addr is a shared-window byte address
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
         "setp.ne.u32 p, %1, 0;\n\t"
         "@p red.shared.or.b32 [%0], %1;\n\t}"
         :
-        : "r"(smem_addr(word)), "r"(v)
+        : "r"(word_addr), "r"(v)
         : "memory");
 }
 
-__device__ __forceinline__ void put_bits(uint32_t* buf, uint32_t end, uint64_t v) {
+// buf_addr: shared-window byte address of the chunk's bit buffer.
+__device__ __forceinline__ void put_bits(uint32_t buf_addr, uint32_t end, uint64_t v) {
     const uint32_t lo = (uint32_t)v, hi = (uint32_t)(v >> 32);
     const uint32_t q = (0u - end) & 31u;  // free bits behind the value in its last word
-    uint32_t* last = buf + ((end + 31u) >> 5);  // one past the last word touched
-    or_if_nonzero(last - 1, lo << q);
-    or_if_nonzero(last - 2, __funnelshift_l(lo, hi, q));
-    or_if_nonzero(last - 3, __funnelshift_l(hi, 0u, q));
+    const uint32_t last = buf_addr + (((end + 31u) >> 5) << 2);  // one past the last word touched
+    or_if_nonzero(last - 4u, lo << q);
+    or_if_nonzero(last - 8u, __funnelshift_l(lo, hi, q));
+    or_if_nonzero(last - 12u, __funnelshift_l(hi, 0u, q));
 }
 
-constexpr int kBitWords = kSlotWords + 4;  // bit buffer of one chunk, multiple of four words
+constexpr int kBitWords = kSlotWords;  // bit buffer of one chunk: one uint4 per thread
 
 // Exclusive prefix sum over the 256 threads of a block with one barrier; *total receives the block sum.
 // scratch: 8 words that no thread writes again before the block's next barrier after this call.
@@ -587,7 +588,7 @@ struct PackSmem {
 // Returns the chunk's total bit count; `missing` reports a symbol without codeword.
 template <bool kFromSym, bool kWhole>
 __device__ __forceinline__ uint32_t pack_item(const PackArgs& a, PackSmem& sm, const FeedArgs& fa, const FeedItem& it,
-                                              uint64_t k, uint32_t& parity, uint32_t& enc_seg, uint32_t& n_sat,
+                                              uint32_t k, uint32_t& parity, uint32_t& enc_seg, uint32_t& n_sat,
                                               uint32_t& n_nf, bool& hw_fail, bool& missing, uint32_t& off_out) {
     const uint32_t tid = threadIdx.x, i0 = tid * 8;
     const uint32_t nv = kWhole ? 8u : (it.d.cnt > i0 ? min(8u, it.d.cnt - i0) : 0u);
@@ -633,8 +634,8 @@ __device__ __forceinline__ uint32_t pack_item(const PackArgs& a, PackSmem& sm, c
     const uint32_t off = block_exclusive_scan_once(la + lb, sm.scan[k & 1u], &total);
     // Behind the scan's barrier every thread has finished the previous item's copy-out and this item's table
     // look-ups: clear the other bit buffer and fetch the next item's tables.
-    for (uint32_t i = tid; i < (uint32_t)kBitWords / 4; i += kThreads)
-        reinterpret_cast<uint4*>(sm.bits[(k + 1) & 1u])[i] = make_uint4(0, 0, 0, 0);
+    static_assert(kBitWords == 4 * kThreads, "one uint4 of the bit buffer per thread");
+    reinterpret_cast<uint4*>(sm.bits[(k + 1) & 1u])[tid] = make_uint4(0, 0, 0, 0);
     const FeedItem& nx = sm.feed.item[(k + 1) & 1u];
     if (nx.valid && nx.d.seg != enc_seg) {
         enc_seg = nx.d.seg;
@@ -642,9 +643,9 @@ __device__ __forceinline__ uint32_t pack_item(const PackArgs& a, PackSmem& sm, c
     }
     if (!kFromSym) feed_fetch_fmt(sm.feed, a.ws, (uint32_t)(k + 1) & 1u);
     if (!missing) {
-        uint32_t* bits = sm.bits[k & 1u];
-        put_bits(bits, off + la, wa);
-        put_bits(bits, off + la + lb, wb);
+        const uint32_t bits_addr = smem_addr(sm.bits[k & 1u]);
+        put_bits(bits_addr, off + la, wa);
+        put_bits(bits_addr, off + la + lb, wb);
     }
     off_out = off;
     return total;
@@ -668,7 +669,7 @@ __global__ void __launch_bounds__(kThreads, 4) pack_kernel(PackArgs a) {
         next = a.ws.chunk_desc[blockIdx.x % n_chunks];
         feed_issue(sm.feed, fa, a.ws, n_chunks, 0, next, !kFromSym);
     }
-    for (uint32_t i = tid; i < (uint32_t)kBitWords / 4; i += kThreads) reinterpret_cast<uint4*>(sm.bits[0])[i] = make_uint4(0, 0, 0, 0);
+    reinterpret_cast<uint4*>(sm.bits[0])[tid] = make_uint4(0, 0, 0, 0);
     __syncthreads();
     uint32_t enc_seg = sm.feed.item[0].valid ? sm.feed.item[0].d.seg : 0u;
     sm.enc[tid] = a.ws.enc_lut[enc_seg * 256 + tid];
@@ -678,7 +679,7 @@ __global__ void __launch_bounds__(kThreads, 4) pack_kernel(PackArgs a) {
 
     uint32_t n_sat = 0, n_nf = 0, cur_client = 0, parity = 0;
     bool hw_fail = false;
-    for (uint64_t k = 0;; ++k) {
+    for (uint32_t k = 0;; ++k) {
         // item k + 1 goes into the ring slot and descriptor that item k - 1 used; every thread is past the
         // last barrier of item k - 1 and read them before it
         if (tid == 0) feed_issue(sm.feed, fa, a.ws, n_chunks, k + 1, next, !kFromSym);
@@ -708,9 +709,11 @@ __global__ void __launch_bounds__(kThreads, 4) pack_kernel(PackArgs a) {
         const size_t ci = (size_t)it.client * a.ws.n_chunks_max + chunk;
         if (tid == 0) a.ws.chunk_bits[ci] = total;
         const uint32_t words = (total + 31u) >> 5;
-        uint32_t* slot = a.ws.slots + ci * kSlotWords;
-        const uint32_t* bits = sm.bits[k & 1u];
-        for (uint32_t i = tid; i < words; i += kThreads) slot[i] = bits[i];
+        uint32_t* slot = a.ws.slots + ci * kSlotWords + tid;
+        const uint32_t* bits = sm.bits[k & 1u] + tid;
+#pragma unroll
+        for (int r = 0; r < kSlotWords / kThreads; ++r)
+            if (tid + r * kThreads < words) slot[r * kThreads] = bits[r * kThreads];
     }
     if (!kFromSym) add_counts(&a.res[cur_client], n_sat, n_nf);
     if (__syncthreads_or(hw_fail) && tid == 0) set_status(&a.res[cur_client], CO3_ERR_CUDA);
