@@ -322,12 +322,31 @@ struct FeedItem {
     uint32_t chunk;   // chunk index inside the client
 };
 
+// Thread 0's position in the item sequence: item i of this block is item blockIdx.x + i * gridDim.x of the
+// batch, i.e. (client, chunk) advanced by gridDim.x chunks per step, without any 64-bit division.
+struct FeedCursor {
+    uint32_t client, chunk;            // the item to publish next
+    uint32_t step_client, step_chunk;  // gridDim.x as (whole clients, chunks)
+    __device__ __forceinline__ void init(uint32_t n_chunks) {
+        client = blockIdx.x / n_chunks;
+        chunk = blockIdx.x % n_chunks;
+        step_client = gridDim.x / n_chunks;
+        step_chunk = gridDim.x % n_chunks;
+    }
+    __device__ __forceinline__ void advance(uint32_t n_chunks) {
+        client += step_client;
+        chunk += step_chunk;
+        if (chunk >= n_chunks) { chunk -= n_chunks; ++client; }
+    }
+};
+
 struct Feed {
     float g[2][kC];
     float m[2][kC];
     uint64_t bar[2];
     FeedItem item[2];
     FmtDev fmt[2];    // converter constants of the item in each slot
+    FeedCursor cur;   // thread 0's place in the item sequence (kept here to spare every thread the registers)
 };
 
 struct FeedArgs {
@@ -337,27 +356,23 @@ struct FeedArgs {
     uint32_t n_clients;
 };
 
-// Thread 0 only: publishes item k in ring slot k & 1 and starts its copies.  `next` holds the chunk
-// descriptor fetched one call earlier for exactly this item; it is refilled for item k + 1.
-__device__ __forceinline__ void feed_issue(Feed& fd, const FeedArgs& fa, const Ws& ws, uint32_t n_chunks, uint64_t k,
+// Thread 0 only: publishes the cursor's item in ring slot `slot` and starts its copies.  `next` holds the chunk
+// descriptor fetched one call earlier for exactly this item; the cursor moves on and `next` is refilled.
+__device__ __forceinline__ void feed_issue(Feed& fd, const FeedArgs& fa, const Ws& ws, uint32_t n_chunks, uint32_t slot,
                                            ChunkDesc& next, bool use_tma) {
-    const uint64_t total = (uint64_t)n_chunks * fa.n_clients;
-    const uint64_t idx = blockIdx.x + k * gridDim.x;
+    FeedCursor cur = fd.cur;
     FeedItem it;
-    it.valid = idx < total ? 1u : 0u;
+    it.valid = cur.client < fa.n_clients ? 1u : 0u;
     it.d = next;
-    it.client = 0;
+    it.client = cur.client;
+    it.chunk = cur.chunk;
     it.base = 0;
     it.tma = 0;
-    it.chunk = 0;
     if (it.valid) {
-        it.client = (uint32_t)(idx / n_chunks);
-        it.chunk = (uint32_t)(idx - (uint64_t)it.client * n_chunks);
         it.base = (uint64_t)it.client * fa.client_stride + it.d.elem0;
         const uintptr_t pg = reinterpret_cast<uintptr_t>(fa.grad + it.base), pm = reinterpret_cast<uintptr_t>(fa.mem + it.base);
         it.tma = (use_tma && it.d.cnt == (uint32_t)kC && ((pg | pm) & 15u) == 0) ? 1u : 0u;
     }
-    const uint32_t slot = (uint32_t)k & 1u;
     fd.item[slot] = it;
     if (it.tma) {
         fence_async_smem();
@@ -365,8 +380,9 @@ __device__ __forceinline__ void feed_issue(Feed& fd, const FeedArgs& fa, const W
         bulk_copy_g2s(fd.g[slot], fa.grad + it.base, kC * 4u, &fd.bar[slot]);
         bulk_copy_g2s(fd.m[slot], fa.mem + it.base, kC * 4u, &fd.bar[slot]);
     }
-    const uint64_t idx_next = idx + gridDim.x;
-    if (idx_next < total) next = ws.chunk_desc[idx_next % n_chunks];
+    cur.advance(n_chunks);
+    fd.cur = cur;
+    if (cur.client < fa.n_clients) next = ws.chunk_desc[cur.chunk];
 }
 
 // The first threads of warp 0 copy the converter constants of the item in ring slot `slot` next to it; visible to the
@@ -420,7 +436,7 @@ constexpr int kHistCopies = 8;    // private histograms per block, spread over t
 constexpr int kHistStride = 260;  // words between copies: shifts each copy by four banks
 
 template <bool kSym, bool kHist>
-__global__ void __launch_bounds__(kThreads, 4) convert_kernel(ConvertArgs a) {
+__global__ void __launch_bounds__(kThreads, 3) convert_kernel(ConvertArgs a) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     Feed& fd = *reinterpret_cast<Feed*>(smem_raw);
     uint32_t* s_hist = reinterpret_cast<uint32_t*>(smem_raw + sizeof(Feed));
@@ -435,7 +451,8 @@ __global__ void __launch_bounds__(kThreads, 4) convert_kernel(ConvertArgs a) {
     if (tid == 0) {
         mbar_init(&fd.bar[0], 1);
         mbar_init(&fd.bar[1], 1);
-        next = a.ws.chunk_desc[blockIdx.x % n_chunks];
+        fd.cur.init(n_chunks);
+        next = a.ws.chunk_desc[fd.cur.chunk];
         feed_issue(fd, fa, a.ws, n_chunks, 0, next, true);
     }
     if (kHist)
@@ -448,7 +465,7 @@ __global__ void __launch_bounds__(kThreads, 4) convert_kernel(ConvertArgs a) {
     bool hw_fail = false;
     const uint32_t i0 = tid * 8;
     for (uint64_t k = 0;; ++k) {
-        if (tid == 0) feed_issue(fd, fa, a.ws, n_chunks, k + 1, next, true);
+        if (tid == 0) feed_issue(fd, fa, a.ws, n_chunks, (uint32_t)(k + 1) & 1u, next, true);
         const FeedItem it = fd.item[k & 1u];
         if (!it.valid) break;
         if (it.client != cur_client) {  // counters are per client
@@ -575,11 +592,20 @@ __device__ __forceinline__ uint32_t block_exclusive_scan_once(uint32_t x, uint32
     return base + inc - x;
 }
 
+// Where the results of one work item go, worked out once per item by thread 0.
+struct PackOut {
+    uint16_t* sub;       // the chunk's 16 sub-chunk offsets in the client's container
+    uint32_t* slot;      // the chunk's worst-case slot in the workspace
+    uint32_t* chunk_bits;
+    co3_result* res;     // the client's result
+};
+
 struct PackSmem {
     Feed feed;
     uint32_t bits[2][kBitWords];
     uint32_t enc[256];
     uint32_t scan[2][8];
+    PackOut out[2];
 };
 
 // One work item of the pack kernel for one thread: symbols of its 8 elements (converted here unless
@@ -651,8 +677,20 @@ __device__ __forceinline__ uint32_t pack_item(const PackArgs& a, PackSmem& sm, c
     return total;
 }
 
+// Thread 0 only: output locations of the item just published in ring slot `slot`.
+__device__ __forceinline__ void pack_out_set(const PackArgs& a, PackSmem& sm, uint32_t slot, uint64_t sub_off) {
+    const FeedItem& it = sm.feed.item[slot];
+    PackOut o;
+    const size_t ci = (size_t)it.client * a.ws.n_chunks_max + it.chunk;
+    o.sub = reinterpret_cast<uint16_t*>(a.streams + (size_t)it.client * a.stream_capacity + sub_off) + (size_t)it.chunk * kSubs;
+    o.slot = a.ws.slots + ci * kSlotWords;
+    o.chunk_bits = a.ws.chunk_bits + ci;
+    o.res = a.res + it.client;
+    sm.out[slot] = o;
+}
+
 template <bool kFromSym>
-__global__ void __launch_bounds__(kThreads, 4) pack_kernel(PackArgs a) {
+__global__ void __launch_bounds__(kThreads, 3) pack_kernel(PackArgs a) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     PackSmem& sm = *reinterpret_cast<PackSmem*>(smem_raw);
     const Ctrl* ctrl = a.ws.ctrl;
@@ -661,20 +699,22 @@ __global__ void __launch_bounds__(kThreads, 4) pack_kernel(PackArgs a) {
     const uint32_t n_chunks = ctrl->n_chunks;
     const FeedArgs fa{a.grad, a.mem, a.client_stride, a.n_clients};
     if ((uint64_t)blockIdx.x >= (uint64_t)n_chunks * a.n_clients) return;
+    const uint64_t sub_off = ctrl->sub_off;
 
     ChunkDesc next{};
     if (tid == 0) {
         mbar_init(&sm.feed.bar[0], 1);
         mbar_init(&sm.feed.bar[1], 1);
-        next = a.ws.chunk_desc[blockIdx.x % n_chunks];
+        sm.feed.cur.init(n_chunks);
+        next = a.ws.chunk_desc[sm.feed.cur.chunk];
         feed_issue(sm.feed, fa, a.ws, n_chunks, 0, next, !kFromSym);
+        pack_out_set(a, sm, 0, sub_off);
     }
     reinterpret_cast<uint4*>(sm.bits[0])[tid] = make_uint4(0, 0, 0, 0);
     __syncthreads();
     uint32_t enc_seg = sm.feed.item[0].valid ? sm.feed.item[0].d.seg : 0u;
     sm.enc[tid] = a.ws.enc_lut[enc_seg * 256 + tid];
     feed_fetch_fmt(sm.feed, a.ws, 0);
-    const uint64_t sub_off = ctrl->sub_off;
     __syncthreads();
 
     uint32_t n_sat = 0, n_nf = 0, cur_client = 0, parity = 0;
@@ -682,7 +722,10 @@ __global__ void __launch_bounds__(kThreads, 4) pack_kernel(PackArgs a) {
     for (uint32_t k = 0;; ++k) {
         // item k + 1 goes into the ring slot and descriptor that item k - 1 used; every thread is past the
         // last barrier of item k - 1 and read them before it
-        if (tid == 0) feed_issue(sm.feed, fa, a.ws, n_chunks, k + 1, next, !kFromSym);
+        if (tid == 0) {
+            feed_issue(sm.feed, fa, a.ws, n_chunks, (k + 1) & 1u, next, !kFromSym);
+            pack_out_set(a, sm, (k + 1) & 1u, sub_off);
+        }
         const FeedItem it = sm.feed.item[k & 1u];
         if (!it.valid) break;
         if (!kFromSym && it.client != cur_client) {
@@ -695,21 +738,18 @@ __global__ void __launch_bounds__(kThreads, 4) pack_kernel(PackArgs a) {
         const bool whole = kFromSym ? it.d.cnt == (uint32_t)kC : it.tma != 0;
         if (whole) total = pack_item<kFromSym, true>(a, sm, fa, it, k, parity, enc_seg, n_sat, n_nf, hw_fail, missing, off);
         else total = pack_item<kFromSym, false>(a, sm, fa, it, k, parity, enc_seg, n_sat, n_nf, hw_fail, missing, off);
-        uint8_t* stream = a.streams + (size_t)it.client * a.stream_capacity;
-        const uint32_t chunk = it.chunk;
-        if ((tid & 15u) == 0)
-            *reinterpret_cast<uint16_t*>(stream + sub_off + 2ull * ((uint64_t)chunk * kSubs + (tid >> 4))) = (uint16_t)off;
+        const PackOut out = sm.out[k & 1u];
+        if ((tid & 15u) == 0) out.sub[tid >> 4] = (uint16_t)off;
         if (__syncthreads_or(missing)) {  // bit buffer complete
             if (tid == 0) {
-                set_status(&a.res[it.client], CO3_ERR_NO_CODEWORD);
-                atomicMin(&a.res[it.client].first_bad_chunk, chunk);
+                set_status(out.res, CO3_ERR_NO_CODEWORD);
+                atomicMin(&out.res->first_bad_chunk, it.chunk);
                 a.ws.client_fail[it.client] = 1u;
             }
         }
-        const size_t ci = (size_t)it.client * a.ws.n_chunks_max + chunk;
-        if (tid == 0) a.ws.chunk_bits[ci] = total;
+        if (tid == 0) *out.chunk_bits = total;
         const uint32_t words = (total + 31u) >> 5;
-        uint32_t* slot = a.ws.slots + ci * kSlotWords + tid;
+        uint32_t* slot = out.slot + tid;
         const uint32_t* bits = sm.bits[k & 1u] + tid;
 #pragma unroll
         for (int r = 0; r < kSlotWords / kThreads; ++r)
