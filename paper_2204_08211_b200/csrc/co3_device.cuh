@@ -150,27 +150,25 @@ __device__ __forceinline__ float convert_one(float g, float m, float decay, cons
 // The same update without branches, for formats with M >= 1 that keep the sub-normal levels.
 // Rounding by one fp32 addition: with ae the (clamped) exponent of |t|, |t| + 2^(ae + 23 - M) is rounded by
 // the adder to a multiple of the format's step in that binade, ties to the even multiple, which has the
-// even code when M >= 1.  Saturation and non-finite inputs are only detected here (a_max > top_bits,
-// nf_acc != nf_acc); the caller then repeats the element group with convert_one, which also counts them.
+// even code when M >= 1.  Saturating and non-finite inputs all land on the largest code (NaN and Inf compare
+// above the largest level), so the caller only watches for that code (code_max) and, when it shows up in a
+// group, repeats the group with convert_one, which tells those cases apart and counts them.
 __device__ __forceinline__ float convert_fast(float g, float m, float decay, const FmtDev& f, uint32_t& sym,
-                                              uint32_t& a_max, float& nf_acc) {
+                                              uint32_t& code_max) {
     const float v = __fmaf_rn(decay, m, g);
     const float t = __fmul_rn(v, f.scale);
-    const uint32_t tb = __float_as_uint(t);
-    const uint32_t a = tb & 0x7fffffffu;
-    const uint32_t ac = min(a, f.top_bits);
-    a_max = max(a_max, a);  // beyond f.top_bits iff some input saturated
+    const float at = fminf(fabsf(t), __uint_as_float(f.top_bits));  // NaN -> largest level
+    const uint32_t ac = __float_as_uint(at);
     const uint32_t ae = max(ac & 0x7f800000u, f.min_normal_bits);
     const uint32_t mg = ae + (f.drop << 23);
-    const float s = __fadd_rn(__uint_as_float(ac), __uint_as_float(mg));
+    const float s = __fadd_rn(at, __uint_as_float(mg));
     const uint32_t code = ((ae - f.min_normal_bits) >> f.drop) + (__float_as_uint(s) - mg);
+    code_max = max(code_max, code);
     const float qmag = __fsub_rn(s, __uint_as_float(mg));
-    const uint32_t sgn = code ? (tb & 0x80000000u) : 0u;
+    const uint32_t sgn = code ? (__float_as_uint(t) & 0x80000000u) : 0u;
     sym = code | (sgn >> f.sign_shift);
     const float ghat = __fmul_rn(__uint_as_float(__float_as_uint(qmag) | sgn), f.inv_scale);
-    const float m_new = __fsub_rn(v, ghat);
-    nf_acc = __fmaf_rn(m_new, 0.0f, nf_acc);  // NaN iff some m_new is not finite, i.e. some v was not
-    return m_new;
+    return __fsub_rn(v, ghat);
 }
 
 // ------------------------------------------------------------------------------------------------
