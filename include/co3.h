@@ -220,12 +220,12 @@ int co3_decode(const uint8_t* stream_in, size_t stream_bytes,
  * 16384 launches are recorded between reads.  Not thread-safe, and not to be left on inside a
  * stream capture.
  */
-#define CO3_KERNEL_PREPARE 0  /* descriptor validation and derived tables */
+#define CO3_KERNEL_PREPARE 0  /* descriptor (and, when decoding, stream header) validation, derived tables */
 #define CO3_KERNEL_CONVERT 1  /* correct + convert + memory update (+ symbols, histogram) */
 #define CO3_KERNEL_PACK 2     /* (correct + convert + memory update +) codeword lookup, scan, bit packing */
 #define CO3_KERNEL_SCAN 3     /* chunk offsets, header, tables */
 #define CO3_KERNEL_COMPACT 4  /* payload compaction */
-#define CO3_KERNEL_CHECK 5    /* stream header validation */
+#define CO3_KERNEL_CHECK 5    /* unused (stream validation is part of CO3_KERNEL_PREPARE) */
 #define CO3_KERNEL_DECODE 6   /* decode + cross-client accumulate */
 #define CO3_KERNEL_COUNT 7
 int co3_profile_enable(int on);

@@ -31,8 +31,41 @@ struct PrepArgs {
     uint32_t tile_chunks;  // chunks per decode tile
     co3_result* res;
     uint32_t n_res;
+    uint32_t want_dec;     // build the decode tables (decode calls only)
+    // decode calls: the streams to validate against the layout (n_streams = 0 otherwise)
+    const uint8_t* const* streams;  // device array of pointers, or null:
+    const uint8_t* single;          // the one stream
+    size_t stream_bytes;
+    uint32_t n_streams;
     Ws ws;
 };
+
+__device__ __forceinline__ const uint8_t* prep_stream(const PrepArgs& a, uint32_t u) {
+    return a.streams ? a.streams[u] : a.single;
+}
+
+// A stream failed validation: the decode kernel must not run.
+__device__ void fail_corrupt(const PrepArgs& a) {
+    a.ws.ctrl->abort = 1u;
+    set_status(&a.res[0], CO3_ERR_CORRUPT);
+}
+
+// Header of stream u against the layout (n_chunks chunks, payload at payload_off).  One thread per stream.
+__device__ bool header_ok(const PrepArgs& a, uint32_t u, uint64_t n_chunks, uint64_t chunk_off, uint64_t payload_off) {
+    const uint8_t* stream = prep_stream(a, u);
+    if (stream == nullptr || (reinterpret_cast<uintptr_t>(stream) & 15u) || a.stream_bytes < payload_off) return false;
+    const uint32_t* h32 = reinterpret_cast<const uint32_t*>(stream);
+    const uint64_t* h64 = reinterpret_cast<const uint64_t*>(stream);
+    const uint64_t cap_words = (a.stream_bytes - payload_off) / 4;
+    if (h32[0] != kMagic || h32[1] != 1u || h32[2] != a.n_seg || h32[3] != (uint32_t)kC || h32[4] != (uint32_t)kS ||
+        h64[3] != a.n_elem || h64[4] != n_chunks || h64[5] > cap_words || h64[7] > a.stream_bytes ||
+        h64[7] != align16(payload_off + 4ull * h64[5]))
+        return false;
+    if (reinterpret_cast<const uint64_t*>(stream + chunk_off)[n_chunks] != h64[5]) return false;
+    atomicAdd(reinterpret_cast<unsigned long long*>(&a.res[0].payload_bits), (unsigned long long)h64[6]);
+    atomicAdd(reinterpret_cast<unsigned long long*>(&a.res[0].container_bytes), (unsigned long long)h64[7]);
+    return true;
+}
 
 __device__ void fail_all(const PrepArgs& a, int code) {
     a.ws.ctrl->abort = 1u;
@@ -87,6 +120,9 @@ __global__ void __launch_bounds__(kThreads) prepare_kernel(PrepArgs a) {
             c->payload_off = c->sub_off;
             a.ws.first_chunk[0] = 0;
             if (a.n_elem != 0) fail_all(a, CO3_ERR_INVALID_ARG);
+            else
+                for (uint32_t u = 0; u < a.n_streams; ++u)
+                    if (!header_ok(a, u, 0, c->chunk_off, c->payload_off)) fail_corrupt(a);
         }
         return;
     }
@@ -111,6 +147,28 @@ __global__ void __launch_bounds__(kThreads) prepare_kernel(PrepArgs a) {
             c->sub_off = align16(c->chunk_off + 8ull * (nc + 1ull));
             c->payload_off = align16(c->sub_off + 2ull * nc * kSubs);
         }
+    }
+    // decode calls: every stream must describe exactly this layout (this block checks its segment's entry, the
+    // last segment's block the headers)
+    if (blockIdx.y == 0 && a.n_streams) {
+        bool corrupt = false;
+        for (uint32_t u = tid; u < a.n_streams; u += kThreads) {
+            const uint8_t* stream = prep_stream(a, u);
+            if (stream == nullptr || (reinterpret_cast<uintptr_t>(stream) & 15u) ||
+                a.stream_bytes < kHeaderBytes + 24ull * (k + 1ull)) {
+                corrupt = true;
+                continue;
+            }
+            const uint64_t* e = reinterpret_cast<const uint64_t*>(stream + kHeaderBytes + 24ull * k);
+            if (e[0] != sg.n_elem || e[1] != c_before) corrupt = true;
+            if (k == a.n_seg - 1) {
+                const uint64_t nc = c_before + my_chunks;
+                const uint64_t chunk_off = align16(kHeaderBytes + 24ull * a.n_seg);
+                const uint64_t payload_off = align16(align16(chunk_off + 8ull * (nc + 1ull)) + 2ull * nc * kSubs);
+                if (!header_ok(a, u, nc, chunk_off, payload_off)) corrupt = true;
+            }
+        }
+        if (corrupt) fail_corrupt(a);
     }
     // descriptors: blockIdx.y strides over them, so that one long segment is laid out by many blocks
     for (uint64_t c = (uint64_t)blockIdx.y * kThreads + tid; c < my_chunks; c += (uint64_t)gridDim.y * kThreads) {
@@ -182,24 +240,30 @@ __global__ void __launch_bounds__(kThreads) prepare_kernel(PrepArgs a) {
     // ---- code tables
     bool code_ok = true;
     if (a.codes) {
+        __shared__ uint32_t s_code[256];  // bits << 8 | len of every symbol
         const uint32_t len = a.codes[k].len[tid], bits = a.codes[k].bits[tid];
         if (tid == 0) s_kraft = 0;
         __syncthreads();
         if (len > CO3_MAX_CODE_LEN || (len && (bits >> len))) code_ok = false;
         if (tid == 255 && len) code_ok = false;  // 0xff is a symbol of no format: the decoder uses it as its error mark
         if (code_ok && len) atomicAdd(&s_kraft, 1u << (CO3_MAX_CODE_LEN - len));
+        s_code[tid] = code_ok ? ((bits << 8) | len) : 0u;
         a.ws.enc_lut[k * 256 + tid] = (code_ok && len) ? ((bits << 8) | len) : kEncMissing;
         uint16_t* lut = a.ws.dec_lut + (size_t)k * kDecLut;
         uint16_t* sub = a.ws.dec_sub + (size_t)k * kSubLut;
-        for (uint32_t i = tid; i < (uint32_t)kDecLut; i += kThreads) lut[i] = (uint16_t)kDecInvalid;
-        for (uint32_t i = tid; i < (uint32_t)kSubLut; i += kThreads) sub[i] = (uint16_t)kDecInvalid;
+        if (a.want_dec) {
+            for (uint32_t i = tid; i < (uint32_t)kDecLut / 2; i += kThreads)
+                reinterpret_cast<uint32_t*>(lut)[i] = kDecInvalid | (kDecInvalid << 16);
+            for (uint32_t i = tid; i < (uint32_t)kSubLut / 2; i += kThreads)
+                reinterpret_cast<uint32_t*>(sub)[i] = kDecInvalid | (kDecInvalid << 16);
+        }
         __syncthreads();
         if (s_kraft > (1u << CO3_MAX_CODE_LEN)) code_ok = false;  // over-subscribed: cannot be prefix-free
         code_ok = __syncthreads_and(code_ok);
-        if (code_ok) {
+        if (code_ok && a.want_dec) {
             // short codewords fill every table entry they prefix: one warp per symbol, lanes over the span
             for (uint32_t sym = tid >> 5; sym < 256; sym += kThreads / 32) {
-                const uint32_t l = a.codes[k].len[sym], b = a.codes[k].bits[sym];
+                const uint32_t l = s_code[sym] & 0xffu, b = s_code[sym] >> 8;
                 if (l == 0 || l > (uint32_t)kDecBits) continue;
                 const uint32_t span = 1u << (kDecBits - l), first = b << (kDecBits - l);
                 for (uint32_t i = tid & 31u; i < span; i += 32) lut[first + i] = (uint16_t)((l << 8) | sym);
@@ -1014,46 +1078,6 @@ __device__ __forceinline__ const uint8_t* stream_of(const DecArgs& a, uint32_t u
     return a.streams ? a.streams[u] : a.single;
 }
 
-// One block per client: the header and the tables must describe exactly the expected layout.
-__global__ void __launch_bounds__(kThreads) check_streams_kernel(DecArgs a) {
-    const Ctrl* ctrl = a.ws.ctrl;
-    if (ctrl->abort) return;
-    const uint32_t u = blockIdx.x, tid = threadIdx.x;
-    const uint8_t* stream = stream_of(a, u);
-    bool bad = false;
-    if (stream == nullptr || (reinterpret_cast<uintptr_t>(stream) & 15u)) {
-        bad = true;
-    } else {
-        const uint32_t* h32 = reinterpret_cast<const uint32_t*>(stream);
-        const uint64_t* h64 = reinterpret_cast<const uint64_t*>(stream);
-        const uint64_t n = ctrl->n_chunks;
-        if (a.stream_bytes < ctrl->payload_off) {
-            bad = true;
-        } else {
-            const uint64_t cap_words = (a.stream_bytes - ctrl->payload_off) / 4;
-            if (h32[0] != kMagic || h32[1] != 1u || h32[2] != a.n_seg || h32[3] != (uint32_t)kC || h32[4] != (uint32_t)kS ||
-                h64[3] != a.n_elem || h64[4] != n || h64[5] > cap_words || h64[7] > a.stream_bytes ||
-                h64[7] != align16(ctrl->payload_off + 4ull * h64[5]))
-                bad = true;
-            if (!bad && reinterpret_cast<const uint64_t*>(stream + ctrl->chunk_off)[n] != h64[5]) bad = true;
-            if (!bad) {
-                for (uint32_t k = tid; k < a.n_seg; k += kThreads) {
-                    const uint64_t* e = reinterpret_cast<const uint64_t*>(stream + kHeaderBytes + 24ull * k);
-                    if (e[0] != a.segs[k].n_elem || e[1] != a.ws.first_chunk[k]) bad = true;
-                }
-            }
-            if (!bad && tid == 0) {
-                atomicAdd(reinterpret_cast<unsigned long long*>(&a.res->payload_bits), (unsigned long long)h64[6]);
-                atomicAdd(reinterpret_cast<unsigned long long*>(&a.res->container_bytes), (unsigned long long)h64[7]);
-            }
-        }
-    }
-    if (__syncthreads_or(bad) && tid == 0) {
-        set_status(a.res, CO3_ERR_CORRUPT);
-        a.ws.ctrl->abort = 1u;
-    }
-}
-
 constexpr int kMaxPairs = 16;          // (chunk, client) pairs decoded side by side in one block
 constexpr int kPaySlotWords = 456;     // staging per pair: 7 bits/symbol plus alignment; larger chunks are read in place
 constexpr int kPaySlack = 72;          // words a reader may run past its chunk before the end check
@@ -1532,11 +1556,12 @@ Profiler g_prof;
 
 int begin_call(const WsLayout& L, const Ws& ws, co3_result* res, uint32_t n_res, cudaStream_t st,
                const co3_fmt* fmts, const co3_code* codes, const co3_seg* segs, uint32_t n_seg, uint64_t n_elem,
-               uint32_t tile_chunks, uint32_t n_fail) {
+               uint32_t tile_chunks, uint32_t n_fail, const uint8_t* const* streams = nullptr,
+               const uint8_t* single = nullptr, size_t stream_bytes = 0, uint32_t n_streams = 0) {
     CO3_CUDA(cudaMemsetAsync(ws.ctrl, 0, sizeof(Ctrl), st));
     CO3_CUDA(cudaMemsetAsync(res, 0, sizeof(co3_result) * (size_t)n_res, st));
     CO3_CUDA(cudaMemsetAsync(ws.client_fail, 0, 4 * (size_t)(n_fail ? n_fail : 1), st));
-    PrepArgs pa{fmts, codes, segs, n_seg, n_elem, tile_chunks, res, n_res, ws};
+    PrepArgs pa{fmts, codes, segs, n_seg, n_elem, tile_chunks, res, n_res, n_streams ? 1u : 0u, streams, single, stream_bytes, n_streams, ws};
     // extra blocks per segment when segments are long (their chunk descriptors are written in parallel)
     const uint64_t per_seg = L.n_chunks_max / (n_seg ? n_seg : 1);
     const uint32_t helpers = (uint32_t)std::min<uint64_t>(128, per_seg / (8 * kThreads) + 1);
@@ -1568,10 +1593,9 @@ int decode_common(const uint8_t* const* streams, const uint8_t* single, size_t s
         const uint64_t want = L.n_chunks_max / (2 * 148) + 1;  // chunks per block that still give two waves
         if (want < G) G = (uint32_t)(want < g_min ? g_min : want);
     }
-    const int rc = begin_call(L, ws, res, 1, st, fmts, codes, segs, n_seg, n_elem, G, 1);
+    const int rc = begin_call(L, ws, res, 1, st, fmts, codes, segs, n_seg, n_elem, G, 1, streams, single, stream_bytes, n_clients);
     if (rc != CO3_OK) return rc;
     DecArgs da{streams, single, stream_bytes, n_clients, segs, n_seg, n_elem, out, sym_out, res, B, G, ws};
-    CO3_LAUNCH(CO3_KERNEL_CHECK, st, check_streams_kernel<<<n_clients, kThreads, 0, st>>>(da));
     const uint32_t tiles = (uint32_t)(L.n_chunks_max / G + n_seg);  // upper bound; surplus blocks return at once
     if (tiles == 0) return CO3_OK;
     const uint32_t n_pairs = B * G;
