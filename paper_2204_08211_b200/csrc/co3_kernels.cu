@@ -1,11 +1,11 @@
 // CUDA kernels of the CO3 uplink pipeline and its parameter-server inverse (sm_100a).
 //
-//   prepare_kernel        descriptor validation + derived tables (chunk map, encode/decode LUTs)
+//   prepare_kernel        descriptor validation + derived tables (chunk map, encode/decode LUTs);
+//                         for decode calls also header / table validation of every stream
 //   convert_kernel        v = g + gamma*m, ghat = Q_fp(v), m = v - ghat, symbols, histogram
 //   pack_kernel           (convert +) codeword lookup, block scan of lengths, bit packing of one chunk
 //   scan_kernel           chunk word offsets, header and tables of one client's container
 //   compact_kernel        chunk payloads from their worst-case slots to their final place
-//   check_streams_kernel  header / table validation before decoding
 //   decode_kernel         chunk-indexed prefix-code decoder fused with the ordered cross-client sum
 #include <cuda_runtime.h>
 #include <stddef.h>
