@@ -644,14 +644,10 @@ __device__ __forceinline__ uint32_t block_exclusive_scan_once(uint32_t x, uint32
     }
     if (lane == 31u) scratch[warp] = inc;
     __syncthreads();
-    uint32_t base = 0, sum = 0;
-#pragma unroll
-    for (int w = 0; w < 8; ++w) {
-        const uint32_t s = scratch[w];
-        if ((uint32_t)w < warp) base += s;
-        sum += s;
-    }
-    *total = sum;
+    // lanes 0..7 hold the warp sums; two warp-wide reductions give the block total and this warp's base
+    const uint32_t s = lane < 8u ? scratch[lane] : 0u;
+    *total = __reduce_add_sync(0xffffffffu, s);
+    const uint32_t base = __reduce_add_sync(0xffffffffu, lane < warp ? s : 0u);
     return base + inc - x;
 }
 
