@@ -251,19 +251,26 @@ def run_ours(args):
     fit = bool(cfg.get("fit_per_round"))
     sym_step = sess.new_client_buffer(torch.uint8) if fit else None
 
-    def step(i):
-        if fit:     # the code is fitted to this round's symbols: convert + histogram, host Huffman, then pack
-            sess.set_codes_from_weights(sess.histogram(grads[i % n_rounds], mems, stream, sym_step))
+    def step_on(g):
+        if fit:     # the code is fitted to this round's symbols: convert + histogram, Huffman tables built on
+                    # the device from that histogram, then pack from the symbols; nothing goes through the host
+            sess.histogram(g, mems, stream, sym_step, to_host=False)
+            sess.set_codes_from_histogram_device(stream)
             sess.encode_symbols(sym_step, stream)
         else:
-            sess.encode(grads[i % n_rounds], mems, stream)
-        sess.decode_aggregate(stream)
+            sess.encode(g, mems, stream)
+        return sess.decode_aggregate(stream)
+
+    def step(i):
+        step_on(grads[i % n_rounds])
 
     def check():
         er = sess.encode_results()
         dr = sess.decode_result()
         if (er["status"] != co3.OK).any() or dr["status"][0] != co3.OK:
             raise RuntimeError("device status: encode %s decode %s" % (er["status"], dr["status"]))
+        if fit and sess.fit_result()["status"][0] != co3.OK:
+            raise RuntimeError("device status: code build %s" % sess.fit_result()["status"])
         return er, dr
 
     def barrier():
@@ -353,8 +360,7 @@ def run_ours(args):
 
     def e2e_step(i):
         dev_g.copy_(host_g[i % n_rounds], non_blocking=True)
-        sess.encode(dev_g, mems, stream)
-        host_avg.copy_(sess.decode_aggregate(stream), non_blocking=True)
+        host_avg.copy_(step_on(dev_g), non_blocking=True)
 
     e2e_step(0)
     barrier()
@@ -425,7 +431,7 @@ def run_ours(args):
                    "layers": sess.n_seg, "format": "[1,%d,%d]" % tuple(cfg["fmt"]), "decay": cfg["decay"],
                    "mean_code_bits": bits / n_local, "container_bits_per_element": 8.0 * container / n_local,
                    "l2": "inputs larger than L2 (%.0f MB of gradients and memory per step)" % (8.0 * n_local / 1e6),
-                   "code": "fitted every step (convert + histogram, host Huffman, pack from symbols)" if fit
+                   "code": "fitted every step (convert + histogram, Huffman tables built on the device, pack from symbols)" if fit
                            else "fitted once before the timed steps, then reused",
                    "parallelism": "replicas" if world > 1 else "single"},
         "gpu_launches": launches_per_step * args.steps,

@@ -165,6 +165,20 @@ int co3_convert_static(const float* grad, float* mem, float decay,
 int co3_code_build(const uint64_t* weights, const co3_fmt* fmt, co3_code* out);
 
 /*
+ * The same construction for n_seg layers at once on the device (one thread block per layer), so that a
+ * code fitted to this round's histogram (co3_convert's hist_out) never leaves the GPU.  Tables are
+ * identical, entry for entry, to co3_code_build's for the same weights and formats.
+ *   weights   [device] uint64[n_seg][256]
+ *   fmts      [device] n_seg
+ *   codes_out [device] n_seg, fully overwritten (length 0, bits 0 for symbols without codeword)
+ *   res       [device] one co3_result: CO3_ERR_INVALID_ARG if any layer has a bad fmt or a weight sum >= 2^63
+ *                      (that layer's table is all zero then); 8-byte aligned
+ * Asynchronous on `stream`; the return value covers only the host-side argument checks.
+ */
+int co3_code_build_device(const uint64_t* weights, const co3_fmt* fmts, uint32_t n_seg, co3_code* codes_out,
+                          co3_result* res, void* stream);
+
+/*
  * Client uplink for n_clients clients: correct + convert + encode + memory update, codes given.
  *   streams_out [device]  client u's container starts at streams_out + u * stream_capacity
  *                         (stream_capacity a multiple of 16); layout below
@@ -225,7 +239,7 @@ int co3_decode(const uint8_t* stream_in, size_t stream_bytes,
 #define CO3_KERNEL_PACK 2     /* (correct + convert + memory update +) codeword lookup, scan, bit packing */
 #define CO3_KERNEL_SCAN 3     /* chunk offsets, header, tables */
 #define CO3_KERNEL_COMPACT 4  /* payload compaction */
-#define CO3_KERNEL_CHECK 5    /* unused (stream validation is part of CO3_KERNEL_PREPARE) */
+#define CO3_KERNEL_CODE_BUILD 5 /* Huffman tables from weights on the device */
 #define CO3_KERNEL_DECODE 6   /* decode + cross-client accumulate */
 #define CO3_KERNEL_COUNT 7
 int co3_profile_enable(int on);

@@ -45,13 +45,14 @@ def _load():
     L.co3_convert.argtypes = [vp, vp, f32, vp, vp, u32, u64, u32, u64, vp, vp, vp, vp, sz, vp]
     L.co3_convert_static.argtypes = [vp, vp, f32, vp, vp, u32, u64, u32, u64, vp, vp, vp, vp]
     L.co3_code_build.argtypes = [vp, vp, vp]
+    L.co3_code_build_device.argtypes = [vp, vp, u32, vp, vp, vp]
     L.co3_encode.argtypes = [vp, vp, f32, vp, vp, vp, u32, u64, u32, u64, vp, sz, u32, vp, sz, vp, vp]
     L.co3_encode_symbols.argtypes = [vp, vp, vp, u32, u64, u32, u64, vp, sz, u32, vp, sz, vp, vp]
     L.co3_decode_aggregate.argtypes = [vp, sz, u32, vp, vp, vp, u32, u64, u32, vp, vp, sz, vp, vp]
     L.co3_decode.argtypes = [vp, sz, vp, vp, vp, u32, u64, u32, vp, vp, vp, sz, vp, vp]
     L.co3_profile_enable.argtypes = [C.c_int]
     L.co3_profile_read.argtypes = [vp, vp]
-    for name in ("co3_profile_enable", "co3_profile_read", "co3_convert_static", "co3_workspace_bytes", "co3_stream_capacity_bytes", "co3_convert", "co3_code_build", "co3_encode",
+    for name in ("co3_profile_enable", "co3_profile_read", "co3_convert_static", "co3_workspace_bytes", "co3_stream_capacity_bytes", "co3_convert", "co3_code_build", "co3_code_build_device", "co3_encode",
                  "co3_encode_symbols", "co3_decode_aggregate", "co3_decode"):
         getattr(L, name).restype = C.c_int
     _lib = L
@@ -139,6 +140,11 @@ def co3_code_build(weights: np.ndarray, fmt: np.ndarray) -> tuple[int, np.ndarra
     return st, out
 
 
+def co3_code_build_device(weights, fmts, n_seg, codes_out, res, stream=None) -> int:
+    """Device call: weights uint64/int64[n_seg * 256], fmts and codes_out as uploaded descriptor arrays."""
+    return _load().co3_code_build_device(_dev(weights), _dev(fmts), n_seg, _dev(codes_out), _dev(res), _stream(stream))
+
+
 def co3_convert(grad, mem, decay, fmts, segs, n_seg, n_elem, n_clients, client_stride_elems, sym_out, hist_out,
                 res, workspace, stream=None) -> int:
     return _load().co3_convert(_dev(grad), _dev(mem), float(decay), _dev(fmts), _dev(segs), n_seg, n_elem,
@@ -191,7 +197,7 @@ def co3_decode(stream_in, stream_bytes, fmts, codes, segs, n_seg, n_elem, ghat_o
                               workspace.numel() * workspace.element_size(), _dev(res), _stream(stream))
 
 
-KERNEL_NAMES = ("prepare", "convert", "pack", "scan", "compact", "check", "decode")
+KERNEL_NAMES = ("prepare", "convert", "pack", "scan", "compact", "code_build", "decode")
 
 
 def co3_profile_enable(on: bool) -> int:

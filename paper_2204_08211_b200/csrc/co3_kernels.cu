@@ -1420,6 +1420,198 @@ __global__ void __launch_bounds__(kThreads) decode_kernel(DecArgs a) {
     }
 }
 
+// ------------------------------------------------------------------------------------------------
+// code build: Huffman code of one segment from its 256 weights (Sec. IV-A (ii)), one block per segment,
+// thread = symbol.  Same construction and tie order as the host function co3_code_build: leaves ordered
+// by (weight, symbol), merged nodes by age, a leaf before a merged node of equal weight; weights are halved
+// and the construction repeated while the longest codeword exceeds CO3_MAX_CODE_LEN; canonical codewords.
+// ------------------------------------------------------------------------------------------------
+struct CodeBuildArgs {
+    const uint64_t* weights;  // [n_seg][256]
+    const co3_fmt* fmts;
+    co3_code* out;
+    co3_result* res;
+};
+
+// Same rule as the prepare kernel applies to symbols: the exponent code is not all ones, no "minus zero",
+// and with flushed sub-normals exponent code 0 carries mantissa code 0.
+__device__ __forceinline__ bool symbol_has_level(const co3_fmt& f, uint32_t sym) {
+    const uint32_t nb = (uint32_t)f.exp_bits + f.mant_bits;
+    if (sym >= (2u << nb)) return false;
+    const uint32_t sign = sym >> nb, mag = sym & ((1u << nb) - 1u);
+    const uint32_t efield = mag >> f.mant_bits, mfield = mag & ((1u << f.mant_bits) - 1u);
+    if (efield == (1u << f.exp_bits) - 1u) return false;
+    if (mag == 0) return sign == 0;
+    if (efield == 0 && (f.flags & CO3_FMT_FLUSH_SUBNORMALS) && mfield != 0) return false;
+    return true;
+}
+
+// Number of lanes, counted from lane 0, for which `ok` holds without a gap.
+__device__ __forceinline__ uint32_t leading_lanes(bool ok) {
+    const uint32_t bal = __ballot_sync(0xffffffffu, ok);
+    return bal == 0xffffffffu ? 32u : (uint32_t)__ffs((int)~bal) - 1u;
+}
+
+// The two-queue merge of one tree, run by one warp.  node[0..n) holds the leaf weights in order; merged nodes
+// are appended behind them; parent[] receives every node's parent.  Each step of the sequential method takes
+// the two smallest of the queue heads, a leaf winning ties.  The warp takes whole runs of steps at once:
+//   * while the second waiting leaf is not heavier than the merged queue's head, both picks are leaves, and
+//     none of the nodes created meanwhile is consumed: up to 32 leaf pairs are merged side by side;
+//   * while the second waiting merged node is lighter than the leaf head, both picks are merged nodes: up to 32
+//     pairs of nodes that already exist are merged side by side;
+//   * otherwise the step takes one of each.
+// T is wide enough for the weight sum, and ~0 is larger than any sum.
+template <typename T>
+__device__ __forceinline__ void merge_queues(T* node, uint16_t* parent, uint32_t n) {
+    const T kNone = ~(T)0;
+    const uint32_t lane = threadIdx.x & 31u;
+    uint32_t qa = 0, qb = n, t = n;  // leaves qa..n-1 and merged nodes qb..t-1 are waiting (same in every lane)
+    while (t < 2 * n - 1) {
+        const T a0 = qa < n ? node[qa] : kNone, a1 = qa + 1 < n ? node[qa + 1] : kNone;
+        const T b0 = qb < t ? node[qb] : kNone, b1 = qb + 1 < t ? node[qb + 1] : kNone;
+        uint32_t m;
+        if (a1 != kNone && a1 <= b0) {
+            // leaf pairs; with an empty merged queue the first pair's node becomes the head the others face
+            const T head = b0 != kNone ? b0 : a0 + a1;
+            const uint32_t i0 = qa + 2 * lane;
+            m = leading_lanes(lane == 0 || (i0 + 1 < n && node[i0 + 1] <= head));
+            if (lane < m) {
+                node[t + lane] = node[i0] + node[i0 + 1];
+                parent[i0] = parent[i0 + 1] = (uint16_t)(t + lane);
+            }
+            qa += 2 * m;
+        } else if (b1 != kNone && b1 < a0) {
+            // pairs of merged nodes that exist already (the ones created here wait behind them)
+            const uint32_t i0 = qb + 2 * lane;
+            m = leading_lanes(lane == 0 || (i0 + 1 < t && node[i0 + 1] < a0));
+            if (lane < m) {
+                node[t + lane] = node[i0] + node[i0 + 1];
+                parent[i0] = parent[i0 + 1] = (uint16_t)(t + lane);
+            }
+            qb += 2 * m;
+        } else {
+            // one leaf and one merged node
+            m = 1;
+            if (lane == 0) {
+                node[t] = a0 + b0;
+                parent[qa] = parent[qb] = (uint16_t)t;
+            }
+            ++qa;
+            ++qb;
+        }
+        t += m;
+        __syncwarp();
+    }
+}
+
+// One candidate tree, built by one warp: the weights after `h` halvings, max(1, w >> h) (halving h times
+// with a floor of 1 gives exactly that).  Lanes rank their symbols among the leaves, the warp merges, the lanes
+// walk from their leaves to the root.  Returns the longest codeword; len_out[sym] receives the lengths.
+template <typename T>
+__device__ __forceinline__ uint32_t build_tree(const uint64_t* s_w, uint32_t h, uint32_t n, T* node, uint16_t* parent,
+                                               uint8_t* len_out) {
+    const uint32_t lane = threadIdx.x & 31u;
+    T w[8];
+    uint32_t rank[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const uint64_t x = s_w[lane + 32 * i];
+        w[i] = x ? (T)max(x >> h, (uint64_t)1) : (T)0;
+        rank[i] = 0;
+    }
+    for (uint32_t j = 0; j < 256; ++j) {
+        const uint64_t x = s_w[j];
+        if (x == 0) continue;  // takes no part (the same for every lane)
+        const T wj = (T)max(x >> h, (uint64_t)1);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) rank[i] += (wj < w[i] || (wj == w[i] && j < lane + 32 * i)) ? 1u : 0u;
+    }
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+        if (w[i]) node[rank[i]] = w[i];
+    __syncwarp();
+    merge_queues<T>(node, parent, n);
+    uint32_t longest = 0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        uint32_t len = 0;
+        if (w[i]) {
+            for (uint32_t v = rank[i]; v != 2 * n - 2; v = parent[v]) ++len;
+        }
+        len_out[lane + 32 * i] = (uint8_t)len;
+        longest = max(longest, len);
+    }
+    return __reduce_max_sync(0xffffffffu, longest);
+}
+
+constexpr int kCandidates = kThreads / 32;  // trees built side by side, one per warp
+
+__global__ void __launch_bounds__(kThreads) code_build_kernel(CodeBuildArgs a) {
+    __shared__ uint64_t s_w[256];                    // weight of every symbol, 0 = takes no part
+    __shared__ uint64_t s_node[kCandidates][512];    // per candidate: the n leaves in order, then the merged nodes by age
+    __shared__ uint16_t s_parent[kCandidates][512];
+    __shared__ uint8_t s_len[kCandidates][256];
+    __shared__ uint32_t s_longest[kCandidates];
+    __shared__ uint64_t s_red[8];
+    const uint32_t k = blockIdx.x, sym = threadIdx.x, warp = sym >> 5;
+    if (k == 0 && sym == 0) a.res->first_bad_chunk = 0xffffffffu;
+    const co3_fmt f = a.fmts[k];
+    bool fmt_ok = f.exp_bits >= 2 && 1u + f.exp_bits + f.mant_bits <= 8u && !(f.flags & ~CO3_FMT_FLUSH_SUBNORMALS);
+    fmt_ok = fmt_ok && f.scale > 0.0f && f.inv_scale > 0.0f && !isinf(f.scale) && !isinf(f.inv_scale);
+    const bool valid = fmt_ok && symbol_has_level(f, sym);
+    uint64_t w = 0;
+    if (valid) {
+        w = a.weights[(size_t)k * 256 + sym];
+        if (w == 0) w = 1;
+    }
+    // the weights must add up to less than 2^63: sum their halves separately, neither sum can wrap
+    const uint64_t hi = block_sum_u64(w >> 32, s_red), lo = block_sum_u64(w & 0xffffffffull, s_red);
+    const bool sum_ok = hi + (lo >> 32) < (1ull << 31);
+    const uint32_t n = __syncthreads_count(valid);
+    a.out[k].len[sym] = 0;
+    a.out[k].bits[sym] = 0;
+    if (!fmt_ok || !sum_ok || n < 2) {
+        if (sym == 0) set_status(a.res, CO3_ERR_INVALID_ARG);
+        return;
+    }
+    const bool narrow = hi == 0 && lo < 0xffffffffull;  // every weight sum fits 32 bits
+    s_w[sym] = w;
+    __syncthreads();
+    // The code wanted is the one after the fewest halvings whose longest codeword fits.  Each warp tries one
+    // number of halvings; eight at a time, until one fits (63 halvings leave all weights at 1).
+    uint32_t len = 0;
+    for (uint32_t h0 = 0;; h0 += kCandidates) {
+        const uint32_t h = min(h0 + warp, 63u);
+        uint32_t longest;
+        if (narrow) longest = build_tree<uint32_t>(s_w, h, n, reinterpret_cast<uint32_t*>(s_node[warp]), s_parent[warp], s_len[warp]);
+        else longest = build_tree<uint64_t>(s_w, h, n, s_node[warp], s_parent[warp], s_len[warp]);
+        if ((sym & 31u) == 0) s_longest[warp] = longest;
+        __syncthreads();
+        uint32_t pick = kCandidates;
+        for (int c = kCandidates - 1; c >= 0; --c)
+            if (s_longest[c] <= (uint32_t)CO3_MAX_CODE_LEN) pick = (uint32_t)c;
+        if (pick < (uint32_t)kCandidates) {
+            len = s_len[pick][sym];
+            break;
+        }
+        __syncthreads();  // everyone has read the candidates before they are rebuilt
+    }
+    // canonical codewords: in (length, symbol) order the codeword of a symbol is the sum of 2^(16 - length)
+    // over the symbols before it, cut to its own length
+    __syncthreads();
+    s_len[0][sym] = (uint8_t)len;
+    __syncthreads();
+    if (valid) {
+        uint32_t before = 0;
+        for (uint32_t j = 0; j < 256; ++j) {
+            const uint32_t lj = s_len[0][j];
+            if (lj != 0 && (lj < len || (lj == len && j < sym))) before += 1u << (CO3_MAX_CODE_LEN - lj);
+        }
+        a.out[k].len[sym] = (uint8_t)len;
+        a.out[k].bits[sym] = (uint16_t)(before >> (CO3_MAX_CODE_LEN - len));
+    }
+}
+
 }  // namespace co3
 
 // ================================================================================================
@@ -1772,6 +1964,17 @@ int static_scratch_address(void** out) {
     return CO3_OK;
 }
 }  // namespace
+
+int co3_code_build_device(const uint64_t* weights, const co3_fmt* fmts, uint32_t n_seg, co3_code* codes_out,
+                          co3_result* res, void* stream) {
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (!weights || !fmts || !codes_out || !res || n_seg == 0 || n_seg > (1u << 20)) return CO3_ERR_INVALID_ARG;
+    if (!aligned(weights, 8) || !aligned(fmts, 4) || !aligned(codes_out, 2) || !aligned(res, 8)) return CO3_ERR_INVALID_ARG;
+    CO3_CUDA(cudaMemsetAsync(res, 0, sizeof(co3_result), st));
+    CodeBuildArgs ca{weights, fmts, codes_out, res};
+    CO3_LAUNCH(CO3_KERNEL_CODE_BUILD, st, code_build_kernel<<<n_seg, kThreads, 0, st>>>(ca));
+    return CO3_OK;
+}
 
 int co3_convert_static(const float* grad, float* mem, float decay, const co3_fmt* fmts, const co3_seg* segs,
                        uint32_t n_seg, uint64_t n_elem, uint32_t n_clients, uint64_t client_stride_elems,

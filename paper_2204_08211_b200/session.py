@@ -34,6 +34,7 @@ class Co3Session:
                                         dtype=torch.int64, device=self.device)
         self.res_enc = torch.zeros(self.n_clients * B.RESULT_DTYPE.itemsize, dtype=torch.uint8, device=self.device)
         self.res_dec = torch.zeros(B.RESULT_DTYPE.itemsize, dtype=torch.uint8, device=self.device)
+        self.res_fit = torch.zeros(B.RESULT_DTYPE.itemsize, dtype=torch.uint8, device=self.device)
         self.avg = torch.empty(self.n_elem, dtype=torch.float32, device=self.device)
         self.hist = torch.zeros(max(1, self.n_seg) * 256, dtype=torch.int64, device=self.device)
 
@@ -46,12 +47,15 @@ class Co3Session:
         return buf[u * self.stride:u * self.stride + self.n_elem]
 
     # -- code fitting -------------------------------------------------------------------------
-    def histogram(self, grads: torch.Tensor, mems: torch.Tensor, stream=None, sym_out=None) -> np.ndarray:
+    def histogram(self, grads: torch.Tensor, mems: torch.Tensor, stream=None, sym_out=None, to_host: bool = True):
         """Symbol counts per layer summed over clients for this round; `mems` is updated like a real round
-        and, if `sym_out` is given, the symbols are kept for co3_encode_symbols."""
+        and, if `sym_out` is given, the symbols are kept for co3_encode_symbols.  The counts stay in
+        self.hist on the device; to_host=False skips the copy to the host (and its synchronisation)."""
         st = B.co3_convert(grads, mems, self.decay, self.fmts, self.segs, self.n_seg, self.n_elem, self.n_clients,
                            self.stride, sym_out, self.hist, self.res_enc, self.workspace, stream)
         self._check(st, "co3_convert")
+        if not to_host:
+            return None
         return self.hist.cpu().numpy().astype(np.uint64).reshape(-1, 256)[:self.n_seg]
 
     def set_codes_from_weights(self, weights: np.ndarray) -> None:
@@ -62,6 +66,15 @@ class Co3Session:
             self._check(st, "co3_code_build")
             codes[k] = c[0]
         self.set_codes(codes)
+
+    def set_codes_from_histogram_device(self, stream=None) -> None:
+        """One Huffman code per layer from the histogram the last histogram() call left on the device; the
+        tables are built there too (the host copy of the codes is dropped)."""
+        if self.codes is None:
+            self.codes = torch.zeros(max(1, self.n_seg) * B.CODE_DTYPE.itemsize, dtype=torch.uint8, device=self.device)
+        self.codes_host = None
+        st = B.co3_code_build_device(self.hist, self.fmts, self.n_seg, self.codes, self.res_fit, stream)
+        self._check(st, "co3_code_build_device")
 
     def set_codes(self, codes: np.ndarray) -> None:
         self.codes_host = codes
@@ -89,6 +102,9 @@ class Co3Session:
     # -- results --------------------------------------------------------------------------------
     def encode_results(self) -> np.ndarray:
         return B.read_results(self.res_enc, self.n_clients)
+
+    def fit_result(self) -> np.ndarray:
+        return B.read_results(self.res_fit, 1)
 
     def decode_result(self) -> np.ndarray:
         return B.read_results(self.res_dec, 1)
