@@ -1084,7 +1084,8 @@ struct DecSmem {
     uint16_t lut[kDecLut];
     float val[256];
     uint64_t bar;                          // completion barrier of the bulk copies of one batch
-    uint64_t pad;
+    uint32_t tile_elems;                   // elements of the tile: full chunks and the last one's count
+    uint32_t pad;
     uint64_t chunk_elem0[kMaxPairs];       // first element of each chunk of the tile
     const uint32_t* pair_src[kMaxPairs];   // the pair's first payload word in global memory
     uint32_t pair_off[kMaxPairs];          // staged pairs: index of that word in pay[]
@@ -1184,14 +1185,6 @@ __device__ __forceinline__ void decode_part(const uint32_t* words, uint32_t nwor
     }
 }
 
-// How the block's averages are formed: acc / U, or acc * (1 / U) when U is a power of two (the product with
-// the exact reciprocal rounds the same real number as the division).
-struct Averager {
-    float u, inv;
-    bool pow2;
-    __device__ __forceinline__ float operator()(float acc) const { return pow2 ? __fmul_rn(acc, inv) : __fdiv_rn(acc, u); }
-};
-
 // Adds, in client order, the values of the four symbols of word (s, j) of chunk cl of the tile's current phase
 // for the nb clients of the batch.  Returns the last client's symbol word.
 __device__ __forceinline__ uint32_t sum_word(const float* __restrict__ val, const uint32_t* __restrict__ sym, uint32_t cl,
@@ -1209,25 +1202,41 @@ __device__ __forceinline__ uint32_t sum_word(const float* __restrict__ val, cons
     return symw;
 }
 
-// Averages the sums and stores the (up to four) elements that start at element i0 of chunk cl of the tile.
-__device__ __forceinline__ void write_word(const DecArgs& a, const DecSmem& sm, const TileDesc& td, uint32_t cl, uint32_t i0,
-                                           uint32_t B, const Averager& avg, const float (&acc)[4], uint32_t symw) {
-    if (cl >= td.n_chunks) return;
-    const uint32_t cnt = sm.pair_cnt[cl * B];
-    if (i0 >= cnt) return;
-    const uint32_t nv = min(4u, cnt - i0);
-    const uint64_t e = sm.chunk_elem0[cl] + i0;
-    if (a.out) {
-        float* o = a.out + e;
-        if (nv == 4 && (reinterpret_cast<uintptr_t>(o) & 15u) == 0) {
-            *reinterpret_cast<float4*>(o) = make_float4(avg(acc[0]), avg(acc[1]), avg(acc[2]), avg(acc[3]));
+// Where a tile's results go.  The chunks of a tile follow one another in one segment and all but the last
+// are full, so element e of the tile (chunk index * kC + place in the chunk) is element e behind the tile's
+// first one in the output as well.
+struct TileOut {
+    float* out;         // the tile's first element in the output vector (null: no values wanted)
+    uint8_t* sym;       // the same in the symbol output (nullable)
+    uint32_t n_elem;    // elements of the tile
+    bool out16, sym4;   // out is 16-byte aligned / sym is 4-byte aligned
+    float u, inv;       // the averages are acc / u, or acc * inv when u is a power of two (the product with
+    bool pow2;          // the exact reciprocal rounds the same real number as the division)
+};
+
+// Averages the sums and stores the (up to four) elements that start at element e of the tile; e is a multiple
+// of four below to.n_elem.
+__device__ __forceinline__ void write_word(const TileOut& to, uint32_t e, const float (&acc)[4], uint32_t symw) {
+    const uint32_t nv = min(4u, to.n_elem - e);
+    if (to.out) {
+        float r[4];
+        if (to.pow2) {
+#pragma unroll
+            for (int q = 0; q < 4; ++q) r[q] = __fmul_rn(acc[q], to.inv);
         } else {
-            for (uint32_t q = 0; q < nv; ++q) o[q] = avg(acc[q]);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) r[q] = __fdiv_rn(acc[q], to.u);
+        }
+        float* o = to.out + e;
+        if (nv == 4 && to.out16) {
+            *reinterpret_cast<float4*>(o) = make_float4(r[0], r[1], r[2], r[3]);
+        } else {
+            for (uint32_t q = 0; q < nv; ++q) o[q] = r[q];
         }
     }
-    if (a.sym_out) {
-        uint8_t* o = a.sym_out + e;
-        if (nv == 4 && (reinterpret_cast<uintptr_t>(o) & 3u) == 0) {
+    if (to.sym) {
+        uint8_t* o = to.sym + e;
+        if (nv == 4 && to.sym4) {
             *reinterpret_cast<uint32_t*>(o) = symw;
         } else {
             for (uint32_t q = 0; q < nv; ++q) o[q] = (uint8_t)(symw >> (8 * q));
@@ -1241,7 +1250,7 @@ __device__ __forceinline__ void write_word(const DecArgs& a, const DecSmem& sm, 
 // its share of the tile over the clients in client order.  kMulti: more clients than fit side by side
 // (B = 16, G = 1): the partial sums stay in registers between batches.
 template <bool kMulti>
-__global__ void __launch_bounds__(kThreads) decode_kernel(DecArgs a) {
+__global__ void __launch_bounds__(kThreads, 4) decode_kernel(DecArgs a) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     DecSmem& sm = *reinterpret_cast<DecSmem*>(smem_raw);
     const uint32_t B = kMulti ? 16u : a.B, G = kMulti ? 1u : a.G;
@@ -1261,10 +1270,10 @@ __global__ void __launch_bounds__(kThreads) decode_kernel(DecArgs a) {
 
     if (tid == 0) mbar_init(&sm.bar, 1);
     float carry[kPhases][4];  // running sums across client batches (kMulti only)
-    Averager avg;
-    avg.u = (float)a.n_clients;
-    avg.pow2 = (a.n_clients & (a.n_clients - 1u)) == 0;
-    avg.inv = __fdiv_rn(1.0f, avg.u);
+    TileOut to;
+    to.u = (float)a.n_clients;
+    to.pow2 = (a.n_clients & (a.n_clients - 1u)) == 0;
+    to.inv = __fdiv_rn(1.0f, to.u);
     bool err = false, hw_fail = false;
     uint32_t phase = 0;
 
@@ -1287,6 +1296,7 @@ __global__ void __launch_bounds__(kThreads) decode_kernel(DecArgs a) {
                     const ChunkDesc cd = a.ws.chunk_desc[chunk];
                     cnt = cd.cnt;
                     if (ul == 0) sm.chunk_elem0[cl] = cd.elem0;
+                    if (ul == 0 && cl + 1 == td.n_chunks) sm.tile_elems = cl * kC + cd.cnt;
                     sub_src = reinterpret_cast<const uint16_t*>(stream + ctrl->sub_off) + (uint64_t)chunk * kSubs;
                     if (w0 > w1 || w1 > cap_words || w1 - w0 > (uint64_t)kSlotWords) {
                         err = true;
@@ -1354,6 +1364,12 @@ __global__ void __launch_bounds__(kThreads) decode_kernel(DecArgs a) {
         }
         const bool had_symbols = my != 0;
         const bool first_batch = (u0 == 0), last_batch = (u0 + B >= a.n_clients);
+        const uint32_t tile_words = min(G, td.n_chunks) * kPairPhaseWords;
+        to.n_elem = sm.tile_elems;
+        to.out = a.out ? a.out + sm.chunk_elem0[0] : nullptr;
+        to.sym = a.sym_out ? a.sym_out + sm.chunk_elem0[0] : nullptr;
+        to.out16 = (reinterpret_cast<uintptr_t>(to.out) & 15u) == 0;
+        to.sym4 = (reinterpret_cast<uintptr_t>(to.sym) & 3u) == 0;
 #pragma unroll(kMulti ? kPhases : 1)
         for (int ph = 0; ph < kPhases; ++ph) {
             // ---- decode this phase's 32 symbols of the sub-chunk
@@ -1366,10 +1382,13 @@ __global__ void __launch_bounds__(kThreads) decode_kernel(DecArgs a) {
                 for (uint32_t jj = 0; jj < (uint32_t)kPhaseWords; ++jj) pair_buf[sym_slot(p, sc, jj)] = 0;
             }
             __syncthreads();
-            // ---- ordered sum over the clients of this batch; a thread owns whole symbol words
+            // ---- ordered sum over the clients of this batch; a thread owns whole symbol words: word w of the
+            //      tile's phase is word (s, j) of chunk cl and starts at element e of the tile
+            static_assert(kPairPhaseWords == 128 && kPhaseWords == 8 && kC == 2048 && kS == 128, "shifts below");
             if (kMulti) {
                 if (tid < (uint32_t)kPairPhaseWords) {
-                    const uint32_t s = tid / kPhaseWords, j = tid % kPhaseWords;
+                    const uint32_t s = tid >> 3, j = tid & 7u;
+                    const uint32_t e = (s << 7) + ph * kPhaseSyms + (j << 2);
                     float acc[4];
 #pragma unroll
                     for (int q = 0; q < 4; ++q) acc[q] = first_batch ? 0.0f : carry[ph][q];
@@ -1377,27 +1396,18 @@ __global__ void __launch_bounds__(kThreads) decode_kernel(DecArgs a) {
                     if (!last_batch) {
 #pragma unroll
                         for (int q = 0; q < 4; ++q) carry[ph][q] = acc[q];
-                    } else {
-                        write_word(a, sm, td, 0, s * kS + ph * kPhaseSyms + j * 4, B, avg, acc, symw);
+                    } else if (e < to.n_elem) {
+                        write_word(to, e, acc, symw);
                     }
                 }
-            } else if ((n_thr % kPairPhaseWords) == 0) {
-                // the thread keeps its place inside the chunk and steps over the tile's chunks
-                const uint32_t wi = tid % kPairPhaseWords, s = wi / kPhaseWords, j = wi % kPhaseWords;
-                const uint32_t i0 = s * kS + ph * kPhaseSyms + j * 4;
-                for (uint32_t cl = tid / kPairPhaseWords; cl < G; cl += n_thr / kPairPhaseWords) {
-                    float acc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-                    const uint32_t symw = sum_word(sm.val, sm_sym, cl, s, j, B, nb, acc);
-                    write_word(a, sm, td, cl, i0, B, avg, acc, symw);
-                }
             } else {
-                const uint32_t tile_words = G * kPairPhaseWords;
                 for (uint32_t w = tid; w < tile_words; w += n_thr) {
-                    const uint32_t cl = w / kPairPhaseWords, wi = w % kPairPhaseWords;
-                    const uint32_t s = wi / kPhaseWords, j = wi % kPhaseWords;
+                    const uint32_t cl = w >> 7, s = (w >> 3) & 15u, j = w & 7u;
+                    const uint32_t e = (cl << 11) + (s << 7) + ph * kPhaseSyms + (j << 2);
+                    if (e >= to.n_elem) continue;
                     float acc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
                     const uint32_t symw = sum_word(sm.val, sm_sym, cl, s, j, B, nb, acc);
-                    write_word(a, sm, td, cl, s * kS + ph * kPhaseSyms + j * 4, B, avg, acc, symw);
+                    write_word(to, e, acc, symw);
                 }
             }
             __syncthreads();  // the phase buffer is free again
