@@ -1215,12 +1215,16 @@ struct TileOut {
 };
 
 // Averages the sums and stores the (up to four) elements that start at element e of the tile; e is a multiple
-// of four below to.n_elem.
+// of four below to.n_elem.  kPlain: acc holds values, not sums to be averaged.
+template <bool kPlain>
 __device__ __forceinline__ void write_word(const TileOut& to, uint32_t e, const float (&acc)[4], uint32_t symw) {
     const uint32_t nv = min(4u, to.n_elem - e);
     if (to.out) {
         float r[4];
-        if (to.pow2) {
+        if (kPlain) {  // one client: the average is the value itself
+#pragma unroll
+            for (int q = 0; q < 4; ++q) r[q] = acc[q];
+        } else if (to.pow2) {
 #pragma unroll
             for (int q = 0; q < 4; ++q) r[q] = __fmul_rn(acc[q], to.inv);
         } else {
@@ -1248,12 +1252,12 @@ __device__ __forceinline__ void write_word(const TileOut& to, uint32_t e, const 
 // pair's payload lies and starts one bulk copy per pair into shared memory (plus the segment's tables);
 // then 16 threads per pair (one per sub-chunk) decode into a symbol buffer, and finally every thread sums
 // its share of the tile over the clients in client order.  kMulti: more clients than fit side by side
-// (B = 16, G = 1): the partial sums stay in registers between batches.
-template <bool kMulti>
+// (B = 16, G = 1): the partial sums stay in registers between batches.  kSingle: one client, nothing to sum.
+template <bool kMulti, bool kSingle>
 __global__ void __launch_bounds__(kThreads, 4) decode_kernel(DecArgs a) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     DecSmem& sm = *reinterpret_cast<DecSmem*>(smem_raw);
-    const uint32_t B = kMulti ? 16u : a.B, G = kMulti ? 1u : a.G;
+    const uint32_t B = kMulti ? 16u : (kSingle ? 1u : a.B), G = kMulti ? 1u : a.G;
     const uint32_t n_pairs = B * G, n_thr = 16u * n_pairs;
     uint32_t* const sm_sym = reinterpret_cast<uint32_t*>(smem_raw + sizeof(DecSmem));
     uint32_t* const sm_pay = sm_sym + n_pairs * kPairPhaseWords;
@@ -1397,7 +1401,7 @@ __global__ void __launch_bounds__(kThreads, 4) decode_kernel(DecArgs a) {
 #pragma unroll
                         for (int q = 0; q < 4; ++q) carry[ph][q] = acc[q];
                     } else if (e < to.n_elem) {
-                        write_word(to, e, acc, symw);
+                        write_word<false>(to, e, acc, symw);
                     }
                 }
             } else {
@@ -1405,9 +1409,17 @@ __global__ void __launch_bounds__(kThreads, 4) decode_kernel(DecArgs a) {
                     const uint32_t cl = w >> 7, s = (w >> 3) & 15u, j = w & 7u;
                     const uint32_t e = (cl << 11) + (s << 7) + ph * kPhaseSyms + (j << 2);
                     if (e >= to.n_elem) continue;
-                    float acc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-                    const uint32_t symw = sum_word(sm.val, sm_sym, cl, s, j, B, nb, acc);
-                    write_word(to, e, acc, symw);
+                    if (kSingle) {
+                        const uint32_t symw = sm_sym[cl * kPairPhaseWords + sym_slot(cl, s, j)];
+                        float v[4];
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) v[q] = sm.val[(symw >> (8 * q)) & 0xffu];
+                        write_word<true>(to, e, v, symw);
+                    } else {
+                        float acc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+                        const uint32_t symw = sum_word(sm.val, sm_sym, cl, s, j, B, nb, acc);
+                        write_word<false>(to, e, acc, symw);
+                    }
                 }
             }
             __syncthreads();  // the phase buffer is free again
@@ -1799,11 +1811,14 @@ int decode_common(const uint8_t* const* streams, const uint8_t* single, size_t s
     const uint32_t n_pairs = B * G;
     const size_t smem = sizeof(DecSmem) + 4 * ((size_t)n_pairs * (kPairPhaseWords + kPaySlotWords) + kPaySlack);
     if (multi) {
-        CO3_CUDA(cudaFuncSetAttribute(decode_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        CO3_LAUNCH(CO3_KERNEL_DECODE, st, decode_kernel<true><<<tiles, kThreads, smem, st>>>(da));
+        CO3_CUDA(cudaFuncSetAttribute(decode_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        CO3_LAUNCH(CO3_KERNEL_DECODE, st, decode_kernel<true, false><<<tiles, kThreads, smem, st>>>(da));
+    } else if (n_clients == 1) {
+        CO3_CUDA(cudaFuncSetAttribute(decode_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        CO3_LAUNCH(CO3_KERNEL_DECODE, st, decode_kernel<false, true><<<tiles, 16 * n_pairs, smem, st>>>(da));
     } else {
-        CO3_CUDA(cudaFuncSetAttribute(decode_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        CO3_LAUNCH(CO3_KERNEL_DECODE, st, decode_kernel<false><<<tiles, 16 * n_pairs, smem, st>>>(da));
+        CO3_CUDA(cudaFuncSetAttribute(decode_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        CO3_LAUNCH(CO3_KERNEL_DECODE, st, decode_kernel<false, false><<<tiles, 16 * n_pairs, smem, st>>>(da));
     }
     return CO3_OK;
 }
