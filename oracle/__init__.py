@@ -84,6 +84,8 @@ def lib():
         L.co3o_decode_aggregate.argtypes = [C.c_void_p, C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p,
                                             C.c_void_p, C.c_uint32, C.c_uint32, C.c_uint32, C.c_void_p,
                                             C.c_void_p]
+        L.co3o_ps_update.restype = None
+        L.co3o_ps_update.argtypes = [C.c_void_p, C.c_void_p, C.c_float, C.c_uint64]
         _lib = L
     return _lib
 
@@ -237,3 +239,10 @@ def decode_aggregate(streams, seg_n_elem, fmts, codes, chunk_syms: int = 2048, s
     st = lib().co3o_decode_aggregate(ptrs, _ptr(sizes), len(streams), _ptr(seg), farr, carr, seg.size,
                                      chunk_syms, sub_syms, _ptr(avg), _ptr(scratch))
     return st, avg
+
+
+def ps_update(w: np.ndarray, avg: np.ndarray, eta: float) -> None:
+    """w <- w - eta * avg in place (float32 arrays of equal size)."""
+    assert w.dtype == np.float32 and avg.dtype == np.float32 and w.flags.c_contiguous and avg.flags.c_contiguous
+    assert w.size == avg.size
+    lib().co3o_ps_update(_ptr(w), _ptr(avg), C.c_float(eta), w.size)

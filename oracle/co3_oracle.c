@@ -578,3 +578,16 @@ int co3o_decode_aggregate(const uint8_t *const *streams, const uint64_t *stream_
     for (uint64_t i = 0; i < n; ++i) avg[i] = avg[i] / U;
     return CO3O_OK;
 }
+
+/*
+ * Model update at the parameter server (Algorithm 1, last step; Sec. II-B (iv)):
+ * w <- w - eta * avg with avg = (1/U) * sum_u ghat^(u) as co3o_decode_aggregate forms it.
+ * Per element one fp32 multiplication and one fp32 subtraction, each rounded on its own.
+ */
+void co3o_ps_update(float *w, const float *avg, float eta, uint64_t n)
+{
+    for (uint64_t i = 0; i < n; ++i) {
+        const float step = eta * avg[i];
+        w[i] = w[i] - step;
+    }
+}

@@ -1150,9 +1150,11 @@ __device__ __forceinline__ void decode_two(const uint32_t* words, uint32_t nword
         return;
     }
     uint32_t l0 = e0 >> 8;
-    uint32_t win1 = win << (l0 & 31u);  // a marker's "length" is meaningless: keep the shift defined
+    uint32_t win1 = __funnelshift_l(0u, win, l0);  // win << (l0 mod 32): a marker's "length" is meaningless
     e1 = s_lut[win1 >> (32 - kDecBits)];
-    if ((e0 | e1) >= kDecLong) {
+    uint32_t either = e0 | e1;
+    asm("" : "+r"(either));  // one test, one branch for both entries
+    if (either >= kDecLong) {
         if (e0 >= kDecLong) e0 = decode_long(sub_tab, e0, win);
         l0 = e0 >> 8;
         win1 = win << l0;
