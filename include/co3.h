@@ -219,6 +219,19 @@ int co3_decode_aggregate(const uint8_t* const* streams, size_t stream_bytes, uin
                          uint32_t n_seg, uint64_t n_elem, uint32_t chunk_syms, float* avg_out,
                          void* workspace, size_t workspace_bytes, co3_result* res, void* stream);
 
+/*
+ * The same with the model update of Algorithm 1's last step folded in (w_{t+1} = w_t - eta/U * sum_u ghat^(u),
+ * Sec. II-B (iv)): params[i] <- params[i] - lr * avg[i] with avg[i] exactly as co3_decode_aggregate forms
+ * it; one fp32 multiplication and one fp32 subtraction per element, each rounded on its own.
+ *   params [device]   n_elem model parameters, updated in place; 16-byte aligned
+ *   avg_out [device]  nullable: the average itself, if the caller wants it too
+ */
+int co3_decode_aggregate_update(const uint8_t* const* streams, size_t stream_bytes, uint32_t n_clients,
+                                const co3_fmt* fmts, const co3_code* codes, const co3_seg* segs,
+                                uint32_t n_seg, uint64_t n_elem, uint32_t chunk_syms, float lr, float* params,
+                                float* avg_out, void* workspace, size_t workspace_bytes, co3_result* res,
+                                void* stream);
+
 /* One stream: reconstructed values and/or symbols (either output may be NULL, not both). */
 int co3_decode(const uint8_t* stream_in, size_t stream_bytes,
                const co3_fmt* fmts, const co3_code* codes, const co3_seg* segs,

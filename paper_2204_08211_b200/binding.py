@@ -49,11 +49,12 @@ def _load():
     L.co3_encode.argtypes = [vp, vp, f32, vp, vp, vp, u32, u64, u32, u64, vp, sz, u32, vp, sz, vp, vp]
     L.co3_encode_symbols.argtypes = [vp, vp, vp, u32, u64, u32, u64, vp, sz, u32, vp, sz, vp, vp]
     L.co3_decode_aggregate.argtypes = [vp, sz, u32, vp, vp, vp, u32, u64, u32, vp, vp, sz, vp, vp]
+    L.co3_decode_aggregate_update.argtypes = [vp, sz, u32, vp, vp, vp, u32, u64, u32, f32, vp, vp, vp, sz, vp, vp]
     L.co3_decode.argtypes = [vp, sz, vp, vp, vp, u32, u64, u32, vp, vp, vp, sz, vp, vp]
     L.co3_profile_enable.argtypes = [C.c_int]
     L.co3_profile_read.argtypes = [vp, vp]
     for name in ("co3_profile_enable", "co3_profile_read", "co3_convert_static", "co3_workspace_bytes", "co3_stream_capacity_bytes", "co3_convert", "co3_code_build", "co3_code_build_device", "co3_encode",
-                 "co3_encode_symbols", "co3_decode_aggregate", "co3_decode"):
+                 "co3_encode_symbols", "co3_decode_aggregate", "co3_decode_aggregate_update", "co3_decode"):
         getattr(L, name).restype = C.c_int
     _lib = L
     return L
@@ -188,6 +189,15 @@ def co3_decode_aggregate(stream_ptrs, stream_bytes, n_clients, fmts, codes, segs
     return _load().co3_decode_aggregate(_dev(stream_ptrs), stream_bytes, n_clients, _dev(fmts), _dev(codes),
                                         _dev(segs), n_seg, n_elem, chunk_syms, _dev(avg_out), _dev(workspace),
                                         workspace.numel() * workspace.element_size(), _dev(res), _stream(stream))
+
+
+def co3_decode_aggregate_update(stream_ptrs, stream_bytes, n_clients, fmts, codes, segs, n_seg, n_elem, lr, params,
+                                avg_out, workspace, res, chunk_syms: int = CHUNK_SYMS, stream=None) -> int:
+    """co3_decode_aggregate with params <- params - lr * avg folded in; avg_out may be None."""
+    return _load().co3_decode_aggregate_update(_dev(stream_ptrs), stream_bytes, n_clients, _dev(fmts), _dev(codes),
+                                               _dev(segs), n_seg, n_elem, chunk_syms, float(lr), _dev(params),
+                                               _dev(avg_out, True), _dev(workspace),
+                                               workspace.numel() * workspace.element_size(), _dev(res), _stream(stream))
 
 
 def co3_decode(stream_in, stream_bytes, fmts, codes, segs, n_seg, n_elem, ghat_out, sym_out, workspace, res,

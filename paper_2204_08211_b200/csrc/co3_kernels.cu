@@ -1064,6 +1064,8 @@ struct DecArgs {
     uint64_t n_elem;
     float* out;        // average (or the single client's values); nullable when sym_out is given
     uint8_t* sym_out;  // nullable; only with n_clients == 1
+    float* params;     // nullable: model parameters to update with the average (Algorithm 1, last step)
+    float lr;          // learning rate of that update
     co3_result* res;
     uint32_t B;        // clients decoded side by side in one block
     uint32_t G;        // chunks per block (tile)
@@ -1210,8 +1212,10 @@ __device__ __forceinline__ uint32_t sum_word(const float* __restrict__ val, cons
 struct TileOut {
     float* out;         // the tile's first element in the output vector (null: no values wanted)
     uint8_t* sym;       // the same in the symbol output (nullable)
+    float* params;      // the same in the model parameters to update (nullable)
+    float lr;
     uint32_t n_elem;    // elements of the tile
-    bool out16, sym4;   // out is 16-byte aligned / sym is 4-byte aligned
+    bool out16, sym4, params16;  // out / params are 16-byte aligned, sym is 4-byte aligned
     float u, inv;       // the averages are acc / u, or acc * inv when u is a power of two (the product with
     bool pow2;          // the exact reciprocal rounds the same real number as the division)
 };
@@ -1221,23 +1225,36 @@ struct TileOut {
 template <bool kPlain>
 __device__ __forceinline__ void write_word(const TileOut& to, uint32_t e, const float (&acc)[4], uint32_t symw) {
     const uint32_t nv = min(4u, to.n_elem - e);
+    float r[4];
+    if (kPlain) {  // one client: the average is the value itself
+#pragma unroll
+        for (int q = 0; q < 4; ++q) r[q] = acc[q];
+    } else if (to.pow2) {
+#pragma unroll
+        for (int q = 0; q < 4; ++q) r[q] = __fmul_rn(acc[q], to.inv);
+    } else {
+#pragma unroll
+        for (int q = 0; q < 4; ++q) r[q] = __fdiv_rn(acc[q], to.u);
+    }
     if (to.out) {
-        float r[4];
-        if (kPlain) {  // one client: the average is the value itself
-#pragma unroll
-            for (int q = 0; q < 4; ++q) r[q] = acc[q];
-        } else if (to.pow2) {
-#pragma unroll
-            for (int q = 0; q < 4; ++q) r[q] = __fmul_rn(acc[q], to.inv);
-        } else {
-#pragma unroll
-            for (int q = 0; q < 4; ++q) r[q] = __fdiv_rn(acc[q], to.u);
-        }
         float* o = to.out + e;
         if (nv == 4 && to.out16) {
             *reinterpret_cast<float4*>(o) = make_float4(r[0], r[1], r[2], r[3]);
         } else {
             for (uint32_t q = 0; q < nv; ++q) o[q] = r[q];
+        }
+    }
+    if (to.params) {  // w <- w - lr * avg: one multiplication and one subtraction, each rounded on its own
+        float* w = to.params + e;
+        if (nv == 4 && to.params16) {
+            float4 x = *reinterpret_cast<const float4*>(w);
+            x.x = __fsub_rn(x.x, __fmul_rn(to.lr, r[0]));
+            x.y = __fsub_rn(x.y, __fmul_rn(to.lr, r[1]));
+            x.z = __fsub_rn(x.z, __fmul_rn(to.lr, r[2]));
+            x.w = __fsub_rn(x.w, __fmul_rn(to.lr, r[3]));
+            *reinterpret_cast<float4*>(w) = x;
+        } else {
+            for (uint32_t q = 0; q < nv; ++q) w[q] = __fsub_rn(w[q], __fmul_rn(to.lr, r[q]));
         }
     }
     if (to.sym) {
@@ -1374,6 +1391,9 @@ __global__ void __launch_bounds__(kThreads, 4) decode_kernel(DecArgs a) {
         to.n_elem = sm.tile_elems;
         to.out = a.out ? a.out + sm.chunk_elem0[0] : nullptr;
         to.sym = a.sym_out ? a.sym_out + sm.chunk_elem0[0] : nullptr;
+        to.params = a.params ? a.params + sm.chunk_elem0[0] : nullptr;
+        to.lr = a.lr;
+        to.params16 = (reinterpret_cast<uintptr_t>(to.params) & 15u) == 0;
         to.out16 = (reinterpret_cast<uintptr_t>(to.out) & 15u) == 0;
         to.sym4 = (reinterpret_cast<uintptr_t>(to.sym) & 3u) == 0;
 #pragma unroll(kMulti ? kPhases : 1)
@@ -1784,11 +1804,12 @@ int begin_call(const WsLayout& L, const Ws& ws, co3_result* res, uint32_t n_res,
 
 int decode_common(const uint8_t* const* streams, const uint8_t* single, size_t stream_bytes, uint32_t n_clients,
                   const co3_fmt* fmts, const co3_code* codes, const co3_seg* segs, uint32_t n_seg, uint64_t n_elem,
-                  uint32_t chunk_syms, float* out, uint8_t* sym_out, void* workspace, size_t workspace_bytes,
-                  co3_result* res, cudaStream_t st) {
+                  uint32_t chunk_syms, float* out, uint8_t* sym_out, float* params, float lr, void* workspace,
+                  size_t workspace_bytes, co3_result* res, cudaStream_t st) {
     if ((!streams && !single) || !fmts || !codes || !res || !workspace || n_clients == 0 || chunk_syms != (uint32_t)kC)
         return CO3_ERR_INVALID_ARG;
-    if ((!segs && n_seg) || (!out && !sym_out) || (sym_out && n_clients != 1)) return CO3_ERR_INVALID_ARG;
+    if ((!segs && n_seg) || (!out && !sym_out && !params) || (sym_out && n_clients != 1)) return CO3_ERR_INVALID_ARG;
+    if (params && !aligned(params, 16)) return CO3_ERR_INVALID_ARG;
     if (!aligned(workspace, 256) || (out && !aligned(out, 16)) || !aligned(res, 8)) return CO3_ERR_INVALID_ARG;
     WsLayout L;
     if (!ws_layout(n_elem, n_seg, 0, &L)) return CO3_ERR_INVALID_ARG;
@@ -1807,7 +1828,7 @@ int decode_common(const uint8_t* const* streams, const uint8_t* single, size_t s
     }
     const int rc = begin_call(L, ws, res, 1, st, fmts, codes, segs, n_seg, n_elem, G, 1, streams, single, stream_bytes, n_clients);
     if (rc != CO3_OK) return rc;
-    DecArgs da{streams, single, stream_bytes, n_clients, segs, n_seg, n_elem, out, sym_out, res, B, G, ws};
+    DecArgs da{streams, single, stream_bytes, n_clients, segs, n_seg, n_elem, out, sym_out, params, lr, res, B, G, ws};
     const uint32_t tiles = (uint32_t)(L.n_chunks_max / G + n_seg);  // upper bound; surplus blocks return at once
     if (tiles == 0) return CO3_OK;
     const uint32_t n_pairs = B * G;
@@ -2043,15 +2064,25 @@ int co3_decode_aggregate(const uint8_t* const* streams, size_t stream_bytes, uin
     if (!avg_out) return CO3_ERR_INVALID_ARG;
     if (!streams) return CO3_ERR_INVALID_ARG;
     return decode_common(streams, nullptr, stream_bytes, n_clients, fmts, codes, segs, n_seg, n_elem, chunk_syms, avg_out,
-                         nullptr, workspace, workspace_bytes, res, static_cast<cudaStream_t>(stream));
+                         nullptr, nullptr, 0.0f, workspace, workspace_bytes, res, static_cast<cudaStream_t>(stream));
+}
+
+int co3_decode_aggregate_update(const uint8_t* const* streams, size_t stream_bytes, uint32_t n_clients, const co3_fmt* fmts,
+                                const co3_code* codes, const co3_seg* segs, uint32_t n_seg, uint64_t n_elem,
+                                uint32_t chunk_syms, float lr, float* params, float* avg_out, void* workspace,
+                                size_t workspace_bytes, co3_result* res, void* stream) {
+    if (!params || !streams) return CO3_ERR_INVALID_ARG;
+    return decode_common(streams, nullptr, stream_bytes, n_clients, fmts, codes, segs, n_seg, n_elem, chunk_syms, avg_out,
+                         nullptr, params, lr, workspace, workspace_bytes, res, static_cast<cudaStream_t>(stream));
 }
 
 int co3_decode(const uint8_t* stream_in, size_t stream_bytes, const co3_fmt* fmts, const co3_code* codes,
                const co3_seg* segs, uint32_t n_seg, uint64_t n_elem, uint32_t chunk_syms, float* ghat_out,
                uint8_t* sym_out, void* workspace, size_t workspace_bytes, co3_result* res, void* stream) {
     if (!stream_in || !aligned(stream_in, 16)) return CO3_ERR_INVALID_ARG;
+    if (!ghat_out && !sym_out) return CO3_ERR_INVALID_ARG;
     return decode_common(nullptr, stream_in, stream_bytes, 1, fmts, codes, segs, n_seg, n_elem, chunk_syms, ghat_out,
-                         sym_out, workspace, workspace_bytes, res, static_cast<cudaStream_t>(stream));
+                         sym_out, nullptr, 0.0f, workspace, workspace_bytes, res, static_cast<cudaStream_t>(stream));
 }
 
 }  // extern "C"

@@ -99,6 +99,14 @@ class Co3Session:
         self._check(st, "co3_decode_aggregate")
         return self.avg
 
+    def decode_aggregate_update(self, params: torch.Tensor, lr: float, want_avg: bool = False, stream=None):
+        """Decode, average and apply params <- params - lr * avg in the same kernel."""
+        st = B.co3_decode_aggregate_update(self.stream_ptrs, self.capacity, self.n_clients, self.fmts, self.codes,
+                                           self.segs, self.n_seg, self.n_elem, lr, params,
+                                           self.avg if want_avg else None, self.workspace, self.res_dec, stream=stream)
+        self._check(st, "co3_decode_aggregate_update")
+        return self.avg if want_avg else None
+
     # -- results --------------------------------------------------------------------------------
     def encode_results(self) -> np.ndarray:
         return B.read_results(self.res_enc, self.n_clients)
