@@ -3,7 +3,7 @@
 
 One step = one training round of the workload: every client's gradient is corrected, converted,
 entropy-coded (memory updated) in one batched `co3_encode` call, then all streams are decoded and
-averaged by `co3_decode_aggregate`.  Prints one JSON line (see README for the keys).
+averaged by `co3_decode_aggregate`.  Prints one JSON line (the README lists the keys).
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config 2]
 """

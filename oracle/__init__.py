@@ -84,6 +84,14 @@ def lib():
         L.co3o_decode_aggregate.argtypes = [C.c_void_p, C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p,
                                             C.c_void_p, C.c_uint32, C.c_uint32, C.c_uint32, C.c_void_p,
                                             C.c_void_p]
+        L.co3o_gennorm_kurtosis.restype = C.c_double
+        L.co3o_gennorm_kurtosis.argtypes = [C.c_double]
+        L.co3o_gennorm_shape_from_kurtosis.restype = C.c_double
+        L.co3o_gennorm_shape_from_kurtosis.argtypes = [C.c_double, C.c_double, C.c_double]
+        L.co3o_fit_scale.restype = C.c_int
+        L.co3o_fit_scale.argtypes = [C.c_void_p, C.c_void_p, C.c_float, C.c_uint64, C.c_uint32, C.c_uint64,
+                                     C.c_void_p, C.c_uint32, C.c_float, C.c_float,
+                                     C.POINTER(C.c_float), C.POINTER(C.c_float), C.c_void_p]
         L.co3o_ps_update.restype = None
         L.co3o_ps_update.argtypes = [C.c_void_p, C.c_void_p, C.c_float, C.c_uint64]
         _lib = L
@@ -246,3 +254,27 @@ def ps_update(w: np.ndarray, avg: np.ndarray, eta: float) -> None:
     assert w.dtype == np.float32 and avg.dtype == np.float32 and w.flags.c_contiguous and avg.flags.c_contiguous
     assert w.size == avg.size
     lib().co3o_ps_update(_ptr(w), _ptr(avg), C.c_float(eta), w.size)
+
+
+# ------------------------------------------------------------------------------------------ fitting
+def gennorm_kurtosis(beta: float) -> float:
+    return lib().co3o_gennorm_kurtosis(float(beta))
+
+
+def gennorm_shape_from_kurtosis(kurt: float, lo: float, hi: float) -> float:
+    return lib().co3o_gennorm_shape_from_kurtosis(float(kurt), float(lo), float(hi))
+
+
+def fit_scale(g: np.ndarray, m, decay: float, log_tab: np.ndarray, beta0: float, dbeta: float):
+    """g, m: float32 [n_clients][n] (m may be None).  Returns (status, scale, inv_scale, stats[4])."""
+    g = np.ascontiguousarray(g, dtype=np.float32)
+    if g.ndim == 1:
+        g = g[None, :]
+    if m is not None:
+        m = np.ascontiguousarray(m, dtype=np.float32).reshape(g.shape)
+    tab = np.ascontiguousarray(log_tab, dtype=np.float32)
+    sc, inv = C.c_float(0), C.c_float(0)
+    stats = np.zeros(4, dtype=np.float64)
+    st = lib().co3o_fit_scale(_ptr(g), _ptr(m), C.c_float(decay), g.shape[1], g.shape[0], g.shape[1], _ptr(tab), tab.size,
+                              C.c_float(beta0), C.c_float(dbeta), C.byref(sc), C.byref(inv), _ptr(stats))
+    return st, sc.value, inv.value, stats

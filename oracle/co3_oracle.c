@@ -591,3 +591,75 @@ void co3o_ps_update(float *w, const float *avg, float eta, uint64_t n)
         w[i] = w[i] - step;
     }
 }
+
+/*
+ * Fitting the converter's multiplier to a layer (Sec. III: the gradients of a layer are modelled as
+ * zero-mean generalized normal, GenNorm(0, alpha, beta); Sec. IV-A (i) and Eq. (exp bias): the multiplier
+ * minimises the expected squared conversion error under that model).
+ *
+ * Kurtosis of GenNorm as a function of the shape: Gamma(5/b) Gamma(1/b) / Gamma(3/b)^2 (Sec. III).
+ */
+double co3o_gennorm_kurtosis(double beta)
+{
+    return exp(lgamma(5.0 / beta) + lgamma(1.0 / beta) - 2.0 * lgamma(3.0 / beta));
+}
+
+/* Shape whose kurtosis is `kurt`, searched in [lo, hi] (the kurtosis falls as the shape grows); values
+ * outside the range of the interval's ends give the nearer end. */
+double co3o_gennorm_shape_from_kurtosis(double kurt, double lo, double hi)
+{
+    if (!(kurt < co3o_gennorm_kurtosis(lo))) return lo;
+    if (!(kurt > co3o_gennorm_kurtosis(hi))) return hi;
+    for (int it = 0; it < 200 && hi - lo > 1e-15 * hi; ++it) {
+        const double mid = 0.5 * (lo + hi);
+        if (co3o_gennorm_kurtosis(mid) > kurt) lo = mid; else hi = mid;
+    }
+    return 0.5 * (lo + hi);
+}
+
+/*
+ * One layer: moments of v = g + decay * m (m may be NULL: v = g) over the n_clients vectors of n elements
+ * each (client u at g + u * stride), all of which share the layer's format; from them
+ *   sigma^2 = sum v^2 / N,  kurtosis = N * sum v^4 / (sum v^2)^2  (zero mean: the model's location is 0),
+ *   beta  = shape with that kurtosis, kept inside the table's range,
+ *   alpha = sigma * sqrt(Gamma(1/beta) / Gamma(3/beta))        (variance of GenNorm, Sec. III),
+ *   scale = exp(interp(beta; log_tab)) / alpha, inv_scale = 1 / scale (fp32),
+ * where log_tab[i] is the natural logarithm of the best multiplier for unit alpha at shape
+ * beta0 + i * dbeta (the numerical minimiser of the conversion error, tabulated by the caller) and the
+ * interpolation is linear in the logarithm.  stats (nullable) receives sigma, kurtosis, beta, alpha.
+ * Returns 0, or CO3O_ERR_ARG when the layer is empty, all zero or holds a non-finite value (nothing is
+ * written then).
+ */
+int co3o_fit_scale(const float *g, const float *m, float decay, uint64_t n, uint32_t n_clients, uint64_t stride,
+                   const float *log_tab, uint32_t n_beta, float beta0, float dbeta,
+                   float *scale, float *inv_scale, double *stats)
+{
+    double s2 = 0.0, s4 = 0.0;
+    for (uint32_t u = 0; u < n_clients; ++u) {
+        for (uint64_t i = 0; i < n; ++i) {
+            const float gv = g[u * stride + i];
+            const float v = m ? fmaf(decay, m[u * stride + i], gv) : gv;
+            const double x2 = (double)v * (double)v;
+            s2 += x2;
+            s4 += x2 * x2;
+        }
+    }
+    const double N = (double)n * (double)n_clients;
+    if (n_beta < 2 || !(N > 0.0) || !(s2 > 0.0) || !isfinite(s2) || !isfinite(s4)) return CO3O_ERR_ARG;
+    const double sigma = sqrt(s2 / N), kurt = N * s4 / (s2 * s2);
+    const double blo = (double)beta0, bhi = (double)beta0 + (double)dbeta * (double)(n_beta - 1);
+    const double beta = co3o_gennorm_shape_from_kurtosis(kurt, blo, bhi);
+    const double alpha = sigma * sqrt(exp(lgamma(1.0 / beta) - lgamma(3.0 / beta)));
+    double x = (beta - blo) / (double)dbeta;
+    if (x < 0.0) x = 0.0;
+    uint32_t i = (uint32_t)x;
+    if (i > n_beta - 2) i = n_beta - 2;
+    const double f = x - (double)i;
+    const double log_s = (double)log_tab[i] + f * ((double)log_tab[i + 1] - (double)log_tab[i]);
+    const float sc = (float)(exp(log_s) / alpha);
+    if (!(sc > 0.0f) || isinf(sc)) return CO3O_ERR_ARG;
+    *scale = sc;
+    *inv_scale = 1.0f / sc;
+    if (stats) { stats[0] = sigma; stats[1] = kurt; stats[2] = beta; stats[3] = alpha; }
+    return CO3O_OK;
+}
