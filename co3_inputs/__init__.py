@@ -85,14 +85,28 @@ def client_round_seed(base: int, client: int, rnd: int) -> int:
 _SCALE_TABLE = None
 
 
-def scale_for(exp_bits: int, mant_bits: int, beta: float, alpha: float) -> tuple[float, float]:
-    """(scale, inv_scale) as fp32 values for a layer modelled as GenNorm(0, alpha, beta)."""
+def _scale_table() -> dict:
     global _SCALE_TABLE
     if _SCALE_TABLE is None:
         import json
         import os
         with open(os.path.join(os.path.dirname(os.path.abspath(__file__)), "scale_table.json")) as fh:
             _SCALE_TABLE = json.load(fh)
+    return _SCALE_TABLE
+
+
+def scale_log_table(formats) -> tuple[np.ndarray, float, float]:
+    """(float32[len(formats)][n_beta] natural logarithms of the stored multipliers, beta0, dbeta) for the given
+    (exp_bits, mant_bits) pairs: the table a data-driven fit of the multiplier interpolates in."""
+    t = _scale_table()
+    betas = np.asarray(t["betas"], dtype=np.float64)
+    rows = [np.log(np.asarray(t["formats"]["%d,%d" % (E, M)], dtype=np.float64)) for (E, M) in formats]
+    return np.asarray(rows, dtype=np.float32), float(betas[0]), float(betas[1] - betas[0])
+
+
+def scale_for(exp_bits: int, mant_bits: int, beta: float, alpha: float) -> tuple[float, float]:
+    """(scale, inv_scale) as fp32 values for a layer modelled as GenNorm(0, alpha, beta)."""
+    _SCALE_TABLE = _scale_table()
     betas = np.asarray(_SCALE_TABLE["betas"], dtype=np.float64)
     row = np.asarray(_SCALE_TABLE["formats"]["%d,%d" % (exp_bits, mant_bits)], dtype=np.float64)
     b = min(max(float(beta), float(betas[0])), float(betas[-1]))

@@ -179,6 +179,34 @@ int co3_code_build_device(const uint64_t* weights, const co3_fmt* fmts, uint32_t
                           co3_result* res, void* stream);
 
 /*
+ * Fit of every layer's multiplier to this round's data, on the device (Sec. III: a layer's gradient entries
+ * are modelled as zero-mean generalized normal, GenNorm(alpha, beta), with kurtosis
+ * Gamma(5/beta) Gamma(1/beta) / Gamma(3/beta)^2 and variance alpha^2 Gamma(3/beta) / Gamma(1/beta);
+ * Sec. IV-A (i): the bias is the one that minimises the expected squared conversion error under that model,
+ * found numerically once per shape and tabulated, Sec. IV-B).  Per layer k, over all n_clients vectors:
+ *     v = g + decay * m (v = g when mem is NULL);  sigma^2 = sum v^2 / N;  kurtosis = N sum v^4 / (sum v^2)^2
+ *     beta = the shape with that kurtosis, kept inside the table's range [beta0, beta0 + (n_beta-1) dbeta]
+ *     alpha = sigma * sqrt(Gamma(1/beta) / Gamma(3/beta))
+ *     fmts[k].scale = exp(table(beta)) / alpha,  fmts[k].inv_scale = fl32(1 / scale)
+ * where table is row seg_tab[k] (row 0 if seg_tab is NULL) of log_tab and is interpolated linearly; its entry i
+ * is the natural logarithm of the best multiplier for alpha = 1 at shape beta0 + i * dbeta.  Sums are fp64 in a
+ * fixed order (results do not depend on the launch shape or on timing); the other fields of fmts are not read.
+ *   grad, mem [device]  as in co3_convert, both read only; mem nullable
+ *   fmts [device]       n_seg entries; scale and inv_scale of every fitted layer are overwritten
+ *   log_tab [device]    float[n_tab][n_beta];  seg_tab [device, nullable] uint32[n_seg], entries < n_tab
+ *   stats_out [device, nullable] double[n_seg][4]: sigma, kurtosis, beta, alpha of every fitted layer
+ *   res [device]        one co3_result: CO3_ERR_INVALID_ARG if a layer is empty, all zero or holds a non-finite
+ *                       value, or its table index is out of range (first_bad_chunk = smallest such layer); those
+ *                       layers' formats are left untouched
+ *   workspace           sized by co3_workspace_bytes with this n_clients (>= 1)
+ */
+int co3_fit_scale(const float* grad, const float* mem, float decay, co3_fmt* fmts, const co3_seg* segs,
+                  uint32_t n_seg, uint64_t n_elem, uint32_t n_clients, uint64_t client_stride_elems,
+                  const float* log_tab, const uint32_t* seg_tab, uint32_t n_tab, uint32_t n_beta,
+                  float beta0, float dbeta, double* stats_out, co3_result* res,
+                  void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * Client uplink for n_clients clients: correct + convert + encode + memory update, codes given.
  *   streams_out [device]  client u's container starts at streams_out + u * stream_capacity
  *                         (stream_capacity a multiple of 16); layout below
@@ -254,7 +282,8 @@ int co3_decode(const uint8_t* stream_in, size_t stream_bytes,
 #define CO3_KERNEL_COMPACT 4  /* payload compaction */
 #define CO3_KERNEL_CODE_BUILD 5 /* Huffman tables from weights on the device */
 #define CO3_KERNEL_DECODE 6   /* decode + cross-client accumulate */
-#define CO3_KERNEL_COUNT 7
+#define CO3_KERNEL_FIT 7      /* moments and multiplier fit */
+#define CO3_KERNEL_COUNT 8
 int co3_profile_enable(int on);
 int co3_profile_read(double* total_ms /* [host] */, uint32_t* launches /* [host] */);
 

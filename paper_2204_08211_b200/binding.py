@@ -46,6 +46,7 @@ def _load():
     L.co3_convert_static.argtypes = [vp, vp, f32, vp, vp, u32, u64, u32, u64, vp, vp, vp, vp]
     L.co3_code_build.argtypes = [vp, vp, vp]
     L.co3_code_build_device.argtypes = [vp, vp, u32, vp, vp, vp]
+    L.co3_fit_scale.argtypes = [vp, vp, f32, vp, vp, u32, u64, u32, u64, vp, vp, u32, u32, f32, f32, vp, vp, vp, sz, vp]
     L.co3_encode.argtypes = [vp, vp, f32, vp, vp, vp, u32, u64, u32, u64, vp, sz, u32, vp, sz, vp, vp]
     L.co3_encode_symbols.argtypes = [vp, vp, vp, u32, u64, u32, u64, vp, sz, u32, vp, sz, vp, vp]
     L.co3_decode_aggregate.argtypes = [vp, sz, u32, vp, vp, vp, u32, u64, u32, vp, vp, sz, vp, vp]
@@ -53,7 +54,7 @@ def _load():
     L.co3_decode.argtypes = [vp, sz, vp, vp, vp, u32, u64, u32, vp, vp, vp, sz, vp, vp]
     L.co3_profile_enable.argtypes = [C.c_int]
     L.co3_profile_read.argtypes = [vp, vp]
-    for name in ("co3_profile_enable", "co3_profile_read", "co3_convert_static", "co3_workspace_bytes", "co3_stream_capacity_bytes", "co3_convert", "co3_code_build", "co3_code_build_device", "co3_encode",
+    for name in ("co3_fit_scale", "co3_profile_enable", "co3_profile_read", "co3_convert_static", "co3_workspace_bytes", "co3_stream_capacity_bytes", "co3_convert", "co3_code_build", "co3_code_build_device", "co3_encode",
                  "co3_encode_symbols", "co3_decode_aggregate", "co3_decode_aggregate_update", "co3_decode"):
         getattr(L, name).restype = C.c_int
     _lib = L
@@ -167,6 +168,15 @@ def co3_convert_static(grad, mem, decay, fmts, segs, n_seg, n_elem, n_clients, c
                                       _dev(res), _stream(stream))
 
 
+def co3_fit_scale(grad, mem, decay, fmts, segs, n_seg, n_elem, n_clients, client_stride_elems, log_tab, seg_tab,
+                  n_tab, n_beta, beta0, dbeta, stats_out, res, workspace, stream=None) -> int:
+    """Writes scale / inv_scale of every layer's co3_fmt on the device; mem, seg_tab, stats_out may be None."""
+    return _load().co3_fit_scale(_dev(grad), _dev(mem, True), float(decay), _dev(fmts), _dev(segs), n_seg, n_elem,
+                                 n_clients, client_stride_elems, _dev(log_tab), _dev(seg_tab, True), n_tab, n_beta,
+                                 float(beta0), float(dbeta), _dev(stats_out, True), _dev(res), _dev(workspace),
+                                 workspace.numel() * workspace.element_size(), _stream(stream))
+
+
 def co3_encode(grad, mem, decay, fmts, codes, segs, n_seg, n_elem, n_clients, client_stride_elems, streams_out,
                stream_capacity, workspace, res, chunk_syms: int = CHUNK_SYMS, stream=None) -> int:
     return _load().co3_encode(_dev(grad), _dev(mem), float(decay), _dev(fmts), _dev(codes), _dev(segs), n_seg,
@@ -207,7 +217,7 @@ def co3_decode(stream_in, stream_bytes, fmts, codes, segs, n_seg, n_elem, ghat_o
                               workspace.numel() * workspace.element_size(), _dev(res), _stream(stream))
 
 
-KERNEL_NAMES = ("prepare", "convert", "pack", "scan", "compact", "code_build", "decode")
+KERNEL_NAMES = ("prepare", "convert", "pack", "scan", "compact", "code_build", "decode", "fit")
 
 
 def co3_profile_enable(on: bool) -> int:

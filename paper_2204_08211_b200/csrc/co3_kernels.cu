@@ -1656,6 +1656,181 @@ __global__ void __launch_bounds__(kThreads) code_build_kernel(CodeBuildArgs a) {
     }
 }
 
+// ------------------------------------------------------------------------------------------------
+// Fit of the converter's multiplier (Sec. III: a layer's gradients are zero-mean GenNorm(alpha, beta);
+// Sec. IV-A (i): the multiplier minimises the expected squared conversion error under that model).
+//   moments_kernel   per (chunk, client): sum v^2 and sum v^4 in fp64, v = g + gamma*m, fixed summation tree
+//   fit_kernel       per layer: partial sums in fixed order -> sigma, kurtosis -> shape by bisection on
+//                    Gamma(5/b)Gamma(1/b)/Gamma(3/b)^2 -> alpha -> tabulated best multiplier / alpha
+// ------------------------------------------------------------------------------------------------
+struct FitArgs {
+    const float* grad;
+    const float* mem;  // nullable: v = g
+    float decay;
+    uint64_t client_stride;
+    uint32_t n_clients;
+    co3_fmt* fmts;
+    const co3_seg* segs;
+    uint32_t n_seg;
+    const float* log_tab;     // [n_tab][n_beta]
+    const uint32_t* seg_tab;  // nullable: every layer uses table 0
+    uint32_t n_tab, n_beta;
+    float beta0, dbeta;
+    double* stats;  // nullable, [n_seg][4]
+    double2* part;  // [n_clients][n_chunks_max]
+    co3_result* res;
+    Ws ws;
+};
+
+constexpr int kMomChunks = 4;  // chunks of one client per block
+
+__device__ __forceinline__ void moments_add(float g, float m, float decay, bool has_m, double& s2, double& s4) {
+    const float v = has_m ? __fmaf_rn(decay, m, g) : g;
+    const double x2 = __dmul_rn((double)v, (double)v);
+    s2 = __dadd_rn(s2, x2);
+    s4 = __dadd_rn(s4, __dmul_rn(x2, x2));
+}
+
+__global__ void __launch_bounds__(kThreads) moments_kernel(FitArgs a) {
+    __shared__ double s_red[kMomChunks][2][kThreads / 32];
+    const Ctrl* ctrl = a.ws.ctrl;
+    if (ctrl->abort) return;
+    const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
+    const uint32_t n_chunks = ctrl->n_chunks, client = blockIdx.y;
+    const bool has_m = a.mem != nullptr;
+    const uint32_t i0 = tid * 8;
+    const uint32_t c_first = blockIdx.x * kMomChunks;
+    float g[kMomChunks][8], m[kMomChunks][8];
+    uint32_t nv[kMomChunks];
+    // all loads of the block's chunks first, then the arithmetic
+#pragma unroll
+    for (int j = 0; j < kMomChunks; ++j) {
+        const uint32_t c = c_first + j;
+        nv[j] = 0;
+        if (c >= n_chunks) continue;
+        const ChunkDesc d = a.ws.chunk_desc[c];
+        const uint64_t base = (uint64_t)client * a.client_stride + d.elem0;
+        const float* gp = a.grad + base;
+        const float* mp = has_m ? a.mem + base : gp;
+        nv[j] = d.cnt > i0 ? min(8u, d.cnt - i0) : 0u;
+        const bool vec = d.cnt == (uint32_t)kC && ((reinterpret_cast<uintptr_t>(gp) | reinterpret_cast<uintptr_t>(mp)) & 15u) == 0;
+        if (vec) {
+            load8_vec(gp + i0, g[j]);
+            if (has_m) load8_vec(mp + i0, m[j]);
+        } else {
+            load8_any(gp + i0, nv[j], g[j]);
+            if (has_m) load8_any(mp + i0, nv[j], m[j]);
+        }
+    }
+#pragma unroll
+    for (int j = 0; j < kMomChunks; ++j) {
+        double s2 = 0.0, s4 = 0.0;
+#pragma unroll
+        for (int e = 0; e < 8; ++e)
+            if ((uint32_t)e < nv[j]) moments_add(g[j][e], has_m ? m[j][e] : 0.0f, a.decay, has_m, s2, s4);
+#pragma unroll
+        for (int w = 16; w > 0; w >>= 1) {
+            s2 = __dadd_rn(s2, __shfl_xor_sync(0xffffffffu, s2, w));
+            s4 = __dadd_rn(s4, __shfl_xor_sync(0xffffffffu, s4, w));
+        }
+        if (lane == 0) { s_red[j][0][warp] = s2; s_red[j][1][warp] = s4; }
+    }
+    __syncthreads();
+    if (tid < (uint32_t)kMomChunks && c_first + tid < n_chunks) {
+        double t2 = 0.0, t4 = 0.0;
+#pragma unroll
+        for (int w = 0; w < kThreads / 32; ++w) { t2 = __dadd_rn(t2, s_red[tid][0][w]); t4 = __dadd_rn(t4, s_red[tid][1][w]); }
+        a.part[(size_t)client * a.ws.n_chunks_max + c_first + tid] = make_double2(t2, t4);
+    }
+}
+
+__device__ __forceinline__ double gennorm_kurtosis(double beta) {
+    return exp(lgamma(5.0 / beta) + lgamma(1.0 / beta) - 2.0 * lgamma(3.0 / beta));
+}
+
+__global__ void __launch_bounds__(kThreads) fit_kernel(FitArgs a) {
+    __shared__ double s_red[2][kThreads / 32];
+    const Ctrl* ctrl = a.ws.ctrl;
+    if (ctrl->abort) return;
+    const uint32_t k = blockIdx.x, tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
+    const uint32_t c0 = a.ws.first_chunk[k], nck = a.ws.first_chunk[k + 1] - c0;
+    const uint64_t items = (uint64_t)nck * a.n_clients;
+    double s2 = 0.0, s4 = 0.0;
+    for (uint64_t i = tid; i < items; i += kThreads) {
+        const uint32_t u = (uint32_t)(i / nck), c = (uint32_t)(i % nck);
+        const double2 p = a.part[(size_t)u * a.ws.n_chunks_max + c0 + c];
+        s2 = __dadd_rn(s2, p.x);
+        s4 = __dadd_rn(s4, p.y);
+    }
+#pragma unroll
+    for (int w = 16; w > 0; w >>= 1) {
+        s2 = __dadd_rn(s2, __shfl_xor_sync(0xffffffffu, s2, w));
+        s4 = __dadd_rn(s4, __shfl_xor_sync(0xffffffffu, s4, w));
+    }
+    if (lane == 0) { s_red[0][warp] = s2; s_red[1][warp] = s4; }
+    __syncthreads();
+    if (warp != 0) return;
+    s2 = s4 = 0.0;
+#pragma unroll
+    for (int w = 0; w < kThreads / 32; ++w) { s2 = __dadd_rn(s2, s_red[0][w]); s4 = __dadd_rn(s4, s_red[1][w]); }
+
+    // warp 0, every lane with the same values
+    const double N = (double)a.segs[k].n_elem * (double)a.n_clients;
+    bool ok = a.n_beta >= 2 && N > 0.0 && s2 > 0.0 && isfinite(s2) && isfinite(s4);
+    const uint32_t tab = a.seg_tab ? a.seg_tab[k] : 0u;
+    if (tab >= a.n_tab) ok = false;
+    float sc = 0.0f;
+    double sigma = 0.0, kurt = 0.0, beta = 0.0, alpha = 0.0;
+    if (ok) {
+        sigma = sqrt(s2 / N);
+        kurt = N * s4 / (s2 * s2);
+        const double blo = (double)a.beta0, bhi = (double)a.beta0 + (double)a.dbeta * (double)(a.n_beta - 1);
+        // the kurtosis falls as the shape grows; outside the table's range the nearer end is taken.  Inside, the
+        // interval is cut into 33 parts per round, one interior point per lane, until it is as narrow as fp64 allows
+        double lo = blo, hi = bhi;
+        const double k_end = gennorm_kurtosis(lane == 0 ? lo : hi);
+        const bool below_lo = !(kurt < __shfl_sync(0xffffffffu, k_end, 0));
+        const bool above_hi = !(kurt > __shfl_sync(0xffffffffu, k_end, 1));
+        if (below_lo) beta = lo;
+        else if (above_hi) beta = hi;
+        else {
+            for (int it = 0; it < 64 && hi - lo > 1e-15 * hi; ++it) {
+                const double w = hi - lo;
+                const double x = lo + w * ((double)(lane + 1) / 33.0);
+                const uint32_t left = __popc(__ballot_sync(0xffffffffu, gennorm_kurtosis(x) > kurt));  // points left of the root
+                const double nlo = left == 0 ? lo : lo + w * ((double)left / 33.0);
+                const double nhi = left == 32 ? hi : lo + w * ((double)(left + 1) / 33.0);
+                if (!(nhi - nlo < w)) break;  // no further progress in fp64
+                lo = nlo;
+                hi = nhi;
+            }
+            beta = 0.5 * (lo + hi);
+        }
+        alpha = sigma * sqrt(exp(lgamma(1.0 / beta) - lgamma(3.0 / beta)));
+        double x = (beta - blo) / (double)a.dbeta;
+        if (x < 0.0) x = 0.0;
+        uint32_t i = (uint32_t)x;
+        if (i > a.n_beta - 2) i = a.n_beta - 2;
+        const double f = x - (double)i;
+        const float* t = a.log_tab + (size_t)tab * a.n_beta;
+        const double log_s = (double)t[i] + f * ((double)t[i + 1] - (double)t[i]);
+        sc = (float)(exp(log_s) / alpha);
+        if (!(sc > 0.0f) || isinf(sc)) ok = false;
+    }
+    if (lane != 0) return;
+    if (!ok) {  // empty, all-zero or non-finite layer, or no usable table: the format is left as it was
+        set_status(&a.res[0], CO3_ERR_INVALID_ARG);
+        atomicMin(&a.res[0].first_bad_chunk, k);
+        return;
+    }
+    a.fmts[k].scale = sc;
+    a.fmts[k].inv_scale = __fdiv_rn(1.0f, sc);
+    if (a.stats) {
+        double* st = a.stats + 4 * (size_t)k;
+        st[0] = sigma; st[1] = kurt; st[2] = beta; st[3] = alpha;
+    }
+}
+
 }  // namespace co3
 
 // ================================================================================================
@@ -2036,6 +2211,36 @@ int co3_convert_static(const float* grad, float* mem, float decay, const co3_fmt
     if (ra != CO3_OK) return ra;
     return co3_convert(grad, mem, decay, fmts, segs, n_seg, n_elem, n_clients, client_stride_elems, sym_out, hist_out,
                        res, scratch, (size_t)CO3_STATIC_SCRATCH_BYTES, stream);
+}
+
+int co3_fit_scale(const float* grad, const float* mem, float decay, co3_fmt* fmts, const co3_seg* segs, uint32_t n_seg,
+                  uint64_t n_elem, uint32_t n_clients, uint64_t client_stride_elems, const float* log_tab,
+                  const uint32_t* seg_tab, uint32_t n_tab, uint32_t n_beta, float beta0, float dbeta, double* stats_out,
+                  co3_result* res, void* workspace, size_t workspace_bytes, void* stream) {
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (!grad || !fmts || !segs || !log_tab || !res || !workspace || n_seg == 0 || n_clients == 0 || n_clients > 65535u)
+        return CO3_ERR_INVALID_ARG;
+    if (n_tab == 0 || n_beta < 2 || !(dbeta > 0.0f) || !(beta0 > 0.0f)) return CO3_ERR_INVALID_ARG;
+    if (!aligned(grad, 16) || (mem && !aligned(mem, 16)) || !aligned(workspace, 256) || !aligned(res, 8) ||
+        !aligned(fmts, 4) || !aligned(log_tab, 4) || (stats_out && !aligned(stats_out, 8)))
+        return CO3_ERR_INVALID_ARG;
+    if (n_clients > 1 && client_stride_elems < n_elem) return CO3_ERR_INVALID_ARG;
+    WsLayout L;
+    if (!ws_layout(n_elem, n_seg, n_clients, &L)) return CO3_ERR_INVALID_ARG;
+    if (workspace_bytes < L.total) return CO3_ERR_CAPACITY;
+    const Ws ws = ws_pointers(workspace, L);
+    // layout only: the formats' multipliers are what this call produces, so they are not validated here
+    const int rc = begin_call(L, ws, res, 1, st, nullptr, nullptr, segs, n_seg, n_elem, 1, 1);
+    if (rc != CO3_OK) return rc;
+    // the per-(chunk, client) partial sums take the place of the encoder's chunk slots (16 of 4096 bytes each)
+    FitArgs fa{grad, mem, decay, client_stride_elems, n_clients, fmts, segs, n_seg, log_tab, seg_tab, n_tab, n_beta,
+               beta0, dbeta, stats_out, reinterpret_cast<double2*>(ws.slots), res, ws};
+    if (L.n_chunks_max) {
+        const dim3 grid((L.n_chunks_max + kMomChunks - 1) / kMomChunks, n_clients);
+        CO3_LAUNCH(CO3_KERNEL_FIT, st, moments_kernel<<<grid, kThreads, 0, st>>>(fa));
+    }
+    CO3_LAUNCH(CO3_KERNEL_FIT, st, fit_kernel<<<n_seg, kThreads, 0, st>>>(fa));
+    return CO3_OK;
 }
 
 int co3_encode(const float* grad, float* mem, float decay, const co3_fmt* fmts, const co3_code* codes,

@@ -46,6 +46,22 @@ class Co3Session:
     def client_view(self, buf: torch.Tensor, u: int) -> torch.Tensor:
         return buf[u * self.stride:u * self.stride + self.n_elem]
 
+    # -- multiplier fitting -------------------------------------------------------------------
+    def fit_scales(self, grads: torch.Tensor, mems, log_tab: torch.Tensor, beta0: float, dbeta: float,
+                   seg_tab=None, stats_out=None, stream=None) -> None:
+        """Refits scale / inv_scale of every layer's format on the device from this round's gradients (and
+        memories, if given): log_tab float32[n_tab][n_beta] and seg_tab int32[n_seg] (optional) are CUDA tensors.
+        The host copy of the formats is stale afterwards until fmts_from_device() is called."""
+        st = B.co3_fit_scale(grads, mems, self.decay, self.fmts, self.segs, self.n_seg, self.n_elem, self.n_clients,
+                             self.stride, log_tab, seg_tab, log_tab.shape[0], log_tab.shape[1], beta0, dbeta,
+                             stats_out, self.res_fit, self.workspace, stream)
+        self._check(st, "co3_fit_scale")
+
+    def fmts_from_device(self) -> np.ndarray:
+        raw = self.fmts.cpu().numpy().tobytes()[:self.n_seg * B.FMT_DTYPE.itemsize]
+        self.fmts_host = np.frombuffer(raw, dtype=B.FMT_DTYPE).copy()
+        return self.fmts_host
+
     # -- code fitting -------------------------------------------------------------------------
     def histogram(self, grads: torch.Tensor, mems: torch.Tensor, stream=None, sym_out=None, to_host: bool = True):
         """Symbol counts per layer summed over clients for this round; `mems` is updated like a real round
