@@ -71,6 +71,16 @@ def symbol_probabilities(fmt: Fmt, beta: float, alpha: float) -> np.ndarray:
     return p
 
 
+MODEL_WEIGHT_ONE = 1 << 30  # weight of probability 1
+
+
+def model_weights(fmt: Fmt, beta: float, alpha: float) -> np.ndarray:
+    """Integer Huffman weights of the 256 symbols from the model pmf (Sec. IV-A (ii): the code is designed for
+    the GenNorm distribution fitted to the layer): floor(p * 2^30), 0 for symbols the format never produces."""
+    p = symbol_probabilities(fmt, beta, alpha)
+    return np.floor(p * float(MODEL_WEIGHT_ONE)).astype(np.uint64)
+
+
 def optimal_scale(exp_bits: int, mant_bits: int, beta: float, flush_subnormals: bool = False,
                   lo: float = 1e-4, hi: float = 1e6, grid: int = 2001) -> tuple[float, float]:
     """argmin over s of quantization_mse for unit-scale GenNorm: log grid, then golden section."""

@@ -88,3 +88,48 @@ def test_gennorm_generator_moments():
             assert abs(k - kurt) < 1e-9
         assert abs((x ** 4).mean() / x.var() ** 2 - k) / k < 0.08
         assert abs(x.mean()) < 5e-6
+
+
+def test_model_weights_closed_forms_for_laplace_and_normal_layers():
+    """Cell probabilities of the model pmf against the two shapes with elementary distribution functions:
+    beta = 1 (Laplace, P(|X| <= e) = 1 - exp(-e/alpha)) and beta = 2 (normal, P(|X| <= e) = erf(e/alpha))."""
+    alpha = 2e-3
+    for E, M, flush in ((4, 3, False), (2, 1, False), (3, 0, False), (4, 3, True)):
+        for beta, cdf in ((1.0, lambda e: -math.expm1(-e / alpha)), (2.0, lambda e: math.erf(e / alpha))):
+            fmt = oracle.make_fmt(E, M, 37.0 / alpha, flush)
+            codes, lv = oracle.levels(fmt)
+            rec = lv / float(fmt.scale)
+            edges = np.concatenate([[0.0], 0.5 * (rec[1:] + rec[:-1]), [np.inf]])
+            want = np.zeros(256)
+            nb = E + M
+            for c, lo, hi in zip(codes, edges[:-1], edges[1:]):
+                ph = 0.5 * ((1.0 if np.isinf(hi) else cdf(hi)) - cdf(lo))
+                if c == 0:
+                    want[0] = 2 * ph
+                else:
+                    want[int(c)] = want[int(c) | (1 << nb)] = ph
+            w = bias.model_weights(fmt, beta, alpha)
+            assert w.dtype == np.uint64
+            assert np.abs(w.astype(np.float64) - want * 2.0 ** 30).max() < 1.001     # the flooring, nothing else
+            # mass is complete up to the flooring, symmetric in the sign, zero where the format has no symbol
+            assert 2 ** 30 - 256 <= int(w.sum()) <= 2 ** 30
+            assert np.array_equal(w[1:1 << nb], w[(1 << nb) + 1:2 << nb]) and w[1 << nb] == 0
+            for sym in range(256):
+                if not oracle.symbol_valid(fmt, sym):
+                    assert w[sym] == 0
+
+
+def test_model_weights_follow_the_histogram_of_model_samples():
+    from co3_inputs import gennorm, scale_for
+    beta, alpha = 0.8, 1e-3
+    s, inv = scale_for(4, 3, beta, alpha)
+    fmt = oracle.Fmt(4, 3, 0, s, inv)
+    x = gennorm(1 << 21, beta, alpha, seed=33).numpy()
+    sym = oracle.convert(x, np.zeros_like(x), 0.0, fmt)["sym"]
+    freq = np.bincount(sym, minlength=256) / x.size
+    w = bias.model_weights(fmt, beta, alpha).astype(np.float64) / 2.0 ** 30
+    assert np.abs(freq - w).max() < 3e-3
+    # and the code built from them is within a few hundredths of a bit of the one fitted to the data itself
+    ln_model, _ = oracle.code_arrays(oracle.code_build(bias.model_weights(fmt, beta, alpha), fmt))
+    ln_hist, _ = oracle.code_arrays(oracle.code_build(np.bincount(sym, minlength=256).astype(np.uint64), fmt))
+    assert (freq * ln_model).sum() - (freq * ln_hist).sum() < 0.05
