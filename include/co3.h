@@ -207,6 +207,21 @@ int co3_fit_scale(const float* grad, const float* mem, float decay, co3_fmt* fmt
                   void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * Huffman weights of every layer from its fitted model instead of from counted symbols (Sec. IV-A (ii): the code
+ * is designed for the GenNorm distribution of the layer).  The weight of a symbol is floor(p * 2^30), p the
+ * GenNorm(0, alpha, beta) mass of the inputs that the converter, with the layer's multiplier, sends to that
+ * symbol's level (between the midpoints to the neighbouring levels; beyond the last level everything; zero
+ * collects both signs); symbols the format never produces get 0.  Feed the result to co3_code_build_device.
+ *   fmts [device]        n_seg formats with their multipliers (as left by co3_fit_scale, or the caller's)
+ *   stats [device]       double[n_seg][4] laid out as co3_fit_scale's stats_out: beta at [2], alpha at [3]
+ *   weights_out [device] uint64[n_seg][256], fully overwritten
+ *   res [device]         one co3_result: CO3_ERR_INVALID_ARG if a layer's format, beta or alpha is unusable
+ *                        (first_bad_chunk = smallest such layer; its weights are all zero)
+ */
+int co3_model_weights(const co3_fmt* fmts, const double* stats, uint32_t n_seg, uint64_t* weights_out,
+                      co3_result* res, void* stream);
+
+/*
  * Client uplink for n_clients clients: correct + convert + encode + memory update, codes given.
  *   streams_out [device]  client u's container starts at streams_out + u * stream_capacity
  *                         (stream_capacity a multiple of 16); layout below
@@ -282,7 +297,7 @@ int co3_decode(const uint8_t* stream_in, size_t stream_bytes,
 #define CO3_KERNEL_COMPACT 4  /* payload compaction */
 #define CO3_KERNEL_CODE_BUILD 5 /* Huffman tables from weights on the device */
 #define CO3_KERNEL_DECODE 6   /* decode + cross-client accumulate */
-#define CO3_KERNEL_FIT 7      /* moments and multiplier fit */
+#define CO3_KERNEL_FIT 7      /* moments, multiplier fit, model weights */
 #define CO3_KERNEL_COUNT 8
 int co3_profile_enable(int on);
 int co3_profile_read(double* total_ms /* [host] */, uint32_t* launches /* [host] */);

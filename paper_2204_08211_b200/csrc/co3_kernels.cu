@@ -1831,6 +1831,96 @@ __global__ void __launch_bounds__(kThreads) fit_kernel(FitArgs a) {
     }
 }
 
+// ------------------------------------------------------------------------------------------------
+// Huffman weights from the model (Sec. IV-A (ii): the code of a layer is designed for the GenNorm distribution
+// fitted to it).  The probability of a symbol is the GenNorm mass of the interval of inputs the converter sends
+// to its level: between the midpoints to the neighbouring levels, divided by the multiplier; the last level's
+// interval has no upper end.  With F the distribution function of GenNorm(0, alpha, beta),
+// F(x) - 1/2 = P(1/beta, (x/alpha)^beta) / 2 for x >= 0, P the regularised lower incomplete gamma function.
+// ------------------------------------------------------------------------------------------------
+struct WeightArgs {
+    const co3_fmt* fmts;
+    const double* stats;  // [n_seg][4]: beta at [2], alpha at [3]
+    uint64_t* weights;    // [n_seg][256]
+    co3_result* res;
+};
+
+// P(a, x) for a > 0, x >= 0: power series below x = a + 1, continued fraction of the complement above.
+__device__ double gamma_p(double a, double x, double lgamma_a) {
+    if (!(x > 0.0)) return 0.0;
+    if (isinf(x)) return 1.0;
+    const double front = exp(a * log(x) - x - lgamma_a);  // x^a e^-x / Gamma(a)
+    if (x < a + 1.0) {
+        double term = 1.0 / a, sum = term;
+        for (int n = 1; n < 1000; ++n) {
+            term *= x / (a + (double)n);
+            sum += term;
+            if (term < sum * 1e-17) break;
+        }
+        return fmin(1.0, front * sum);
+    }
+    const double tiny = 1e-300;
+    double b = x + 1.0 - a, c = 1.0 / tiny, d = 1.0 / b, h = d;
+    for (int i = 1; i < 1000; ++i) {
+        const double an = -(double)i * ((double)i - a);
+        b += 2.0;
+        d = an * d + b;
+        if (fabs(d) < tiny) d = tiny;
+        c = b + an / c;
+        if (fabs(c) < tiny) c = tiny;
+        d = 1.0 / d;
+        const double del = d * c;
+        h *= del;
+        if (fabs(del - 1.0) < 1e-16) break;
+    }
+    return fmax(0.0, 1.0 - front * h);
+}
+
+// Value of magnitude code c in the format (E, M), before the multiplier.
+__device__ __forceinline__ double level_of(uint32_t c, uint32_t M, int emin) {
+    const uint32_t efield = c >> M, mfield = c & ((1u << M) - 1u);
+    if (efield == 0) return ldexp((double)mfield, emin - (int)M);
+    return ldexp(1.0 + ldexp((double)mfield, -(int)M), (int)efield - 1 + emin);
+}
+
+__global__ void __launch_bounds__(kThreads) model_weights_kernel(WeightArgs a) {
+    const uint32_t k = blockIdx.x, sym = threadIdx.x;
+    const co3_fmt f = a.fmts[k];
+    const double beta = a.stats[4 * (size_t)k + 2], alpha = a.stats[4 * (size_t)k + 3];
+    const uint32_t E = f.exp_bits, M = f.mant_bits;
+    const bool ok = E >= 2 && 1 + E + M <= 8 && (f.flags & ~CO3_FMT_FLUSH_SUBNORMALS) == 0 && f.scale > 0.0f &&
+                    !isinf(f.scale) && beta > 0.0 && alpha > 0.0 && isfinite(beta) && isfinite(alpha);
+    uint64_t w = 0;
+    if (ok) {
+        const bool flush = (f.flags & CO3_FMT_FLUSH_SUBNORMALS) != 0;
+        const int emin = -((1 << (E - 1)) - 2);
+        const uint32_t nb = E + M, max_code = (((1u << E) - 2u) << M) | ((1u << M) - 1u);
+        const uint32_t sign = sym >> nb, c = sym & ((1u << nb) - 1u);
+        const bool valid = sym < (2u << nb) && c <= max_code && !(sign && c == 0) && !(flush && c != 0 && (c >> M) == 0);
+        if (valid) {
+            const double inv_a = 1.0 / beta, lg = lgamma(inv_a);
+            const double here = level_of(c, M, emin);
+            double lo = 0.0, hi = INFINITY;  // ends of the interval, in units of the input
+            if (c != 0) {
+                const uint32_t prev = (flush && c == (1u << M)) ? 0u : c - 1u;
+                lo = 0.5 * (level_of(prev, M, emin) + here) / (double)f.scale;
+            }
+            if (c != max_code) {
+                const uint32_t next = (flush && c == 0) ? (1u << M) : c + 1u;
+                hi = 0.5 * (here + level_of(next, M, emin)) / (double)f.scale;
+            }
+            const double p_lo = gamma_p(inv_a, pow(lo / alpha, beta), lg);
+            const double p_hi = isinf(hi) ? 1.0 : gamma_p(inv_a, pow(hi / alpha, beta), lg);
+            const double p = (c == 0 ? 1.0 : 0.5) * (p_hi - p_lo);  // zero collects both signs
+            w = p > 0.0 ? (uint64_t)floor(p * 1073741824.0) : 0ull;
+        }
+    } else if (sym == 0) {
+        set_status(&a.res[0], CO3_ERR_INVALID_ARG);
+        atomicMin(&a.res[0].first_bad_chunk, k);
+    }
+    a.weights[(size_t)k * 256 + sym] = w;
+}
+
 }  // namespace co3
 
 // ================================================================================================
@@ -2240,6 +2330,18 @@ int co3_fit_scale(const float* grad, const float* mem, float decay, co3_fmt* fmt
         CO3_LAUNCH(CO3_KERNEL_FIT, st, moments_kernel<<<grid, kThreads, 0, st>>>(fa));
     }
     CO3_LAUNCH(CO3_KERNEL_FIT, st, fit_kernel<<<n_seg, kThreads, 0, st>>>(fa));
+    return CO3_OK;
+}
+
+int co3_model_weights(const co3_fmt* fmts, const double* stats, uint32_t n_seg, uint64_t* weights_out, co3_result* res,
+                      void* stream) {
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (!fmts || !stats || !weights_out || !res || n_seg == 0 || n_seg > (1u << 20)) return CO3_ERR_INVALID_ARG;
+    if (!aligned(fmts, 4) || !aligned(stats, 8) || !aligned(weights_out, 8) || !aligned(res, 8)) return CO3_ERR_INVALID_ARG;
+    CO3_CUDA(cudaMemsetAsync(res, 0, sizeof(co3_result), st));
+    CO3_CUDA(cudaMemsetAsync(&res->first_bad_chunk, 0xff, 4, st));
+    WeightArgs wa{fmts, stats, weights_out, res};
+    CO3_LAUNCH(CO3_KERNEL_FIT, st, model_weights_kernel<<<n_seg, kThreads, 0, st>>>(wa));
     return CO3_OK;
 }
 

@@ -35,6 +35,7 @@ class Co3Session:
         self.res_enc = torch.zeros(self.n_clients * B.RESULT_DTYPE.itemsize, dtype=torch.uint8, device=self.device)
         self.res_dec = torch.zeros(B.RESULT_DTYPE.itemsize, dtype=torch.uint8, device=self.device)
         self.res_fit = torch.zeros(B.RESULT_DTYPE.itemsize, dtype=torch.uint8, device=self.device)
+        self.res_model = torch.zeros(B.RESULT_DTYPE.itemsize, dtype=torch.uint8, device=self.device)
         self.avg = torch.empty(self.n_elem, dtype=torch.float32, device=self.device)
         self.hist = torch.zeros(max(1, self.n_seg) * 256, dtype=torch.int64, device=self.device)
 
@@ -92,6 +93,14 @@ class Co3Session:
         st = B.co3_code_build_device(self.hist, self.fmts, self.n_seg, self.codes, self.res_fit, stream)
         self._check(st, "co3_code_build_device")
 
+    def set_codes_from_model_device(self, stats: torch.Tensor, stream=None) -> None:
+        """One Huffman code per layer from the GenNorm model: `stats` is the float64[n_seg][4] tensor a fit_scales
+        call filled (beta and alpha per layer); weights and tables are built on the device (self.hist then holds
+        the model weights, not counts)."""
+        st = B.co3_model_weights(self.fmts, stats, self.n_seg, self.hist, self.res_model, stream)
+        self._check(st, "co3_model_weights")
+        self.set_codes_from_histogram_device(stream)
+
     def set_codes(self, codes: np.ndarray) -> None:
         self.codes_host = codes
         self.codes = B.to_device(codes, self.device)
@@ -129,6 +138,9 @@ class Co3Session:
 
     def fit_result(self) -> np.ndarray:
         return B.read_results(self.res_fit, 1)
+
+    def model_result(self) -> np.ndarray:
+        return B.read_results(self.res_model, 1)
 
     def decode_result(self) -> np.ndarray:
         return B.read_results(self.res_dec, 1)
