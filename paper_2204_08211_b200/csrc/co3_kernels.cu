@@ -1118,32 +1118,44 @@ __device__ __noinline__ uint32_t decode_long(const uint16_t* __restrict__ sub_ta
     return __ldg(sub_tab + ((ent & 0xffu) << kSubBits) + ((win >> (32 - CO3_MAX_CODE_LEN)) & ((1u << kSubBits) - 1u)));
 }
 
-// The 32 stream bits that start at bit `pos` of the chunk.
+// A thread's view of its chunk's bits: two consecutive payload words held in registers and replaced one at a
+// time as the position crosses a word boundary, so that a shared-memory load is issued only for the lanes that
+// need a new word (about one per 32 bits consumed instead of two per window).
 // kChecked: words beyond the chunk read as 0 (needed when the words are read in place from global memory);
 // otherwise the words sit in shared memory with kPaySlack readable words behind them.
 template <bool kChecked>
-__device__ __forceinline__ uint32_t window_at(const uint32_t* words, uint32_t nwords, uint32_t pos) {
-    const uint32_t i = pos >> 5;
-    uint32_t hi, lo;
-    if (kChecked) {
-        hi = i < nwords ? __ldg(words + i) : 0u;
-        lo = i + 1 < nwords ? __ldg(words + i + 1) : 0u;
-    } else {
-        hi = words[i];
-        lo = words[i + 1];
+struct BitWindow {
+    uint32_t hi, lo, wi;  // words wi and wi + 1 of the chunk
+    __device__ __forceinline__ uint32_t word(const uint32_t* words, uint32_t nwords, uint32_t i) const {
+        if (kChecked) return i < nwords ? __ldg(words + i) : 0u;
+        return words[i];
     }
-    return __funnelshift_l(lo, hi, pos);  // shift count taken modulo 32
-}
+    __device__ __forceinline__ void start(const uint32_t* words, uint32_t nwords, uint32_t pos) {
+        wi = pos >> 5;
+        hi = word(words, nwords, wi);
+        lo = word(words, nwords, wi + 1);
+    }
+    // The 32 stream bits that start at bit `pos`; pos lies in word wi or wi + 1 (it moved by at most 32 bits
+    // since the last call).
+    __device__ __forceinline__ uint32_t at(const uint32_t* words, uint32_t nwords, uint32_t pos) {
+        if ((pos >> 5) != wi) {
+            hi = lo;
+            ++wi;
+            lo = word(words, nwords, wi + 1);
+        }
+        return __funnelshift_l(lo, hi, pos);  // shift count taken modulo 32
+    }
+};
 
 // Decodes two symbols from the position `pos` on (a codeword has at most 16 bits, so one 32-bit window holds
 // both) and advances it.  Returns the two table entries: symbol in the low byte, 0xff = no codeword matched.
 // Both look-ups are done assuming short codewords and tested together; if either hit a second-level marker
 // the pair is redone step by step.
 template <bool kChecked, bool kSecond>
-__device__ __forceinline__ void decode_two(const uint32_t* words, uint32_t nwords, uint32_t& pos,
+__device__ __forceinline__ void decode_two(BitWindow<kChecked>& bw, const uint32_t* words, uint32_t nwords, uint32_t& pos,
                                            const uint16_t* __restrict__ s_lut, const uint16_t* __restrict__ sub_tab,
                                            uint32_t& e0, uint32_t& e1) {
-    const uint32_t win = window_at<kChecked>(words, nwords, pos);
+    const uint32_t win = bw.at(words, nwords, pos);
     e0 = s_lut[win >> (32 - kDecBits)];
     if (!kSecond) {
         if (e0 >= kDecLong) e0 = decode_long(sub_tab, e0, win);
@@ -1172,16 +1184,18 @@ template <bool kChecked, bool kWhole>
 __device__ __forceinline__ void decode_part(const uint32_t* words, uint32_t nwords, uint32_t& pos, uint32_t j0, uint32_t my,
                                             const uint16_t* __restrict__ s_lut, const uint16_t* __restrict__ sub_tab,
                                             uint32_t* pair_buf, uint32_t p, uint32_t s, uint32_t& marks) {
+    BitWindow<kChecked> bw;
+    bw.start(words, nwords, pos);
 #pragma unroll 2
     for (uint32_t jj = 0; jj < (uint32_t)kPhaseWords; ++jj) {
         const uint32_t j = j0 + jj;
         uint32_t w = 0;
         if (kWhole || j * 4 < my) {
             uint32_t e0, e1, e2 = 0, e3 = 0;
-            if (kWhole || j * 4 + 1 < my) decode_two<kChecked, true>(words, nwords, pos, s_lut, sub_tab, e0, e1);
-            else decode_two<kChecked, false>(words, nwords, pos, s_lut, sub_tab, e0, e1);
-            if (kWhole || j * 4 + 3 < my) decode_two<kChecked, true>(words, nwords, pos, s_lut, sub_tab, e2, e3);
-            else if (j * 4 + 2 < my) decode_two<kChecked, false>(words, nwords, pos, s_lut, sub_tab, e2, e3);
+            if (kWhole || j * 4 + 1 < my) decode_two<kChecked, true>(bw, words, nwords, pos, s_lut, sub_tab, e0, e1);
+            else decode_two<kChecked, false>(bw, words, nwords, pos, s_lut, sub_tab, e0, e1);
+            if (kWhole || j * 4 + 3 < my) decode_two<kChecked, true>(bw, words, nwords, pos, s_lut, sub_tab, e2, e3);
+            else if (j * 4 + 2 < my) decode_two<kChecked, false>(bw, words, nwords, pos, s_lut, sub_tab, e2, e3);
             w = __byte_perm(__byte_perm(e0, e1, 0x0040), __byte_perm(e2, e3, 0x0040), 0x5410);
             marks |= (~w - 0x01010101u) & w;  // bit 7 of a byte survives iff that byte of ~w is zero (symbol 0xff)
         }
