@@ -1692,6 +1692,8 @@ struct FitArgs {
     float beta0, dbeta;
     double* stats;  // nullable, [n_seg][4]
     double2* part;  // [n_clients][n_chunks_max]
+    double2* range_part;   // [n_seg][kFitRanges]
+    uint32_t* range_done;  // [n_seg], zero at launch
     co3_result* res;
     Ws ws;
 };
@@ -1762,15 +1764,22 @@ __device__ __forceinline__ double gennorm_kurtosis(double beta) {
     return exp(lgamma(5.0 / beta) + lgamma(1.0 / beta) - 2.0 * lgamma(3.0 / beta));
 }
 
+constexpr int kFitRanges = 64;  // a layer's partial sums are added up by this many blocks, each over a fixed share
+
 __global__ void __launch_bounds__(kThreads) fit_kernel(FitArgs a) {
     __shared__ double s_red[2][kThreads / 32];
+    __shared__ uint32_t s_last;
     const Ctrl* ctrl = a.ws.ctrl;
     if (ctrl->abort) return;
-    const uint32_t k = blockIdx.x, tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
+    const uint32_t k = blockIdx.x, r = blockIdx.y, tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
     const uint32_t c0 = a.ws.first_chunk[k], nck = a.ws.first_chunk[k + 1] - c0;
     const uint64_t items = (uint64_t)nck * a.n_clients;
+    // block (k, r) adds the r-th share of the layer's (client, chunk) sums, every thread its own items in order;
+    // the shares and the order in which they are combined do not depend on the GPU or on timing
+    const uint64_t per = (items + kFitRanges - 1) / kFitRanges;
+    const uint64_t i_lo = min(items, (uint64_t)r * per), i_hi = min(items, i_lo + per);
     double s2 = 0.0, s4 = 0.0;
-    for (uint64_t i = tid; i < items; i += kThreads) {
+    for (uint64_t i = i_lo + tid; i < i_hi; i += kThreads) {
         const uint32_t u = (uint32_t)(i / nck), c = (uint32_t)(i % nck);
         const double2 p = a.part[(size_t)u * a.ws.n_chunks_max + c0 + c];
         s2 = __dadd_rn(s2, p.x);
@@ -1783,10 +1792,23 @@ __global__ void __launch_bounds__(kThreads) fit_kernel(FitArgs a) {
     }
     if (lane == 0) { s_red[0][warp] = s2; s_red[1][warp] = s4; }
     __syncthreads();
-    if (warp != 0) return;
-    s2 = s4 = 0.0;
+    if (tid == 0) {
+        s2 = s4 = 0.0;
 #pragma unroll
-    for (int w = 0; w < kThreads / 32; ++w) { s2 = __dadd_rn(s2, s_red[0][w]); s4 = __dadd_rn(s4, s_red[1][w]); }
+        for (int w = 0; w < kThreads / 32; ++w) { s2 = __dadd_rn(s2, s_red[0][w]); s4 = __dadd_rn(s4, s_red[1][w]); }
+        a.range_part[(size_t)k * kFitRanges + r] = make_double2(s2, s4);
+        __threadfence();
+        s_last = atomicAdd(&a.range_done[k], 1u) == (uint32_t)kFitRanges - 1u ? 1u : 0u;
+    }
+    __syncthreads();
+    if (!s_last || warp != 0) return;  // the block that finishes a layer's sums last fits the layer
+    __threadfence();
+    s2 = s4 = 0.0;
+    for (int q = 0; q < kFitRanges; ++q) {
+        const double2 p = __ldcg(&a.range_part[(size_t)k * kFitRanges + q]);
+        s2 = __dadd_rn(s2, p.x);
+        s4 = __dadd_rn(s4, p.y);
+    }
 
     // warp 0, every lane with the same values
     const double N = (double)a.segs[k].n_elem * (double)a.n_clients;
@@ -2337,13 +2359,19 @@ int co3_fit_scale(const float* grad, const float* mem, float decay, co3_fmt* fmt
     const int rc = begin_call(L, ws, res, 1, st, nullptr, nullptr, segs, n_seg, n_elem, 1, 1);
     if (rc != CO3_OK) return rc;
     // the per-(chunk, client) partial sums take the place of the encoder's chunk slots (16 of 4096 bytes each)
+    // and behind them the per-layer range sums and completion counters of the fit
+    double2* part = reinterpret_cast<double2*>(ws.slots);
+    double2* range_part = part + (size_t)n_clients * L.n_chunks_max;
+    uint32_t* range_done = reinterpret_cast<uint32_t*>(range_part + (size_t)n_seg * kFitRanges);
+    static_assert(16 * (kFitRanges + 1) + 4 <= 4 * kSlotWords, "the fit's scratch fits in the slots of n_seg chunks");
+    CO3_CUDA(cudaMemsetAsync(range_done, 0, 4 * (size_t)n_seg, st));
     FitArgs fa{grad, mem, decay, client_stride_elems, n_clients, fmts, segs, n_seg, log_tab, seg_tab, n_tab, n_beta,
-               beta0, dbeta, stats_out, reinterpret_cast<double2*>(ws.slots), res, ws};
+               beta0, dbeta, stats_out, part, range_part, range_done, res, ws};
     if (L.n_chunks_max) {
         const dim3 grid((L.n_chunks_max + kMomChunks - 1) / kMomChunks, n_clients);
         CO3_LAUNCH(CO3_KERNEL_FIT, st, moments_kernel<<<grid, kThreads, 0, st>>>(fa));
     }
-    CO3_LAUNCH(CO3_KERNEL_FIT, st, fit_kernel<<<n_seg, kThreads, 0, st>>>(fa));
+    CO3_LAUNCH(CO3_KERNEL_FIT, st, fit_kernel<<<dim3(n_seg, kFitRanges), kThreads, 0, st>>>(fa));
     return CO3_OK;
 }
 
