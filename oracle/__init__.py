@@ -92,6 +92,8 @@ def lib():
         L.co3o_fit_scale.argtypes = [C.c_void_p, C.c_void_p, C.c_float, C.c_uint64, C.c_uint32, C.c_uint64,
                                      C.c_void_p, C.c_uint32, C.c_float, C.c_float,
                                      C.POINTER(C.c_float), C.POINTER(C.c_float), C.c_void_p]
+        L.co3o_error_magnitude.restype = None
+        L.co3o_error_magnitude.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_void_p]
         L.co3o_ps_update.restype = None
         L.co3o_ps_update.argtypes = [C.c_void_p, C.c_void_p, C.c_float, C.c_uint64]
         _lib = L
@@ -278,3 +280,13 @@ def fit_scale(g: np.ndarray, m, decay: float, log_tab: np.ndarray, beta0: float,
     st = lib().co3o_fit_scale(_ptr(g), _ptr(m), C.c_float(decay), g.shape[1], g.shape[0], g.shape[1], _ptr(tab), tab.size,
                               C.c_float(beta0), C.c_float(dbeta), C.byref(sc), C.byref(inv), _ptr(stats))
     return st, sc.value, inv.value, stats
+
+
+def error_magnitude(g: np.ndarray, m: np.ndarray) -> np.ndarray:
+    """[sum |g|, sum |m|] of one layer of one client (float64)."""
+    g = np.ascontiguousarray(g, dtype=np.float32)
+    m = np.ascontiguousarray(m, dtype=np.float32)
+    assert g.shape == m.shape and g.ndim == 1
+    out = np.zeros(2, dtype=np.float64)
+    lib().co3o_error_magnitude(_ptr(g), _ptr(m), g.size, _ptr(out))
+    return out

@@ -663,3 +663,19 @@ int co3o_fit_scale(const float *g, const float *m, float decay, uint64_t n, uint
     if (stats) { stats[0] = sigma; stats[1] = kurt; stats[2] = beta; stats[3] = alpha; }
     return CO3O_OK;
 }
+
+/*
+ * Error magnitude (Sec. VI, "Error magnitude"): the size of the memory term against the size of the gradient
+ * term, both as l1 norms, the quantity by which the memory decay gamma is judged.  One layer of one client:
+ * norms[0] = sum |g_i|, norms[1] = sum |m_i|, added in fp64 in element order.  A NaN anywhere gives NaN.
+ */
+void co3o_error_magnitude(const float *g, const float *m, uint64_t n, double *norms)
+{
+    double sg = 0.0, sm = 0.0;
+    for (uint64_t i = 0; i < n; ++i) {
+        sg += fabs((double)g[i]);
+        sm += fabs((double)m[i]);
+    }
+    norms[0] = sg;
+    norms[1] = sm;
+}
