@@ -207,6 +207,21 @@ int co3_fit_scale(const float* grad, const float* mem, float decay, co3_fmt* fmt
                   void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * Error magnitude (Sec. VI, "Error magnitude": the memory term m_t against the gradient term g_t, the figure the
+ * memory decay gamma is judged by): per client u and layer k
+ *     norms_out[(u * n_seg + k) * 2 + 0] = sum |g_i|,   norms_out[(u * n_seg + k) * 2 + 1] = sum |m_i|
+ * over the layer's elements, fp64 sums in a fixed order (independent of the launch shape and of timing).  A
+ * NaN in a layer gives NaN for that layer, an infinity gives infinity; nothing is reported as an error.
+ *   grad, mem [device]  as in co3_convert, both read only
+ *   norms_out [device]  double[n_clients][n_seg][2], fully overwritten
+ *   res [device]        one co3_result (CO3_ERR_INVALID_ARG if the segment table is inconsistent)
+ *   workspace           sized by co3_workspace_bytes with this n_clients (>= 1)
+ */
+int co3_error_magnitude(const float* grad, const float* mem, const co3_seg* segs, uint32_t n_seg, uint64_t n_elem,
+                        uint32_t n_clients, uint64_t client_stride_elems, double* norms_out, co3_result* res,
+                        void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * Huffman weights of every layer from its fitted model instead of from counted symbols (Sec. IV-A (ii): the code
  * is designed for the GenNorm distribution of the layer).  The weight of a symbol is floor(p * 2^30), p the
  * GenNorm(0, alpha, beta) mass of the inputs that the converter, with the layer's multiplier, sends to that
@@ -297,7 +312,7 @@ int co3_decode(const uint8_t* stream_in, size_t stream_bytes,
 #define CO3_KERNEL_COMPACT 4  /* payload compaction */
 #define CO3_KERNEL_CODE_BUILD 5 /* Huffman tables from weights on the device */
 #define CO3_KERNEL_DECODE 6   /* decode + cross-client accumulate */
-#define CO3_KERNEL_FIT 7      /* moments, multiplier fit, model weights */
+#define CO3_KERNEL_FIT 7      /* moments, multiplier fit, model weights, error magnitude */
 #define CO3_KERNEL_COUNT 8
 int co3_profile_enable(int on);
 int co3_profile_read(double* total_ms /* [host] */, uint32_t* launches /* [host] */);

@@ -47,6 +47,7 @@ def _load():
     L.co3_code_build.argtypes = [vp, vp, vp]
     L.co3_code_build_device.argtypes = [vp, vp, u32, vp, vp, vp]
     L.co3_fit_scale.argtypes = [vp, vp, f32, vp, vp, u32, u64, u32, u64, vp, vp, u32, u32, f32, f32, vp, vp, vp, sz, vp]
+    L.co3_error_magnitude.argtypes = [vp, vp, vp, u32, u64, u32, u64, vp, vp, vp, sz, vp]
     L.co3_model_weights.argtypes = [vp, vp, u32, vp, vp, vp]
     L.co3_encode.argtypes = [vp, vp, f32, vp, vp, vp, u32, u64, u32, u64, vp, sz, u32, vp, sz, vp, vp]
     L.co3_encode_symbols.argtypes = [vp, vp, vp, u32, u64, u32, u64, vp, sz, u32, vp, sz, vp, vp]
@@ -55,7 +56,7 @@ def _load():
     L.co3_decode.argtypes = [vp, sz, vp, vp, vp, u32, u64, u32, vp, vp, vp, sz, vp, vp]
     L.co3_profile_enable.argtypes = [C.c_int]
     L.co3_profile_read.argtypes = [vp, vp]
-    for name in ("co3_model_weights", "co3_fit_scale", "co3_profile_enable", "co3_profile_read", "co3_convert_static", "co3_workspace_bytes", "co3_stream_capacity_bytes", "co3_convert", "co3_code_build", "co3_code_build_device", "co3_encode",
+    for name in ("co3_error_magnitude", "co3_model_weights", "co3_fit_scale", "co3_profile_enable", "co3_profile_read", "co3_convert_static", "co3_workspace_bytes", "co3_stream_capacity_bytes", "co3_convert", "co3_code_build", "co3_code_build_device", "co3_encode",
                  "co3_encode_symbols", "co3_decode_aggregate", "co3_decode_aggregate_update", "co3_decode"):
         getattr(L, name).restype = C.c_int
     _lib = L
@@ -176,6 +177,14 @@ def co3_fit_scale(grad, mem, decay, fmts, segs, n_seg, n_elem, n_clients, client
                                  n_clients, client_stride_elems, _dev(log_tab), _dev(seg_tab, True), n_tab, n_beta,
                                  float(beta0), float(dbeta), _dev(stats_out, True), _dev(res), _dev(workspace),
                                  workspace.numel() * workspace.element_size(), _stream(stream))
+
+
+def co3_error_magnitude(grad, mem, segs, n_seg, n_elem, n_clients, client_stride_elems, norms_out, res, workspace,
+                        stream=None) -> int:
+    """norms_out float64[n_clients * n_seg * 2]: l1 norms of gradient and memory per client and layer."""
+    return _load().co3_error_magnitude(_dev(grad), _dev(mem), _dev(segs), n_seg, n_elem, n_clients, client_stride_elems,
+                                       _dev(norms_out), _dev(res), _dev(workspace),
+                                       workspace.numel() * workspace.element_size(), _stream(stream))
 
 
 def co3_model_weights(fmts, stats, n_seg, weights_out, res, stream=None) -> int:

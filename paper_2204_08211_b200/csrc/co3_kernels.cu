@@ -1707,6 +1707,8 @@ __device__ __forceinline__ void moments_add(float g, float m, float decay, bool 
     s4 = __dadd_rn(s4, __dmul_rn(x2, x2));
 }
 
+// kNorms: the two sums are |g| and |m| (error magnitude, Sec. VI) instead of v^2 and v^4.
+template <bool kNorms>
 __global__ void __launch_bounds__(kThreads) moments_kernel(FitArgs a) {
     __shared__ double s_red[kMomChunks][2][kThreads / 32];
     const Ctrl* ctrl = a.ws.ctrl;
@@ -1743,7 +1745,14 @@ __global__ void __launch_bounds__(kThreads) moments_kernel(FitArgs a) {
         double s2 = 0.0, s4 = 0.0;
 #pragma unroll
         for (int e = 0; e < 8; ++e)
-            if ((uint32_t)e < nv[j]) moments_add(g[j][e], has_m ? m[j][e] : 0.0f, a.decay, has_m, s2, s4);
+            if ((uint32_t)e < nv[j]) {
+                if (kNorms) {
+                    s2 = __dadd_rn(s2, fabs((double)g[j][e]));
+                    s4 = __dadd_rn(s4, fabs((double)m[j][e]));
+                } else {
+                    moments_add(g[j][e], has_m ? m[j][e] : 0.0f, a.decay, has_m, s2, s4);
+                }
+            }
 #pragma unroll
         for (int w = 16; w > 0; w >>= 1) {
             s2 = __dadd_rn(s2, __shfl_xor_sync(0xffffffffu, s2, w));
@@ -1865,6 +1874,58 @@ __global__ void __launch_bounds__(kThreads) fit_kernel(FitArgs a) {
         double* st = a.stats + 4 * (size_t)k;
         st[0] = sigma; st[1] = kurt; st[2] = beta; st[3] = alpha;
     }
+}
+
+// Error magnitude (Sec. VI): per client and layer the l1 norms of the gradient and of the memory, from the
+// per-chunk sums of moments_kernel<true>.  Block (k, r, u) adds the r-th share of the chunk sums of layer k of
+// client u; the block that finishes a (layer, client) last adds the shares in order and writes the result.
+struct MagArgs {
+    const double2* part;  // [n_clients][n_chunks_max]
+    double2* range_part;  // [n_clients][n_seg][kFitRanges]
+    uint32_t* range_done; // [n_clients][n_seg], zero at launch
+    double* out;          // [n_clients][n_seg][2]
+    uint32_t n_seg;
+    Ws ws;
+};
+
+__global__ void __launch_bounds__(kThreads) magnitude_kernel(MagArgs a) {
+    __shared__ double s_red[2][kThreads / 32];
+    if (a.ws.ctrl->abort) return;
+    const uint32_t k = blockIdx.x, r = blockIdx.y, u = blockIdx.z, tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
+    const uint32_t c0 = a.ws.first_chunk[k], nck = a.ws.first_chunk[k + 1] - c0;
+    const uint32_t per = (nck + kFitRanges - 1) / kFitRanges;
+    const uint32_t i_lo = min(nck, r * per), i_hi = min(nck, i_lo + per);
+    const double2* part = a.part + (size_t)u * a.ws.n_chunks_max + c0;
+    double sg = 0.0, sm = 0.0;
+    for (uint32_t i = i_lo + tid; i < i_hi; i += kThreads) {
+        const double2 p = part[i];
+        sg = __dadd_rn(sg, p.x);
+        sm = __dadd_rn(sm, p.y);
+    }
+#pragma unroll
+    for (int w = 16; w > 0; w >>= 1) {
+        sg = __dadd_rn(sg, __shfl_xor_sync(0xffffffffu, sg, w));
+        sm = __dadd_rn(sm, __shfl_xor_sync(0xffffffffu, sm, w));
+    }
+    if (lane == 0) { s_red[0][warp] = sg; s_red[1][warp] = sm; }
+    __syncthreads();
+    if (tid != 0) return;
+    sg = sm = 0.0;
+#pragma unroll
+    for (int w = 0; w < kThreads / 32; ++w) { sg = __dadd_rn(sg, s_red[0][w]); sm = __dadd_rn(sm, s_red[1][w]); }
+    const size_t cell = (size_t)u * a.n_seg + k;
+    a.range_part[cell * kFitRanges + r] = make_double2(sg, sm);
+    __threadfence();
+    if (atomicAdd(&a.range_done[cell], 1u) != (uint32_t)kFitRanges - 1u) return;
+    __threadfence();
+    sg = sm = 0.0;
+    for (int q = 0; q < kFitRanges; ++q) {
+        const double2 p = __ldcg(&a.range_part[cell * kFitRanges + q]);
+        sg = __dadd_rn(sg, p.x);
+        sm = __dadd_rn(sm, p.y);
+    }
+    a.out[2 * cell] = sg;
+    a.out[2 * cell + 1] = sm;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -2369,9 +2430,45 @@ int co3_fit_scale(const float* grad, const float* mem, float decay, co3_fmt* fmt
                beta0, dbeta, stats_out, part, range_part, range_done, res, ws};
     if (L.n_chunks_max) {
         const dim3 grid((L.n_chunks_max + kMomChunks - 1) / kMomChunks, n_clients);
-        CO3_LAUNCH(CO3_KERNEL_FIT, st, moments_kernel<<<grid, kThreads, 0, st>>>(fa));
+        CO3_LAUNCH(CO3_KERNEL_FIT, st, moments_kernel<false><<<grid, kThreads, 0, st>>>(fa));
     }
     CO3_LAUNCH(CO3_KERNEL_FIT, st, fit_kernel<<<dim3(n_seg, kFitRanges), kThreads, 0, st>>>(fa));
+    return CO3_OK;
+}
+
+int co3_error_magnitude(const float* grad, const float* mem, const co3_seg* segs, uint32_t n_seg, uint64_t n_elem,
+                        uint32_t n_clients, uint64_t client_stride_elems, double* norms_out, co3_result* res,
+                        void* workspace, size_t workspace_bytes, void* stream) {
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (!grad || !mem || !segs || !norms_out || !res || !workspace || n_seg == 0 || n_clients == 0 || n_clients > 65535u)
+        return CO3_ERR_INVALID_ARG;
+    if (!aligned(grad, 16) || !aligned(mem, 16) || !aligned(workspace, 256) || !aligned(res, 8) || !aligned(norms_out, 8))
+        return CO3_ERR_INVALID_ARG;
+    if (n_clients > 1 && client_stride_elems < n_elem) return CO3_ERR_INVALID_ARG;
+    WsLayout L;
+    if (!ws_layout(n_elem, n_seg, n_clients, &L)) return CO3_ERR_INVALID_ARG;
+    if (workspace_bytes < L.total) return CO3_ERR_CAPACITY;
+    const Ws ws = ws_pointers(workspace, L);
+    const int rc = begin_call(L, ws, res, 1, st, nullptr, nullptr, segs, n_seg, n_elem, 1, 1);
+    if (rc != CO3_OK) return rc;
+    // scratch inside the encoder's chunk slots: 16 bytes per (chunk, client), then 16 * kFitRanges + 4 per (layer, client)
+    double2* part = reinterpret_cast<double2*>(ws.slots);
+    double2* range_part = part + (size_t)n_clients * L.n_chunks_max;
+    uint32_t* range_done = reinterpret_cast<uint32_t*>(range_part + (size_t)n_seg * n_clients * kFitRanges);
+    CO3_CUDA(cudaMemsetAsync(range_done, 0, 4 * (size_t)n_seg * n_clients, st));
+    FitArgs fa{};
+    fa.grad = grad;
+    fa.mem = mem;
+    fa.client_stride = client_stride_elems;
+    fa.n_clients = n_clients;
+    fa.part = part;
+    fa.ws = ws;
+    if (L.n_chunks_max) {
+        const dim3 grid((L.n_chunks_max + kMomChunks - 1) / kMomChunks, n_clients);
+        CO3_LAUNCH(CO3_KERNEL_FIT, st, moments_kernel<true><<<grid, kThreads, 0, st>>>(fa));
+    }
+    MagArgs ma{part, range_part, range_done, norms_out, n_seg, ws};
+    CO3_LAUNCH(CO3_KERNEL_FIT, st, magnitude_kernel<<<dim3(n_seg, kFitRanges, n_clients), kThreads, 0, st>>>(ma));
     return CO3_OK;
 }
 

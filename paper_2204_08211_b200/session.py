@@ -58,6 +58,14 @@ class Co3Session:
                              stats_out, self.res_fit, self.workspace, stream)
         self._check(st, "co3_fit_scale")
 
+    def error_magnitude(self, grads: torch.Tensor, mems: torch.Tensor, stream=None) -> torch.Tensor:
+        """float64[n_clients][n_seg][2] on the device: l1 norm of each layer's gradient and memory per client."""
+        out = torch.empty((self.n_clients, self.n_seg, 2), dtype=torch.float64, device=self.device)
+        st = B.co3_error_magnitude(grads, mems, self.segs, self.n_seg, self.n_elem, self.n_clients, self.stride, out,
+                                   self.res_fit, self.workspace, stream)
+        self._check(st, "co3_error_magnitude")
+        return out
+
     def fmts_from_device(self) -> np.ndarray:
         raw = self.fmts.cpu().numpy().tobytes()[:self.n_seg * B.FMT_DTYPE.itemsize]
         self.fmts_host = np.frombuffer(raw, dtype=B.FMT_DTYPE).copy()
