@@ -150,20 +150,22 @@ __device__ __forceinline__ float convert_one(float g, float m, float decay, cons
 // The same update without branches, for formats with M >= 1 that keep the sub-normal levels.
 // Rounding by one fp32 addition: with ae the (clamped) exponent of |t|, |t| + 2^(ae + 23 - M) is rounded by
 // the adder to a multiple of the format's step in that binade, ties to the even multiple, which has the
-// even code when M >= 1.  Saturating and non-finite inputs all land on the largest code (NaN and Inf compare
-// above the largest level), so the caller only watches for that code (code_max) and, when it shows up in a
-// group, repeats the group with convert_one, which tells those cases apart and counts them.
+// even code when M >= 1.  Inputs beyond the largest level and non-finite ones are clamped to it here and
+// reported in `beyond` (a NaN fails the comparison too); the caller repeats a group that holds one with
+// convert_one, which tells those cases apart and counts them.  Inputs that land on the largest level from
+// inside the range (common in the narrow formats) need no second look.
 __device__ __forceinline__ float convert_fast(float g, float m, float decay, const FmtDev& f, uint32_t& sym,
-                                              uint32_t& code_max) {
+                                              bool& beyond) {
     const float v = __fmaf_rn(decay, m, g);
     const float t = __fmul_rn(v, f.scale);
-    const float at = fminf(fabsf(t), __uint_as_float(f.top_bits));  // NaN -> largest level
+    const float top = __uint_as_float(f.top_bits);
+    beyond |= !(fabsf(t) <= top);
+    const float at = fminf(fabsf(t), top);  // NaN -> largest level
     const uint32_t ac = __float_as_uint(at);
     const uint32_t ae = max(ac & 0x7f800000u, f.min_normal_bits);
     const uint32_t mg = ae + (f.drop << 23);
     const float s = __fadd_rn(at, __uint_as_float(mg));
     const uint32_t code = ((ae - f.min_normal_bits) >> f.drop) + (__float_as_uint(s) - mg);
-    code_max = max(code_max, code);
     const float qmag = __fsub_rn(s, __uint_as_float(mg));
     const uint32_t sgn = code ? (__float_as_uint(t) & 0x80000000u) : 0u;
     sym = code | (sgn >> f.sign_shift);

@@ -354,10 +354,10 @@ __device__ __forceinline__ void convert8(const float (&g)[8], const float (&m)[8
                                          uint32_t& n_nf) {
     bool redo = true;
     if (kWhole && f.fast) {
-        uint32_t code_max = 0;
+        bool beyond = false;
 #pragma unroll
-        for (int j = 0; j < 8; ++j) mo[j] = convert_fast(g[j], m[j], decay, f, s[j], code_max);
-        redo = code_max >= f.max_code;  // the largest level: maybe a saturating or non-finite input
+        for (int j = 0; j < 8; ++j) mo[j] = convert_fast(g[j], m[j], decay, f, s[j], beyond);
+        redo = beyond;  // a saturating or non-finite input
     }
     if (redo) {  // generic formats, ragged groups, and groups that hold a saturating or non-finite input
 #pragma unroll
