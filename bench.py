@@ -28,7 +28,7 @@ METRIC = "co3_encode_decode_aggregate_throughput"
 UNIT = "gradient elements/s"
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch, from the ncu captures summarised under profiles/
 # (config 2, 10 clients).  Only meaningful for that workload and for the kernels as they were captured.
-NCU_TRAFFIC_BYTES = {"pack": 1396.8e6, "decode": 116.4e6, "convert": 1406.0e6}
+NCU_TRAFFIC_BYTES = {"pack": 1397.6e6, "decode": 116.4e6, "convert": 1405.6e6}
 RANK_SEED_STRIDE = 100_000   # ranks draw their synthetic clients from disjoint seed ranges
 
 
