@@ -130,8 +130,9 @@ def test_layers_without_a_fit_are_reported_and_left_alone():
 
 
 def test_fitted_formats_drive_the_conversion():
-    """The formats the fit leaves on the device are the ones the next co3_convert uses: symbols and memories are
-    bit-identical to the oracle's conversion with the same (device-fitted) multipliers."""
+    """Fit then convert, each side on its own: the device converts with the formats its fit left on the device, the
+    oracle with the multipliers of the oracle's fit.  On these layers the two fits give identical fp32 multipliers
+    (asserted), so symbols and memories must be bit-identical."""
     sizes = [36864, 2500, 64]
     beta, alpha = [0.7, 1.1, 1.5], [2e-3, 4e-4, 1e-2]
     g = np.concatenate([gennorm(n, beta[k], alpha[k], 50 + k).numpy() for k, n in enumerate(sizes)])[None, :]
@@ -146,8 +147,11 @@ def test_fitted_formats_drive_the_conversion():
     fm = sess.fmts_from_device()
     offs = np.concatenate([[0], np.cumsum(sizes)])
     for k in range(3):
+        gk = np.ascontiguousarray(g[0, offs[k]:offs[k + 1]])
+        st, sc, inv, _ = oracle.fit_scale(gk, np.zeros_like(gk), 0.9, tab[0], beta0, dbeta)
+        assert st == oracle.OK and fm["scale"][k] == np.float32(sc) and fm["inv_scale"][k] == np.float32(inv)
         m = np.zeros(sizes[k], dtype=np.float32)
-        r = oracle.convert(g[0, offs[k]:offs[k + 1]], m, 0.9, oracle.Fmt(4, 3, 0, float(fm["scale"][k]), float(fm["inv_scale"][k])))
+        r = oracle.convert(gk, m, 0.9, oracle.Fmt(4, 3, 0, sc, inv))
         assert np.array_equal(sym[offs[k]:offs[k + 1]].cpu().numpy(), r["sym"])
         assert np.array_equal(sess.client_view(mems, 0)[offs[k]:offs[k + 1]].cpu().numpy().view(np.uint32), m.view(np.uint32))
         assert r["n_saturated"] < 0.001 * sizes[k]      # the fitted multiplier keeps the layer inside the format
