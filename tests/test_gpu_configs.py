@@ -200,7 +200,10 @@ def test_config2_full_size_sampled_chunks():
 
     C = co3.CHUNK_SYMS
     ofmts = [oracle.Fmt(E, M, 0, s, inv) for (E, M, _, s, inv) in fmts]
-    ocodes = [oracle.make_code(sess.codes_host[k]["len"], sess.codes_host[k]["bits"]) for k in range(len(sizes))]
+    ocodes = [oracle.code_build(hist[k], ofmts[k]) for k in range(len(sizes))]     # the oracle's own tables ...
+    for k in range(len(sizes)):                                                    # ... which the library's equal
+        ln, bits = oracle.code_arrays(ocodes[k])
+        assert np.array_equal(sess.codes_host[k]["len"], ln) and np.array_equal(sess.codes_host[k]["bits"].astype(np.uint32), bits)
     seg_first = np.concatenate([[0], np.cumsum([(n + C - 1) // C for n in sizes])])
     seg_off = np.concatenate([[0], np.cumsum(sizes)])
     n_chunks = int(seg_first[-1])
@@ -245,3 +248,43 @@ def test_config2_full_size_sampled_chunks():
             ghat_sum = gh.copy() if ghat_sum is None else (ghat_sum + gh).astype(np.float32)
         want_avg = (ghat_sum / np.float32(clients)).astype(np.float32)
         assert same_bits(avg[lo:lo + cnt].cpu().numpy(), want_avg)
+
+
+def test_config2_full_size_fit_and_error_magnitude():
+    """The set-up and diagnostic calls at the benchmarked size (10 clients x 11,181,642 elements in 62 layers, live
+    memories after one round): every layer's fitted multiplier within one fp32 ULP of the oracle's (identical on
+    nearly all), its statistics to 1e-10, and the l1 norms of every (client, layer) to 1e-12."""
+    import bench
+    from co3_inputs import scale_log_table
+    cfg, sizes, fmts, clients = bench.workload(2)
+    sess = Co3Session(sizes, fmts, clients, cfg["decay"], "cuda")
+    g0 = bench.make_grads(cfg, sizes, clients, sess.stride, 0, "cuda")
+    g1 = bench.make_grads(cfg, sizes, clients, sess.stride, 1, "cuda")
+    mems = sess.new_client_buffer()
+    sess.histogram(g0, mems, to_host=False)                     # one round: the memories are live
+    norms = sess.error_magnitude(g1, mems).cpu().numpy()
+    tab, beta0, dbeta = scale_log_table([tuple(cfg["fmt"])])
+    stats = torch.zeros((len(sizes), 4), dtype=torch.float64, device="cuda")
+    sess.fit_scales(g1, mems, torch.from_numpy(tab).cuda(), beta0, dbeta, stats_out=stats)
+    torch.cuda.synchronize()
+    assert sess.fit_result()[0]["status"] == co3.OK
+    fm = sess.fmts_from_device()
+    st_dev = stats.cpu().numpy()
+    g_host = g1.cpu().numpy().reshape(clients, sess.stride)
+    m_host = mems.cpu().numpy().reshape(clients, sess.stride)
+    seg_off = np.concatenate([[0], np.cumsum(sizes)])
+    exact = 0
+    for k in range(len(sizes)):
+        gk = np.ascontiguousarray(g_host[:, seg_off[k]:seg_off[k + 1]])
+        mk = np.ascontiguousarray(m_host[:, seg_off[k]:seg_off[k + 1]])
+        st, sc, inv, ost = oracle.fit_scale(gk, mk, cfg["decay"], tab[0], beta0, dbeta)
+        assert st == oracle.OK
+        d = abs(int(np.float32(fm["scale"][k]).view(np.int32)) - int(np.float32(sc).view(np.int32)))
+        assert d <= 1, "layer %d" % k
+        exact += d == 0
+        assert fm["inv_scale"][k] == np.float32(1.0) / np.float32(fm["scale"][k])
+        assert np.allclose(st_dev[k], ost, rtol=1e-10, atol=0.0)
+        for u in (0, clients - 1):
+            want = oracle.error_magnitude(gk[u], mk[u])
+            assert np.allclose(norms[u, k], want, rtol=1e-12, atol=0.0)
+    assert exact >= len(sizes) - 2
