@@ -208,7 +208,7 @@ int co3_fit_scale(const float* grad, const float* mem, float decay, co3_fmt* fmt
 
 /*
  * Error magnitude (Sec. VI, "Error magnitude": the memory term m_t against the gradient term g_t, the figure the
- * memory decay gamma is judged by): per client u and layer k
+ * memory decay gamma is chosen by): per client u and layer k
  *     norms_out[(u * n_seg + k) * 2 + 0] = sum |g_i|,   norms_out[(u * n_seg + k) * 2 + 1] = sum |m_i|
  * over the layer's elements, fp64 sums in a fixed order (independent of the launch shape and of timing).  A
  * NaN in a layer gives NaN for that layer, an infinity gives infinity; nothing is reported as an error.

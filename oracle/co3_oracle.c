@@ -666,7 +666,7 @@ int co3o_fit_scale(const float *g, const float *m, float decay, uint64_t n, uint
 
 /*
  * Error magnitude (Sec. VI, "Error magnitude"): the size of the memory term against the size of the gradient
- * term, both as l1 norms, the quantity by which the memory decay gamma is judged.  One layer of one client:
+ * term, both as l1 norms, the quantity by which the memory decay gamma is chosen.  One layer of one client:
  * norms[0] = sum |g_i|, norms[1] = sum |m_i|, added in fp64 in element order.  A NaN anywhere gives NaN.
  */
 void co3o_error_magnitude(const float *g, const float *m, uint64_t n, double *norms)
