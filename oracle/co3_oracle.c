@@ -314,7 +314,7 @@ int co3o_code_build(const uint64_t weights[256], const co3o_fmt *f, co3o_code *o
 
 /* ------------------------------------------------------------------------------------------
  * Container (the paper only says the codewords form a binary string b of length r; the layout
- * below is this build's, chosen so that a decoder can start at many places at once).
+ * below is this implementation's, chosen so that a decoder can start at many places at once).
  * All fields little-endian.
  *   header, 64 bytes: u32 magic 'CO3S', u32 version 1, u32 n_seg, u32 chunk_syms C,
  *       u32 sub_syms S, u32 0, u64 n_elem, u64 n_chunks, u64 payload_words, u64 payload_bits,
