@@ -171,3 +171,27 @@ def test_argument_checks():
     assert call(n_clients=0) == co3.ERR_INVALID_ARG
     assert call(workspace=sess.workspace[:4096]) == co3.ERR_CAPACITY
     torch.cuda.synchronize()
+
+
+def test_inconsistent_segment_table_is_refused_on_the_device():
+    """A segment table that does not tile the vector is found by the layout check on the device: the status says
+    so, no format is written, and the error-magnitude call on the same table reports it too (output untouched)."""
+    sess = Co3Session([4096, 1000], [fmt_tuple(4, 3, 2.0)] * 2, 1, 0.9, "cuda")
+    bad = B.make_segs([4096, 1000])
+    bad[1]["elem_off"] = 4000                       # overlaps the first layer
+    segs = B.to_device(bad)
+    tab, beta0, dbeta = scale_log_table([(4, 3)])
+    g = sess.new_client_buffer()
+    g.normal_(0.0, 1e-3, generator=torch.Generator(device="cuda").manual_seed(1))
+    st = co3.co3_fit_scale(g, None, 0.9, sess.fmts, segs, 2, sess.n_elem, 1, sess.stride, torch.from_numpy(tab).cuda(),
+                           None, 1, tab.shape[1], beta0, dbeta, None, sess.res_fit, sess.workspace)
+    assert st == co3.OK
+    torch.cuda.synchronize()
+    assert sess.fit_result()[0]["status"] == co3.ERR_INVALID_ARG
+    fm = sess.fmts_from_device()
+    assert (fm["scale"] == np.float32(2.0)).all() and (fm["inv_scale"] == np.float32(0.5)).all()
+    norms = torch.full((1, 2, 2), -7.0, dtype=torch.float64, device="cuda")
+    st = co3.co3_error_magnitude(g, g, segs, 2, sess.n_elem, 1, sess.stride, norms, sess.res_fit, sess.workspace)
+    assert st == co3.OK
+    torch.cuda.synchronize()
+    assert sess.fit_result()[0]["status"] == co3.ERR_INVALID_ARG and (norms == -7.0).all()
