@@ -23,13 +23,16 @@
  *     Everything that depends on device data (descriptor contents, a symbol without codeword, a
  *     payload that does not fit, a corrupt stream) is reported in the device-side co3_result,
  *     valid once the stream has been synchronised.  After a device-side error the outputs of
- *     that client are undefined but nothing is written outside the buffers given.
+ *     that client are undefined but nothing is written outside the buffers given.  CO3_ERR_CUDA
+ *     in a co3_result (a copy inside a kernel never completed) is reported for every client of
+ *     the call: the kernels stop within about one time-out, and the error memories and streams
+ *     of all clients of that call are undefined.
  *   - A gradient of one client is a flat fp32 vector of n_elem elements, cut into n_seg segments
  *     (layers) that are contiguous and in order: segs[0].elem_off == 0,
  *     segs[k+1].elem_off == segs[k].elem_off + segs[k].n_elem, sum of n_elem == n_elem.
- *     Segment k uses fmts[k] and codes[k] for every client ("a different code in each layer,
- *     the same code across users", Sec. IV-A (ii)).  Clients are batched: client u's vector
- *     starts client_stride_elems * u elements after the base pointer.
+ *     Segment k uses fmts[k] and codes[k] for every client: one code per layer, shared by
+ *     all users (Sec. IV-A (ii)).  Clients are batched: client u's vector starts
+ *     client_stride_elems * u elements after the base pointer.
  *   - fp32 buffers and streams must be 16-byte aligned.
  */
 #ifndef CO3_H_
@@ -237,7 +240,11 @@ int co3_model_weights(const co3_fmt* fmts, const double* stats, uint32_t n_seg, 
                       co3_result* res, void* stream);
 
 /*
- * Client uplink for n_clients clients: correct + convert + encode + memory update, codes given.
+ * Client uplink for n_clients clients, the three per-user updates of Algorithm 1 in one call, codes given:
+ *     v = g + decay * m,  ghat = Q_fp(v)   (Sec. IV-A (iii), (i));   b = h_Hf(ghat): the codewords of the symbols
+ *     of ghat concatenated element by element (Sec. II-B (iii), Sec. IV-A (ii));   m <- v - ghat.
+ *   grad, mem, decay, fmts, segs, strides: as in co3_convert; mem is updated in place
+ *   codes [device]        n_seg prefix-code tables; a symbol that occurs must have a codeword
  *   streams_out [device]  client u's container starts at streams_out + u * stream_capacity
  *                         (stream_capacity a multiple of 16); layout below
  *   res [device] co3_result[n_clients]
@@ -257,8 +264,10 @@ int co3_encode(const float* grad, float* mem, float decay,
                uint8_t* streams_out, size_t stream_capacity, uint32_t chunk_syms,
                void* workspace, size_t workspace_bytes, co3_result* res, void* stream);
 
-/* Same container from symbols already converted (the flow in which the code is fitted to this
- * round's histogram between conversion and coding).  sym [device]: one byte per element. */
+/* The coding step alone, b = h_Hf(ghat) (Sec. II-B (iii), Sec. IV-A (ii)): the same container from symbols that
+ * co3_convert produced, for the flow in which the code is fitted to this round's symbol statistics between
+ * conversion and coding (Sec. IV-A (ii): the code is designed for the distribution of the source).
+ * sym [device]: one byte per element, strides as for grad. */
 int co3_encode_symbols(const uint8_t* sym, const co3_code* codes, const co3_seg* segs,
                        uint32_t n_seg, uint64_t n_elem, uint32_t n_clients, uint64_t client_stride_elems,
                        uint8_t* streams_out, size_t stream_capacity, uint32_t chunk_syms,

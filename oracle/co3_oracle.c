@@ -118,7 +118,7 @@ float co3o_symbol_value(const co3o_fmt *f, uint32_t sym)
 }
 
 /* ------------------------------------------------------------------------------------------
- * Converter Q_fp ("closest value of the form ...", Sec. V-B) for one scaled value t.
+ * Converter Q_fp for one scaled value t: rounds to the nearest level of the set in Sec. V-B.
  * The valid magnitude codes are enumerated in increasing order (their levels increase with
  * the code) and the two levels around |t| are compared against their midpoint.  Ties go to
  * the even code (IEEE default rounding, which the format section cites); when both codes are

@@ -259,6 +259,12 @@ __global__ void __launch_bounds__(kThreads) prepare_kernel(PrepArgs a) {
         }
         __syncthreads();
         if (s_kraft > (1u << CO3_MAX_CODE_LEN)) code_ok = false;  // over-subscribed: cannot be prefix-free
+        if (code_ok && len) {  // no other codeword may start with this one (equal codewords included)
+            for (uint32_t j = 0; j < 256; ++j) {
+                const uint32_t lj = s_code[j] & 0xffu, bj = s_code[j] >> 8;
+                if (j != tid && lj >= len && (bj >> (lj - len)) == bits) code_ok = false;
+            }
+        }
         code_ok = __syncthreads_and(code_ok);
         if (code_ok && a.want_dec) {
             // short codewords fill every table entry they prefix: one warp per symbol, lanes over the span
@@ -403,14 +409,17 @@ struct FeedCursor {
     }
 };
 
-struct Feed {
+struct alignas(16) Feed {
     float g[2][kC];
     float m[2][kC];
     uint64_t bar[2];
     FeedItem item[2];
     FmtDev fmt[2];    // converter constants of the item in each slot
     FeedCursor cur;   // thread 0's place in the item sequence (kept here to spare every thread the registers)
+    uint32_t fail;    // set by any thread whose wait for a copy gave up; the block leaves its item loop at the next barrier
 };
+
+static_assert(sizeof(Feed) % 16 == 0, "what follows a Feed in shared memory is accessed 16 bytes at a time");
 
 struct FeedArgs {
     const float* grad;
@@ -467,7 +476,10 @@ __device__ __forceinline__ bool feed_read(Feed& fd, const FeedArgs& fa, const Fe
         const uint32_t slot = (uint32_t)k & 1u;
         const bool ok = mbar_wait(&fd.bar[slot], (parity >> slot) & 1u);
         parity ^= 1u << slot;
-        if (!ok) return false;
+        if (!ok) {
+            fd.fail = 1u;
+            return false;
+        }
         const float4* gs = reinterpret_cast<const float4*>(&fd.g[slot][i0]);
         const float4* ms = reinterpret_cast<const float4*>(&fd.m[slot][i0]);
         const float4 a = gs[0], b = gs[1], c = ms[0], d = ms[1];
@@ -478,6 +490,13 @@ __device__ __forceinline__ bool feed_read(Feed& fd, const FeedArgs& fa, const Fe
         load8_any(fa.mem + it.base + i0, nv, m);
     }
     return true;
+}
+
+// A wait gave up and the block has left its item loop after item k: thread 0 still waits (bounded again) for the
+// copies it had started for item k + 1, so that nothing is in flight into this block's shared memory when it exits.
+__device__ __forceinline__ void feed_drain(Feed& fd, uint32_t k, uint32_t parity) {
+    const uint32_t slot = (k + 1u) & 1u;
+    if (threadIdx.x == 0 && fd.item[slot].valid && fd.item[slot].tma) mbar_wait(&fd.bar[slot], (parity >> slot) & 1u);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -514,6 +533,7 @@ __global__ void __launch_bounds__(kThreads, 3) convert_kernel(ConvertArgs a) {
     if (tid == 0) {
         mbar_init(&fd.bar[0], 1);
         mbar_init(&fd.bar[1], 1);
+        fd.fail = 0u;
         fd.cur.init(n_chunks);
         next = a.ws.chunk_desc[fd.cur.chunk];
         feed_issue(fd, fa, a.ws, n_chunks, 0, next, true);
@@ -551,16 +571,19 @@ __global__ void __launch_bounds__(kThreads, 3) convert_kernel(ConvertArgs a) {
         const uint32_t nv = it.d.cnt > i0 ? min(8u, it.d.cnt - i0) : 0u;
         float g[8], m[8], mo[8];
         uint32_t s[8];
-        if (!feed_read(fd, fa, it, k, i0, nv, parity, g, m)) hw_fail = true;
+        // a copy that never arrived (never expected): this thread writes nothing for the item, the block stops
+        const bool ok = feed_read(fd, fa, it, k, i0, nv, parity, g, m);
         const uint64_t e = it.base + i0;
-        if (it.tma) {
+        if (!ok) {
+            hw_fail = true;
+        } else if (it.tma) {
             convert8<true>(g, m, 8, a.decay, f, mo, s, n_sat, n_nf);
             store8_vec(a.mem + e, mo);
         } else if (nv) {
             convert8<false>(g, m, nv, a.decay, f, mo, s, n_sat, n_nf);
             store8_any(a.mem + e, nv, mo);
         }
-        if (kSym && nv) {
+        if (kSym && nv && ok) {
             if (nv == 8 && (reinterpret_cast<uintptr_t>(a.sym_out + e) & 7u) == 0) {
                 *reinterpret_cast<uint2*>(a.sym_out + e) = pack_sym8(s);
             } else {
@@ -569,7 +592,7 @@ __global__ void __launch_bounds__(kThreads, 3) convert_kernel(ConvertArgs a) {
                     if ((uint32_t)j < nv) a.sym_out[e + j] = (uint8_t)s[j];
             }
         }
-        if (kHist && nv) {
+        if (kHist && nv && ok) {
             uint32_t* h = s_hist + (tid & (kHistCopies - 1)) * kHistStride;
 #pragma unroll
             for (int j = 0; j < 8; ++j)
@@ -577,6 +600,10 @@ __global__ void __launch_bounds__(kThreads, 3) convert_kernel(ConvertArgs a) {
         }
         feed_fetch_fmt(fd, a.ws, (uint32_t)(k + 1) & 1u);  // item k + 1 was published before the previous barrier
         __syncthreads();  // everyone has read ring slot k & 1 and item[k & 1] before thread 0 reuses them
+        if (fd.fail) {    // the same for every thread: written before the barrier
+            feed_drain(fd, (uint32_t)k, parity);
+            break;
+        }
     }
     add_counts(&a.res[cur_client], n_sat, n_nf);
     if (kHist) {
@@ -588,7 +615,9 @@ __global__ void __launch_bounds__(kThreads, 3) convert_kernel(ConvertArgs a) {
             if (c) atomicAdd(reinterpret_cast<unsigned long long*>(&a.hist_out[(size_t)hist_seg * 256 + tid]), (unsigned long long)c);
         }
     }
-    if (__syncthreads_or(hw_fail) && tid == 0) set_status(&a.res[cur_client], CO3_ERR_CUDA);
+    if (__syncthreads_or(hw_fail)) {  // the block stopped early, items of any client may be missing: the call fails
+        for (uint32_t u = tid; u < a.n_clients; u += kThreads) set_status(&a.res[u], CO3_ERR_CUDA);
+    }
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -661,7 +690,7 @@ struct PackOut {
 
 struct PackSmem {
     Feed feed;
-    uint32_t bits[2][kBitWords];
+    alignas(16) uint32_t bits[2][kBitWords];  // cleared and copied out one uint4 per thread
     uint32_t enc[256];
     uint32_t scan[2][8];
     PackOut out[2];
@@ -691,8 +720,13 @@ __device__ __forceinline__ uint32_t pack_item(const PackArgs& a, PackSmem& sm, c
     } else {
         const FmtDev f = sm.feed.fmt[k & 1u];
         float g[8], m[8], mo[8];
-        if (!feed_read(sm.feed, fa, it, k, i0, nv, parity, g, m)) hw_fail = true;
-        if (kWhole) {
+        // a copy that never arrived (never expected): the memory is left alone, the block stops after this item
+        const bool ok = feed_read(sm.feed, fa, it, k, i0, nv, parity, g, m);
+        if (!ok) {
+            hw_fail = true;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) s[j] = 0u;
+        } else if (kWhole) {
             convert8<true>(g, m, 8, a.decay, f, mo, s, n_sat, n_nf);
             store8_vec(a.mem + e, mo);
         } else if (nv) {
@@ -764,6 +798,7 @@ __global__ void __launch_bounds__(kThreads, 3) pack_kernel(PackArgs a) {
     if (tid == 0) {
         mbar_init(&sm.feed.bar[0], 1);
         mbar_init(&sm.feed.bar[1], 1);
+        sm.feed.fail = 0u;
         sm.feed.cur.init(n_chunks);
         next = a.ws.chunk_desc[sm.feed.cur.chunk];
         feed_issue(sm.feed, fa, a.ws, n_chunks, 0, next, !kFromSym);
@@ -806,6 +841,10 @@ __global__ void __launch_bounds__(kThreads, 3) pack_kernel(PackArgs a) {
                 a.ws.client_fail[it.client] = 1u;
             }
         }
+        if (!kFromSym && sm.feed.fail) {  // the same for every thread: written before the barrier above
+            feed_drain(sm.feed, k, parity);
+            break;
+        }
         if (tid == 0) *out.chunk_bits = total;
         const uint32_t words = (total + 31u) >> 5;
         uint32_t* slot = out.slot + tid;
@@ -815,7 +854,10 @@ __global__ void __launch_bounds__(kThreads, 3) pack_kernel(PackArgs a) {
             if (tid + r * kThreads < words) slot[r * kThreads] = bits[r * kThreads];
     }
     if (!kFromSym) add_counts(&a.res[cur_client], n_sat, n_nf);
-    if (__syncthreads_or(hw_fail) && tid == 0) set_status(&a.res[cur_client], CO3_ERR_CUDA);
+    if (__syncthreads_or(hw_fail)) {  // the block stopped early, chunks of any client may be missing: the call fails
+        for (uint32_t u = tid; u < a.n_clients; u += kThreads) set_status(&a.res[u], CO3_ERR_CUDA);
+        if (tid == 0) a.ws.ctrl->abort = 1u;  // the kernels that would assemble the containers return at once
+    }
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -2185,7 +2227,10 @@ int decode_common(const uint8_t* const* streams, const uint8_t* single, size_t s
     uint32_t G = multi ? 1u : (uint32_t)kMaxPairs / B;
     const uint32_t g_min = (B == 1) ? 2u : 1u;  // a block needs at least one full warp
     if (!multi && G > g_min) {
-        const uint64_t want = L.n_chunks_max / (2 * 148) + 1;  // chunks per block that still give two waves
+        int dev = 0, sms = 0;
+        CO3_CUDA(cudaGetDevice(&dev));
+        CO3_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+        const uint64_t want = L.n_chunks_max / (2 * (uint64_t)(sms > 0 ? sms : 1)) + 1;  // chunks per block that still give two waves
         if (want < G) G = (uint32_t)(want < g_min ? g_min : want);
     }
     const int rc = begin_call(L, ws, res, 1, st, fmts, codes, segs, n_seg, n_elem, G, 1, streams, single, stream_bytes, n_clients);

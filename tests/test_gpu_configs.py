@@ -250,6 +250,188 @@ def test_config2_full_size_sampled_chunks():
         assert same_bits(avg[lo:lo + cnt].cpu().numpy(), want_avg)
 
 
+# ---------------------------------------------------------------------------------------------- full sizes
+def _top_level(E, M):
+    """Largest level of the format [1, E, M] before the multiplier: (2 - 2^-M) 2^(2^(E-1)-1), Sec. V-B boundary."""
+    return float((2.0 - 2.0 ** -M) * 2.0 ** (2 ** (E - 1) - 1))
+
+
+def _codes_from_oracle_sample(sess, g0, sizes, ofmts, decay, n_sample=32768):
+    """One code per layer computed by the oracle alone: the symbol counts of the leading elements of client 0's
+    first-round gradient (zero memory).  Any complete code serves the comparison; this one is close to the fitted one."""
+    seg_off = np.concatenate([[0], np.cumsum(sizes)])
+    ocodes = []
+    for k, n in enumerate(sizes):
+        g = g0[int(seg_off[k]):int(seg_off[k]) + min(int(n), n_sample)].cpu().numpy()
+        r = oracle.convert(g, np.zeros(g.size, dtype=np.float32), decay, ofmts[k])
+        ocodes.append(oracle.code_build(oracle.histogram(r["sym"]), ofmts[k]))
+    arr = np.zeros(len(sizes), dtype=co3.CODE_DTYPE)
+    for k, c in enumerate(ocodes):
+        ln, bits = oracle.code_arrays(c)
+        arr[k]["len"] = ln
+        arr[k]["bits"] = bits.astype(np.uint16)
+    sess.set_codes(arr)
+    return ocodes
+
+
+def _full_size_sampled(cfg, sizes, fmts, clients, n_random=24, payload_clients=8, seed=0):
+    """Two rounds of the batched encode and one decode-aggregate at full size through the session (the calls and the
+    launch shapes bench.py times), compared with the oracle on sampled chunks: error memory, payload words, sub-chunk
+    offsets and the averaged gradient bit for bit; plus properties of whole streams and the saturation counters of
+    the first round against a plain fp32 comparison of every element.  Returns what the caller may want to look at."""
+    import bench
+    C = co3.CHUNK_SYMS
+    sess = Co3Session(sizes, fmts, clients, cfg["decay"], "cuda")
+    ofmts = [oracle.Fmt(E, M, 0, s, inv) for (E, M, _, s, inv) in fmts]
+    g0 = bench.make_grads(cfg, sizes, clients, sess.stride, 0, "cuda")
+    ocodes = _codes_from_oracle_sample(sess, g0, sizes, ofmts, cfg["decay"])
+    mems = sess.new_client_buffer()
+    sess.encode(g0, mems)
+    torch.cuda.synchronize()
+    res0 = sess.encode_results()
+    assert (res0["status"] == co3.OK).all(), res0["status"]
+    seg_off = np.concatenate([[0], np.cumsum(sizes)]).astype(np.int64)
+    # first round, zero memory: v = g, so an element saturates exactly when |fl32(g * scale)| exceeds the largest level
+    n_sat = torch.zeros(clients, dtype=torch.int64, device="cuda")
+    g0v = g0.view(clients, sess.stride)
+    for k, (E, M, _, s, _) in enumerate(fmts):
+        t = g0v[:, int(seg_off[k]):int(seg_off[k + 1])] * np.float32(s)
+        n_sat += (t.abs() > _top_level(E, M)).sum(dim=1)
+        del t
+    assert np.array_equal(n_sat.cpu().numpy().astype(np.uint64), res0["n_saturated"])
+    del g0v, g0
+    mem_before = mems.clone()
+    g1 = bench.make_grads(cfg, sizes, clients, sess.stride, 1, "cuda")
+    sess.encode(g1, mems)
+    avg = sess.decode_aggregate()
+    torch.cuda.synchronize()
+    res = sess.encode_results()
+    assert (res["status"] == co3.OK).all() and sess.decode_result()["status"][0] == co3.OK
+
+    seg_first = np.concatenate([[0], np.cumsum([(n + C - 1) // C for n in sizes])]).astype(np.int64)
+    n_chunks = int(seg_first[-1])
+    al = lambda x: (x + 15) & ~15
+    chunk_off = al(64 + 24 * len(sizes))
+    sub_off = al(chunk_off + 8 * (n_chunks + 1))
+    pay_off = al(sub_off + 32 * n_chunks)
+    cap = sess.capacity
+    sv = sess.streams.view(clients, cap)
+
+    # whole-stream properties, on the first, a middle and the last client
+    check_clients = sorted({0, clients // 2, clients - 1})
+    wo_last = None
+    for u in check_clients:
+        head = sv[u, :pay_off].cpu().numpy()
+        h32, h64 = head[:64].view(np.uint32), head[:64].view(np.uint64)
+        assert h32[0] == 0x53334F43 and h32[1] == 1 and h32[2] == len(sizes) and h32[3] == C and h32[4] == co3.SUB_SYMS
+        assert h64[3] == sess.n_elem and h64[4] == n_chunks
+        assert h64[6] == res[u]["payload_bits"] and h64[7] == res[u]["container_bytes"] == al(pay_off + 4 * int(h64[5]))
+        wo = head[chunk_off:chunk_off + 8 * (n_chunks + 1)].view(np.uint64).astype(np.int64)
+        assert wo[0] == 0 and (np.diff(wo) >= 0).all() and (np.diff(wo) <= C * 16 // 32).all() and wo[-1] == h64[5]
+        segtab = head[64:64 + 24 * len(sizes)].view(np.uint64).reshape(-1, 3)
+        assert np.array_equal(segtab[:, 0], np.array(sizes, dtype=np.uint64))
+        assert np.array_equal(segtab[:, 1].astype(np.int64), seg_first[:-1])
+        assert int(segtab[:, 2].sum()) == res[u]["payload_bits"]
+        # payload bits of a chunk round up to its words: the container holds between bits/32 and bits/32 + chunks words
+        assert int(h64[6]) <= 32 * int(h64[5]) < int(h64[6]) + 32 * n_chunks + 32
+        wo_last = wo
+
+    # chunks to compare: ends, segment and scan-range boundaries, the chunks around the 2^31-byte and 2^32-bit marks
+    # of the inputs and of the payload, and random ones
+    rng = np.random.default_rng(seed)
+    picks = {0, n_chunks - 1, int(seg_first[1]) - 1, int(seg_first[len(sizes) // 2]), int(seg_first[-2])}
+    picks |= {c for c in (4095, 4096, 16383, 16384, 65535, 65536, n_chunks - 4097) if 0 <= c < n_chunks}
+    picks |= {int(c) for c in rng.integers(0, n_chunks, size=n_random)}
+    for mark_words in (1 << 27, 1 << 29):                       # payload bit 2^32, payload byte 2^31
+        c = int(np.searchsorted(wo_last, mark_words, side="right")) - 1
+        if 0 <= c < n_chunks - 1:
+            picks |= {c, c + 1}
+    if len(sizes) == 1:
+        for mark_elems in (1 << 29, 1 << 28):                   # input byte 2^31 and 2^30
+            if mark_elems < sizes[0]:
+                picks |= {mark_elems // C - 1, mark_elems // C}
+    pay_clients = list(range(clients)) if clients <= 2 * payload_clients else sorted(
+        {0, 1, clients // 2, clients - 2, clients - 1} | {int(u) for u in rng.integers(0, clients, size=payload_clients)})
+    one_pay = al(al(al(64 + 24) + 16) + 32)                     # payload offset of the oracle's one-chunk stream
+    one_sub = al(al(64 + 24) + 16)
+    g1v, mbv, mv = g1.view(clients, sess.stride), mem_before.view(clients, sess.stride), mems.view(clients, sess.stride)
+    n_outlier_chunks = 0
+    for c in sorted(picks):
+        k = int(np.searchsorted(seg_first, c, side="right") - 1)
+        start = (c - int(seg_first[k])) * C
+        cnt = min(C, sizes[k] - start)
+        lo = int(seg_off[k]) + start
+        g_all = g1v[:, lo:lo + cnt].cpu().numpy()
+        m_all = mbv[:, lo:lo + cnt].cpu().numpy()
+        m_new = mv[:, lo:lo + cnt].cpu().numpy()
+        wo_all = sv[:, chunk_off + 8 * c:chunk_off + 8 * c + 16].cpu().numpy().view(np.uint64).reshape(clients, 2)
+        acc = np.zeros(cnt, dtype=np.float32)
+        for u in range(clients):
+            m = m_all[u].copy()
+            r = oracle.convert(np.ascontiguousarray(g_all[u]), m, cfg["decay"], ofmts[k])
+            assert same_bits(m_new[u], m), (c, u)
+            n_outlier_chunks += int(r["n_saturated"] > 0)
+            acc = (acc + r["ghat"]).astype(np.float32)
+            st, want = oracle.encode(r["sym"], [cnt], [ocodes[k]])
+            assert st == oracle.OK
+            nwords = int(want[40:48].view(np.uint64)[0])
+            assert int(wo_all[u, 1] - wo_all[u, 0]) == nwords, (c, u)
+            if u in pay_clients:
+                w0 = int(wo_all[u, 0])
+                got = sv[u, pay_off + 4 * w0:pay_off + 4 * (w0 + nwords)].cpu().numpy()
+                assert np.array_equal(got, want[one_pay:one_pay + 4 * nwords]), (c, u)
+                got_sub = sv[u, sub_off + 32 * c:sub_off + 32 * c + 32].cpu().numpy()
+                assert np.array_equal(got_sub, want[one_sub:one_sub + 32]), (c, u)
+        want_avg = (acc / np.float32(clients)).astype(np.float32)
+        assert same_bits(avg[lo:lo + cnt].cpu().numpy(), want_avg), c
+    return dict(n_chunks=n_chunks, picks=len(picks), res=res, outlier_chunks=n_outlier_chunks)
+
+
+def test_config3_full_size_sampled_chunks():
+    """100 clients x 11,181,642 elements in 62 layers (4.5 GB of gradients, as much memory; the clients from the 97th
+    on lie beyond byte 2^32 of both), second round with live memories, then the 100-client decode-aggregate."""
+    import bench
+    cfg, sizes, fmts, clients = bench.workload(3)
+    assert clients == 100 and sum(sizes) == 11_181_642
+    out = _full_size_sampled(cfg, list(sizes), fmts, clients, n_random=10, payload_clients=8)
+    assert out["n_chunks"] == 5497
+
+
+@pytest.mark.parametrize("cell", [dict(fmt=(2, 1), beta=1.0, decay=0.9), dict(fmt=(3, 0), beta=0.5, decay=0.5),
+                                  dict(fmt=(4, 3), beta=2.0, decay=0.99), dict(fmt=(5, 2), beta=1.0, decay=0.9)],
+                         ids=lambda c: "fmt%d%d" % c["fmt"])
+def test_config4_full_size_sampled_chunks(cell):
+    """The sweep's 25,600,000-element vector at full length, one cell per format (the 36 cells run at 200 k above)."""
+    cfg = ci.config(4)
+    assert cfg["sizes"] == (25_600_000,)
+    E, M = cell["fmt"]
+    c = dict(cfg, fmt=(E, M), beta=(cell["beta"],), decay=cell["decay"])
+    s, inv = ci.scale_for(E, M, cell["beta"], cfg["alpha"][0])
+    out = _full_size_sampled(c, list(cfg["sizes"]), [(E, M, 0, s, inv)], 1, n_random=40)
+    assert out["n_chunks"] == 12500
+
+
+def test_config5a_full_size_sampled_chunks():
+    """1 client x 1,000,000,000 elements with 0.01 % outliers at 100x scale: 488,282 chunks, the two-level chunk
+    offset scan over 120 ranges, payload bit offsets beyond 2^32."""
+    import bench
+    cfg, sizes, fmts, clients = bench.workload(5)
+    assert clients == 1 and sizes == (1_000_000_000,)
+    out = _full_size_sampled(cfg, list(sizes), fmts, 1, n_random=48)
+    assert out["n_chunks"] == 488_282 and out["outlier_chunks"] > 0
+    assert int(out["res"][0]["payload_bits"]) > 1 << 32
+
+
+def test_config5b_full_size_sampled_chunks():
+    """8 clients x 125,000,000 elements, same distribution with outliers."""
+    import bench
+    cfg, sizes, fmts, _ = bench.workload(5)
+    part = cfg["part_b"]
+    c = dict(cfg, sizes=part["sizes"])
+    out = _full_size_sampled(c, list(part["sizes"]), fmts, part["clients"], n_random=24)
+    assert out["n_chunks"] == 61036
+
+
 def test_config2_full_size_fit_and_error_magnitude():
     """The set-up and diagnostic calls at the benchmarked size (10 clients x 11,181,642 elements in 62 layers, live
     memories after one round): every layer's fitted multiplier within one fp32 ULP of the oracle's (identical on

@@ -158,6 +158,16 @@ def test_invalid_descriptors_are_refused_on_the_device():
     ln[:8] = 2
     out = Gpu(case).encode(g, np.zeros_like(g), [oracle.make_code(ln, np.arange(256) % 4)])
     assert out["res"][0]["status"] == co3.ERR_INVALID_ARG
+    # tables whose Kraft sum is at most 1 but in which one codeword starts another ("0" and "01"), or repeats it
+    for lens, words in (([1, 2], [0, 1]), ([3, 3, 2], [5, 5, 0]), ([2, 5, 3], [1, 0b01101, 0b100])):
+        ln = np.zeros(256, dtype=int)
+        bits = np.zeros(256, dtype=int)
+        ln[:len(lens)] = lens
+        bits[:len(lens)] = words
+        assert sum(2.0 ** -l for l in lens) <= 1.0
+        out = Gpu(case).encode(g, np.zeros_like(g), [oracle.make_code(ln, bits)])
+        assert out["res"][0]["status"] == co3.ERR_INVALID_ARG, (lens, words)
+        assert same_bits(out["mem"], np.zeros_like(g))
 
 
 def test_host_side_argument_checks():
