@@ -68,6 +68,13 @@ def lib():
                                    C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                    C.POINTER(C.c_uint64), C.POINTER(C.c_uint64)]
         L.co3o_histogram.restype = None
+        L.co3o_philox4x32_10.restype = None
+        L.co3o_philox4x32_10.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
+        L.co3o_dither_draws.restype = None
+        L.co3o_dither_draws.argtypes = [C.c_uint32, C.c_uint32, C.c_uint32, C.c_uint64, C.c_uint64, C.c_void_p]
+        L.co3o_convert_dithered.restype = C.c_int
+        L.co3o_convert_dithered.argtypes = [C.c_void_p, C.c_void_p, C.c_float, C.POINTER(Fmt), C.c_uint64, C.c_void_p,
+                                            C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.co3o_histogram.argtypes = [C.c_void_p, C.c_uint64, C.c_void_p]
         L.co3o_code_build.restype = C.c_int
         L.co3o_code_build.argtypes = [C.c_void_p, C.POINTER(Fmt), C.POINTER(Code)]
@@ -157,6 +164,41 @@ def convert(g: np.ndarray, m: np.ndarray, decay: float, fmt: Fmt, want_v: bool =
     if want_v:
         out["v"] = v
     return out
+
+
+def philox4x32_10(ctr, key) -> np.ndarray:
+    """One block of the counter-based generator: four 32-bit words from a 4-word counter and a 2-word key."""
+    c = np.ascontiguousarray(ctr, dtype=np.uint32)
+    k = np.ascontiguousarray(key, dtype=np.uint32)
+    out = np.zeros(4, dtype=np.uint32)
+    assert c.size == 4 and k.size == 2
+    lib().co3o_philox4x32_10(_ptr(c), _ptr(k), _ptr(out))
+    return out
+
+
+def dither_draws(seed: int, client: int, layer: int, first_place: int, n: int) -> np.ndarray:
+    """The 24-bit draws of n consecutive elements of one layer of one client, from place first_place on."""
+    out = np.empty(n, dtype=np.uint32)
+    lib().co3o_dither_draws(seed, client, layer, first_place, n, _ptr(out))
+    return out
+
+
+def convert_dithered(g: np.ndarray, m: np.ndarray, decay: float, fmt: Fmt, draws: np.ndarray):
+    """convert() with the dithered rounding rule; draws: one integer in [0, 2^24) per element.  ``m`` is updated."""
+    g = np.ascontiguousarray(g, dtype=np.float32)
+    d = np.ascontiguousarray(draws, dtype=np.uint32)
+    assert m.dtype == np.float32 and m.flags.c_contiguous and m.shape == g.shape and d.shape == g.shape
+    n = g.size
+    wide = 1 + fmt.exp_bits + fmt.mant_bits > 8
+    sym = np.empty(n, dtype=np.uint16 if wide else np.uint8)
+    ghat = np.empty(n, dtype=np.float32)
+    nsat, nnf = C.c_uint64(0), C.c_uint64(0)
+    st = lib().co3o_convert_dithered(_ptr(g), _ptr(m), C.c_float(decay), C.byref(fmt), n, _ptr(d),
+                                     None if wide else _ptr(sym), _ptr(sym) if wide else None, _ptr(ghat),
+                                     C.byref(nsat), C.byref(nnf))
+    if st != OK:
+        raise ValueError("oracle convert_dithered: status %d" % st)
+    return dict(sym=sym, ghat=ghat, n_saturated=nsat.value, n_nonfinite=nnf.value)
 
 
 def histogram(sym: np.ndarray) -> np.ndarray:

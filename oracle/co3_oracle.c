@@ -19,7 +19,8 @@
  * Pins (tests/test_oracle_*.py): library casts to the standard 8/16-bit layouts, the closed forms
  * of Sec. V-B, exact-rational brute force over the printed level form, the printed bias
  * polynomials of Sec. IV-B, Kraft equality / entropy bounds / brute-force optimality for the
- * code, a hand-worked container example.  Parity unpinned (the paper prints nothing to check
+ * code, a hand-worked container example; for the dithered converter the published test vectors of
+ * its generator and, with all 2^24 draws enumerated, the exact mean of the result.  Parity unpinned (the paper prints nothing to check
  * them against; only this oracle and the CUDA library agreeing): the order among equal Huffman
  * weights and the 16-bit length limit, the container layout, the NaN/Inf reading, and the tie
  * between zero and the smallest normal level when sub-normal levels are flushed.
@@ -217,6 +218,108 @@ int co3o_convert(const float *g, float *m, float decay, const co3o_fmt *f, uint6
         if (sym16) sym16[i] = (uint16_t)s;
         if (ghat) ghat[i] = gh;
         if (v_out) v_out[i] = v;
+        m[i] = mnew;
+    }
+    co3o_levels_free(&L);
+    if (n_saturated) *n_saturated = nsat;
+    if (n_nonfinite) *n_nonfinite = nnf;
+    return CO3O_OK;
+}
+
+/* ------------------------------------------------------------------------------------------
+ * Dithered conversion (Sec. II-B (ii): the quantizer may be a stochastic mapping, so that
+ * non-subtractive dither quantization can be implemented).  Reading taken: the dither is uniform
+ * over the step between the two levels around the scaled value, which is the same as choosing the
+ * upper level with probability (|t| - lower) / (upper - lower): with R a uniform 24-bit integer,
+ * the upper level is taken iff R < (|t| - lower) / (upper - lower) * 2^24.  Every step of the level
+ * set is a power of two, so the right-hand side is exact in fp64; a value that is a level stays
+ * where it is for every R, and averaged over all 2^24 values of R the result is the value itself
+ * whenever that right-hand side is an integer (every fp32 value from the smallest normal level up).
+ * Beyond the largest level the value saturates as before; NaN and infinities are treated as before.
+ * The parameter server does not need the draws (the dither is not subtracted).
+ *
+ * The draws are inputs here.  co3o_dither_draws produces the ones the library uses: Philox-4x32
+ * with 10 rounds (Salmon, Moraes, Dror, Shaw, "Parallel random numbers: as easy as 1, 2, 3", SC 2011),
+ * key (seed, 0), counter (p / 4 low word, p / 4 high word, client, layer) for the element at place
+ * p of its layer, output word p % 4, top 24 bits.
+ * ------------------------------------------------------------------------------------------ */
+void co3o_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4])
+{
+    uint32_t c0 = ctr[0], c1 = ctr[1], c2 = ctr[2], c3 = ctr[3], k0 = key[0], k1 = key[1];
+    for (int round = 0; round < 10; ++round) {
+        if (round > 0) { k0 += 0x9E3779B9u; k1 += 0xBB67AE85u; } /* key schedule: add the Weyl constants */
+        const uint64_t p0 = (uint64_t)0xD2511F53u * c0, p1 = (uint64_t)0xCD9E8D57u * c2;
+        const uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ k0, n1 = (uint32_t)p1;
+        const uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ k1, n3 = (uint32_t)p0;
+        c0 = n0; c1 = n1; c2 = n2; c3 = n3;
+    }
+    out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+void co3o_dither_draws(uint32_t seed, uint32_t client, uint32_t layer, uint64_t first_place, uint64_t n,
+                       uint32_t *draws)
+{
+    const uint32_t key[2] = {seed, 0u};
+    for (uint64_t i = 0; i < n; ++i) {
+        const uint64_t p = first_place + i;
+        const uint32_t ctr[4] = {(uint32_t)(p >> 2), (uint32_t)(p >> 34), client, layer};
+        uint32_t out[4];
+        co3o_philox4x32_10(ctr, key, out);
+        draws[i] = out[p & 3u] >> 8;
+    }
+}
+
+/* Magnitude code for a >= 0 under the draw R (0 <= R < 2^24). */
+static uint32_t co3o_dithered(const co3o_levels *L, double a, uint32_t R, int *saturated)
+{
+    int lo = 0, hi = L->n - 1;
+    *saturated = 0;
+    if (a > L->level[hi]) {
+        *saturated = 1;
+        return L->code[hi];
+    }
+    while (lo < hi) { /* largest index with level <= a */
+        const int mid = (lo + hi + 1) / 2;
+        if (L->level[mid] <= a) lo = mid; else hi = mid - 1;
+    }
+    if (lo == L->n - 1 || a == L->level[lo]) return L->code[lo];
+    const double where = (a - L->level[lo]) / (L->level[lo + 1] - L->level[lo]); /* in (0, 1), exact */
+    return (double)R < where * 16777216.0 ? L->code[lo + 1] : L->code[lo];
+}
+
+/* co3o_convert with the nearest-level rule replaced by the dithered one; draws[i] in [0, 2^24). */
+int co3o_convert_dithered(const float *g, float *m, float decay, const co3o_fmt *f, uint64_t n,
+                          const uint32_t *draws, uint8_t *sym8, uint16_t *sym16, float *ghat,
+                          uint64_t *n_saturated, uint64_t *n_nonfinite)
+{
+    if (!co3o_fmt_ok(f) || !draws) return CO3O_ERR_ARG;
+    co3o_levels L;
+    if (!co3o_levels_init(&L, f)) return CO3O_ERR_ARG;
+    const int nb = f->exp_bits + f->mant_bits;
+    uint64_t nsat = 0, nnf = 0;
+    for (uint64_t i = 0; i < n; ++i) {
+        if (draws[i] >> 24) { co3o_levels_free(&L); return CO3O_ERR_ARG; }
+        const float v = fmaf(decay, m[i], g[i]);
+        uint32_t c, sign;
+        int sat = 0;
+        float gh, mnew;
+        if (isnan(v)) {
+            c = 0; sign = 0; nnf++;
+            gh = 0.0f; mnew = 0.0f;
+        } else {
+            const float t = v * f->scale;
+            c = co3o_dithered(&L, fabs((double)t), draws[i], &sat);
+            sign = (t < 0.0f && c != 0) ? 1u : 0u;
+            float q = (float)co3o_level(f, c);
+            if (sign) q = -q;
+            gh = q * f->inv_scale;
+            if (isinf(v)) { nnf++; mnew = 0.0f; }
+            else { nsat += (uint64_t)sat; mnew = v - gh; }
+        }
+        const uint32_t s = (sign << nb) | c;
+        if (sym8) sym8[i] = (uint8_t)s;
+        if (sym16) sym16[i] = (uint16_t)s;
+        if (ghat) ghat[i] = gh;
         m[i] = mnew;
     }
     co3o_levels_free(&L);
