@@ -496,8 +496,17 @@ def standalone_kernels(state, cfg, clients, steps, warmup, peak):
     out["convert_standalone"] = row(13.0 * n_local / 1e9, n, tot, steps)
     n, tot = timed_calls(conv(sess.hist, sym_buf), "convert")
     out["convert_hist_standalone"] = row(13.0 * n_local / 1e9, n, tot, steps)
+
+    def dry(i):     # the symbol statistics alone: gradient and memory in, nothing but 256 counters per layer out
+        st = co3.co3_histogram(grads[i % 2], mems_k1, sess.decay, sess.fmts, sess.segs, sess.n_seg, sess.n_elem,
+                               clients, sess.stride, sess.hist, sess.res_enc, sess.workspace, stream)
+        if st != co3.OK:
+            raise RuntimeError("co3_histogram: " + co3.co3_status_string(st))
+
+    n, tot = timed_calls(dry, "convert")
+    out["histogram_standalone"] = row(8.0 * n_local / 1e9, n, tot, steps)
     if (sess.encode_results()["status"] != co3.OK).any():
-        raise RuntimeError("device status after co3_convert")
+        raise RuntimeError("device status after co3_convert / co3_histogram")
     del sym_buf
 
     # the data-driven refit of every layer's multiplier (moments of v = g + decay * m, then the per-layer fit), on

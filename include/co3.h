@@ -133,6 +133,46 @@ int co3_convert(const float* grad, float* mem, float decay,
                 void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * Symbol statistics alone (Sec. IV-A (ii): a Huffman code is designed for the distribution of its source, here the
+ * symbols of Q_fp(g + decay * m) of this round): hist_out exactly as co3_convert would fill it, and nothing else is
+ * written: grad and mem are both read only, so that the code can be fitted before the round is encoded in one pass by
+ * co3_encode.  res [device] co3_result[n_clients] receives the saturation and non-finite counts the round will see.
+ */
+int co3_histogram(const float* grad, const float* mem, float decay,
+                  const co3_fmt* fmts /* [device] n_seg */, const co3_seg* segs /* [device] n_seg */,
+                  uint32_t n_seg, uint64_t n_elem, uint32_t n_clients, uint64_t client_stride_elems,
+                  uint64_t* hist_out /* [device] uint64[n_seg][256] */, co3_result* res,
+                  void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * The conversion with dithered rounding, which Sec. II-B (ii) allows for (the quantizer may be a stochastic mapping,
+ * so that non-subtractive dither quantization can be implemented).  Reading: the dither is uniform over the step
+ * between the two levels around the scaled value t, i.e. the upper level is taken iff
+ *     R < (|t| - lower) / (upper - lower) * 2^24,
+ * R a uniform 24-bit integer, so that the result averages to t itself; a t that is a level stays where it is, beyond
+ * the largest level it saturates as in co3_convert, NaN and infinities are treated as there.  R is word p % 4, top
+ * 24 bits, of Philox-4x32-10 (Salmon, Moraes, Dror, Shaw, SC 2011) with key (seed, 0) and counter (p / 4 low word,
+ * p / 4 high word, client, layer index) for the element at place p of its layer: give every round another seed.
+ * Everything else (arguments, outputs, statuses) is as in co3_convert, co3_histogram and co3_encode; the parameter
+ * server needs neither the seed nor to know that the stream was dithered (co3_decode_aggregate as usual).
+ */
+int co3_convert_dither(const float* grad, float* mem, float decay,
+                       const co3_fmt* fmts /* [device] n_seg */, const co3_seg* segs /* [device] n_seg */,
+                       uint32_t n_seg, uint64_t n_elem, uint32_t n_clients, uint64_t client_stride_elems,
+                       uint32_t seed, uint8_t* sym_out, uint64_t* hist_out, co3_result* res,
+                       void* workspace, size_t workspace_bytes, void* stream);
+int co3_histogram_dither(const float* grad, const float* mem, float decay,
+                         const co3_fmt* fmts /* [device] n_seg */, const co3_seg* segs /* [device] n_seg */,
+                         uint32_t n_seg, uint64_t n_elem, uint32_t n_clients, uint64_t client_stride_elems,
+                         uint32_t seed, uint64_t* hist_out, co3_result* res,
+                         void* workspace, size_t workspace_bytes, void* stream);
+int co3_encode_dither(const float* grad, float* mem, float decay,
+                      const co3_fmt* fmts, const co3_code* codes /* [device] n_seg */, const co3_seg* segs,
+                      uint32_t n_seg, uint64_t n_elem, uint32_t n_clients, uint64_t client_stride_elems,
+                      uint32_t seed, uint8_t* streams_out, size_t stream_capacity, uint32_t chunk_syms,
+                      void* workspace, size_t workspace_bytes, co3_result* res, void* stream);
+
+/*
  * co3_convert without a workspace argument (the paper has no counterpart; this exists for the host
  * program's sake).  Some callers are not allowed to obtain device memory at the point where they run
  * the conversion: a plug-in inside a server that handed all device memory to its own pool at start-up,

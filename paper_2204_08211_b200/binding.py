@@ -15,6 +15,7 @@ MAX_CODE_LEN, CHUNK_SYMS, SUB_SYMS = 16, 2048, 128
 
 FMT_DTYPE = np.dtype([("exp_bits", np.uint8), ("mant_bits", np.uint8), ("flags", np.uint16),
                       ("scale", np.float32), ("inv_scale", np.float32)])
+FMT_FLUSH_SUBNORMALS = 1
 CODE_DTYPE = np.dtype([("len", np.uint8, (256,)), ("bits", np.uint16, (256,))])
 SEG_DTYPE = np.dtype([("elem_off", np.uint64), ("n_elem", np.uint64)])
 RESULT_DTYPE = np.dtype([("status", np.int32), ("first_bad_chunk", np.uint32), ("payload_bits", np.uint64),
@@ -43,6 +44,10 @@ def _load():
     L.co3_workspace_bytes.argtypes = [u64, u32, u32, u32, C.POINTER(sz)]
     L.co3_stream_capacity_bytes.argtypes = [u64, u32, u32, C.POINTER(sz)]
     L.co3_convert.argtypes = [vp, vp, f32, vp, vp, u32, u64, u32, u64, vp, vp, vp, vp, sz, vp]
+    L.co3_histogram.argtypes = [vp, vp, f32, vp, vp, u32, u64, u32, u64, vp, vp, vp, sz, vp]
+    L.co3_convert_dither.argtypes = [vp, vp, f32, vp, vp, u32, u64, u32, u64, u32, vp, vp, vp, vp, sz, vp]
+    L.co3_histogram_dither.argtypes = [vp, vp, f32, vp, vp, u32, u64, u32, u64, u32, vp, vp, vp, sz, vp]
+    L.co3_encode_dither.argtypes = [vp, vp, f32, vp, vp, vp, u32, u64, u32, u64, u32, vp, sz, u32, vp, sz, vp, vp]
     L.co3_convert_static.argtypes = [vp, vp, f32, vp, vp, u32, u64, u32, u64, vp, vp, vp, vp]
     L.co3_code_build.argtypes = [vp, vp, vp]
     L.co3_code_build_device.argtypes = [vp, vp, u32, vp, vp, vp]
@@ -56,7 +61,7 @@ def _load():
     L.co3_decode.argtypes = [vp, sz, vp, vp, vp, u32, u64, u32, vp, vp, vp, sz, vp, vp]
     L.co3_profile_enable.argtypes = [C.c_int]
     L.co3_profile_read.argtypes = [vp, vp]
-    for name in ("co3_error_magnitude", "co3_model_weights", "co3_fit_scale", "co3_profile_enable", "co3_profile_read", "co3_convert_static", "co3_workspace_bytes", "co3_stream_capacity_bytes", "co3_convert", "co3_code_build", "co3_code_build_device", "co3_encode",
+    for name in ("co3_histogram", "co3_convert_dither", "co3_histogram_dither", "co3_encode_dither", "co3_error_magnitude", "co3_model_weights", "co3_fit_scale", "co3_profile_enable", "co3_profile_read", "co3_convert_static", "co3_workspace_bytes", "co3_stream_capacity_bytes", "co3_convert", "co3_code_build", "co3_code_build_device", "co3_encode",
                  "co3_encode_symbols", "co3_decode_aggregate", "co3_decode_aggregate_update", "co3_decode"):
         getattr(L, name).restype = C.c_int
     _lib = L
@@ -155,6 +160,41 @@ def co3_convert(grad, mem, decay, fmts, segs, n_seg, n_elem, n_clients, client_s
                                n_clients, client_stride_elems, _dev(sym_out, True), _dev(hist_out, True),
                                _dev(res), _dev(workspace), workspace.numel() * workspace.element_size(),
                                _stream(stream))
+
+
+def co3_histogram(grad, mem, decay, fmts, segs, n_seg, n_elem, n_clients, client_stride_elems, hist_out, res,
+                  workspace, stream=None) -> int:
+    """Symbol counts of this round (uint64/int64[n_seg * 256]) without touching the memory or writing symbols."""
+    return _load().co3_histogram(_dev(grad), _dev(mem), float(decay), _dev(fmts), _dev(segs), n_seg, n_elem,
+                                 n_clients, client_stride_elems, _dev(hist_out), _dev(res), _dev(workspace),
+                                 workspace.numel() * workspace.element_size(), _stream(stream))
+
+
+def co3_convert_dither(grad, mem, decay, fmts, segs, n_seg, n_elem, n_clients, client_stride_elems, seed, sym_out,
+                       hist_out, res, workspace, stream=None) -> int:
+    """co3_convert with dithered (stochastic) rounding; `seed` keys the draw stream: another one every round."""
+    return _load().co3_convert_dither(_dev(grad), _dev(mem), float(decay), _dev(fmts), _dev(segs), n_seg, n_elem,
+                                      n_clients, client_stride_elems, int(seed), _dev(sym_out, True),
+                                      _dev(hist_out, True), _dev(res), _dev(workspace),
+                                      workspace.numel() * workspace.element_size(), _stream(stream))
+
+
+def co3_histogram_dither(grad, mem, decay, fmts, segs, n_seg, n_elem, n_clients, client_stride_elems, seed, hist_out,
+                         res, workspace, stream=None) -> int:
+    """co3_histogram for a round that will be converted with dithered rounding under the same seed."""
+    return _load().co3_histogram_dither(_dev(grad), _dev(mem), float(decay), _dev(fmts), _dev(segs), n_seg, n_elem,
+                                        n_clients, client_stride_elems, int(seed), _dev(hist_out), _dev(res),
+                                        _dev(workspace), workspace.numel() * workspace.element_size(),
+                                        _stream(stream))
+
+
+def co3_encode_dither(grad, mem, decay, fmts, codes, segs, n_seg, n_elem, n_clients, client_stride_elems, seed,
+                      streams_out, stream_capacity, workspace, res, chunk_syms: int = CHUNK_SYMS, stream=None) -> int:
+    """co3_encode with dithered (stochastic) rounding."""
+    return _load().co3_encode_dither(_dev(grad), _dev(mem), float(decay), _dev(fmts), _dev(codes), _dev(segs), n_seg,
+                                     n_elem, n_clients, client_stride_elems, int(seed), _dev(streams_out),
+                                     stream_capacity, chunk_syms, _dev(workspace),
+                                     workspace.numel() * workspace.element_size(), _dev(res), _stream(stream))
 
 
 STATIC_SCRATCH_BYTES = 2 << 20

@@ -40,6 +40,8 @@ struct ChunkDesc {
     uint32_t seg;    // segment (layer) of the chunk
     uint32_t cnt;    // symbols in the chunk (kC except for the last chunk of a segment)
     uint64_t elem0;  // index of its first element inside a client's vector
+    uint32_t cis;    // the chunk's index inside its segment: its first element is at place cis * kC of the layer
+    uint32_t pad;
 };
 
 // A decode tile: up to `tile_chunks` consecutive chunks of one segment.
@@ -65,7 +67,9 @@ struct FmtDev {
     uint32_t half_min_bits;    // fp32 pattern of 2^(emin-1)
     float magic;               // 2^(emin - M + 23): adding it rounds to a multiple of the sub-normal step
     float scale, inv_scale;
+    uint32_t pad[2];           // 64 bytes: the table is addressed in whole 16-byte units
 };
+static_assert(sizeof(FmtDev) == 64, "FmtDev is a whole number of 16-byte units");
 
 // Workspace sections (device pointers), computed on the host from sizes only.
 struct Ws {
@@ -151,9 +155,10 @@ __device__ __forceinline__ float convert_one(float g, float m, float decay, cons
 // Rounding by one fp32 addition: with ae the (clamped) exponent of |t|, |t| + 2^(ae + 23 - M) is rounded by
 // the adder to a multiple of the format's step in that binade, ties to the even multiple, which has the
 // even code when M >= 1.  Inputs beyond the largest level and non-finite ones are clamped to it here and
-// reported in `beyond` (a NaN fails the comparison too); the caller repeats a group that holds one with
-// convert_one, which tells those cases apart and counts them.  Inputs that land on the largest level from
-// inside the range (common in the narrow formats) need no second look.
+// reported in `beyond` (a NaN fails the comparison too): for a finite input that is already the right level
+// and memory (saturation, Sec. V-B boundary) and the caller only counts it; a group that holds a NaN or an
+// infinity is repeated with convert_one.  Inputs that land on the largest level from inside the range (common
+// in the narrow formats) need no second look.
 __device__ __forceinline__ float convert_fast(float g, float m, float decay, const FmtDev& f, uint32_t& sym,
                                               bool& beyond) {
     const float v = __fmaf_rn(decay, m, g);
@@ -171,6 +176,66 @@ __device__ __forceinline__ float convert_fast(float g, float m, float decay, con
     sym = code | (sgn >> f.sign_shift);
     const float ghat = __fmul_rn(__uint_as_float(__float_as_uint(qmag) | sgn), f.inv_scale);
     return __fsub_rn(v, ghat);
+}
+
+// Philox-4x32 with 10 rounds (Salmon, Moraes, Dror, Shaw, SC 2011): a block of four 32-bit words from a counter
+// and a key.  Each round multiplies two counter words by fixed constants, crosses the halves of the products with
+// the other two words and the key, and the key advances by Weyl constants between rounds.
+__device__ __forceinline__ uint4 philox4x32_10(uint4 c, uint32_t k0, uint32_t k1) {
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        if (r > 0) { k0 += 0x9E3779B9u; k1 += 0xBB67AE85u; }
+        const uint32_t lo0 = 0xD2511F53u * c.x, hi0 = __umulhi(0xD2511F53u, c.x);
+        const uint32_t lo1 = 0xCD9E8D57u * c.z, hi1 = __umulhi(0xCD9E8D57u, c.z);
+        c = make_uint4(hi1 ^ c.y ^ k0, lo1, hi0 ^ c.w ^ k1, lo0);
+    }
+    return c;
+}
+
+// convert_one with the nearest-level rule replaced by the dithered one (Sec. II-B (ii): the quantizer as a stochastic
+// mapping): with R the element's 24-bit draw the upper of the two levels around |t| is taken iff
+// R < (|t| - lower) / (upper - lower) * 2^24.  From the smallest normal level up that fraction is the part of
+// the fp32 mantissa below the format's, so adding what the draw leaves of the dropped bits' range and cutting does
+// it; below, |t| is brought to a fixed-point count of 2^-24 steps by one exact multiplication.
+__device__ __forceinline__ float convert_one_dither(float g, float m, float decay, const FmtDev& f, uint32_t R,
+                                                    uint32_t& sym, uint32_t& flags) {
+    const float v = __fmaf_rn(decay, m, g);
+    const uint32_t vb = __float_as_uint(v) & 0x7fffffffu;
+    const float t = __fmul_rn(v, f.scale);
+    const uint32_t tb = __float_as_uint(t);
+    const uint32_t a = tb & 0x7fffffffu;
+    uint32_t code;
+    float qmag;
+    if (a >= f.top_bits) {  // the largest level or beyond it (also +-Inf and NaN patterns, sorted out below)
+        flags |= (a > f.top_bits) ? 1u : 0u;
+        code = f.max_code;
+        qmag = __uint_as_float(f.top_bits);
+    } else if (a >= f.min_normal_bits) {
+        const uint32_t mask = (1u << f.drop) - 1u;
+        const uint32_t r = R >> (f.mant_bits + 1u);  // the draw on the grid of the dropped bits
+        code = ((a + (mask - r)) >> f.drop) - f.code_bias;  // one more iff the dropped bits exceed r
+        qmag = __uint_as_float((code + f.code_bias) << f.drop);
+    } else {
+        // |t| in units of 2^-24 of the step below the smallest normal level (2^(emin - M), or 2^emin without
+        // sub-normal levels): an exact product with a power of two, below 2^(24 + M)
+        const uint32_t step_exp = (f.min_normal_bits >> 23) - (f.flush ? 0u : f.mant_bits);  // biased exponent of the step
+        const float w = __fmul_rn(__uint_as_float(a), __uint_as_float((24u + 254u - step_exp) << 23));
+        const uint32_t wi = __float2uint_rz(w);
+        const uint32_t frac = (wi & 0xffffffu) + (__uint2float_rn(wi) != w ? 1u : 0u);
+        const uint32_t n = (wi >> 24) + (R < frac ? 1u : 0u);  // steps
+        code = f.flush ? n << f.mant_bits : n;
+        qmag = __fmul_rn(__uint2float_rn(n), __uint_as_float(step_exp << 23));
+    }
+    uint32_t sign = (code != 0u) ? (tb >> 31) : 0u;
+    float ghat = __fmul_rn(sign ? -qmag : qmag, f.inv_scale);
+    float m_new = __fsub_rn(v, ghat);
+    if (vb >= 0x7f800000u) {  // NaN is sent as zero, +-Inf as the boundary level; their memory restarts
+        flags = (flags & ~1u) | 2u;
+        m_new = 0.0f;
+        if (vb > 0x7f800000u) { code = 0u; sign = 0u; }
+    }
+    sym = (sign << f.mag_bits) | code;
+    return m_new;
 }
 
 // ------------------------------------------------------------------------------------------------

@@ -176,6 +176,8 @@ __global__ void __launch_bounds__(kThreads) prepare_kernel(PrepArgs a) {
         d.seg = k;
         d.cnt = (uint32_t)min((uint64_t)kC, sg.n_elem - c * kC);
         d.elem0 = sg.elem_off + c * kC;
+        d.cis = (uint32_t)c;
+        d.pad = 0;
         a.ws.chunk_desc[c_before + c] = d;
     }
     for (uint64_t t = (uint64_t)blockIdx.y * kThreads + tid; t < my_tiles; t += (uint64_t)gridDim.y * kThreads) {
@@ -351,21 +353,58 @@ __device__ __forceinline__ void add_counts(co3_result* r, uint32_t n_sat, uint32
     }
 }
 
+// Where a thread's eight elements lie, for the draws of a dithered conversion: the call's seed, client, layer, and
+// the place of the first of them inside the layer (a multiple of 8).
+struct Place {
+    uint32_t seed, client, layer;
+    uint64_t first;
+};
+
 // Correct + convert + memory update of 8 elements held in registers (Algorithm 1, client side).
 // kWhole: all eight are valid, so the branch-free converter may be used.  Symbols land in s[], the new memory
 // in mo[]; counters accumulate in n_sat / n_nf.
-template <bool kWhole>
+// kDither: the instance of the dithered entry points: one draw per element (four per block of the draw stream)
+// decides between the two levels around its value.
+template <bool kWhole, bool kDither>
 __device__ __forceinline__ void convert8(const float (&g)[8], const float (&m)[8], uint32_t nv, float decay,
-                                         const FmtDev& f, float (&mo)[8], uint32_t (&s)[8], uint32_t& n_sat,
-                                         uint32_t& n_nf) {
+                                         const FmtDev& f, const Place& at, float (&mo)[8], uint32_t (&s)[8],
+                                         uint32_t& n_sat, uint32_t& n_nf) {
+    if (kDither) {
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const uint64_t b = (at.first >> 2) + (uint32_t)h;
+            const uint4 r = philox4x32_10(make_uint4((uint32_t)b, (uint32_t)(b >> 32), at.client, at.layer), at.seed, 0u);
+            const uint32_t R[4] = {r.x >> 8, r.y >> 8, r.z >> 8, r.w >> 8};
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const int j = 4 * h + q;
+                uint32_t fl = 0;
+                mo[j] = convert_one_dither(g[j], m[j], decay, f, R[q], s[j], fl);
+                if ((uint32_t)j < nv) { n_sat += fl & 1u; n_nf += fl >> 1; }
+            }
+        }
+        return;
+    }
     bool redo = true;
     if (kWhole && f.fast) {
         bool beyond = false;
 #pragma unroll
         for (int j = 0; j < 8; ++j) mo[j] = convert_fast(g[j], m[j], decay, f, s[j], beyond);
-        redo = beyond;  // a saturating or non-finite input
+        redo = false;
+        if (beyond) {  // a saturating or non-finite input: the clamp above already gave a finite one its level and
+                       // memory, it only has to be counted; a NaN or an infinity sends the group through convert_one
+            const float top = __uint_as_float(f.top_bits);
+            uint32_t sat = 0;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const float v = __fmaf_rn(decay, m[j], g[j]);
+                redo |= !(fabsf(v) < __uint_as_float(0x7f800000u));
+                sat += (fabsf(__fmul_rn(v, f.scale)) > top) ? 1u : 0u;
+            }
+            if (!redo) n_sat += sat;
+        }
     }
-    if (redo) {  // generic formats, ragged groups, and groups that hold a saturating or non-finite input
+    if (redo) {  // generic formats, ragged groups, and groups that hold a non-finite input
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
             uint32_t fl = 0;
@@ -391,20 +430,32 @@ struct FeedItem {
     uint32_t chunk;   // chunk index inside the client
 };
 
-// Thread 0's position in the item sequence: item i of this block is item blockIdx.x + i * gridDim.x of the
-// batch, i.e. (client, chunk) advanced by gridDim.x chunks per step, without any 64-bit division.
+// Thread 0's position in the item sequence.  Items are numbered client-major (item = client * n_chunks + chunk)
+// and handed out in groups of `group` consecutive items: block b takes groups b, b + gridDim.x, ...  Consecutive
+// chunks mostly belong to one layer, so a block changes tables (and flushes its private histograms) rarely.  The
+// cursor moves by one item inside a group and by the distance to the block's next group at its end, both as
+// (whole clients, chunks) pairs worked out once: no 64-bit division per item.
 struct FeedCursor {
     uint32_t client, chunk;            // the item to publish next
-    uint32_t step_client, step_chunk;  // gridDim.x as (whole clients, chunks)
-    __device__ __forceinline__ void init(uint32_t n_chunks) {
-        client = blockIdx.x / n_chunks;
-        chunk = blockIdx.x % n_chunks;
-        step_client = gridDim.x / n_chunks;
-        step_chunk = gridDim.x % n_chunks;
+    uint32_t jump_client, jump_chunk;  // from the last item of a group to the first of the block's next group
+    uint32_t group, j;                 // items per group; place of the next item inside its group
+    __device__ __forceinline__ void init(uint32_t n_chunks, uint32_t grp) {
+        const uint64_t first = (uint64_t)blockIdx.x * grp, jump = (uint64_t)(gridDim.x - 1u) * grp + 1u;
+        client = (uint32_t)(first / n_chunks);
+        chunk = (uint32_t)(first % n_chunks);
+        jump_client = (uint32_t)(jump / n_chunks);
+        jump_chunk = (uint32_t)(jump % n_chunks);
+        group = grp;
+        j = 0;
     }
     __device__ __forceinline__ void advance(uint32_t n_chunks) {
-        client += step_client;
-        chunk += step_chunk;
+        if (++j < group) {
+            ++chunk;
+        } else {
+            j = 0;
+            client += jump_client;
+            chunk += jump_chunk;
+        }
         if (chunk >= n_chunks) { chunk -= n_chunks; ++client; }
     }
 };
@@ -511,13 +562,17 @@ struct ConvertArgs {
     uint8_t* sym_out;    // nullable
     uint64_t* hist_out;  // nullable
     co3_result* res;
+    uint32_t group;      // consecutive items a block takes at a time
+    uint32_t seed;       // key of the draw stream (dithered entry points)
     Ws ws;
 };
 
 constexpr int kHistCopies = 8;    // private histograms per block, spread over the lanes
 constexpr int kHistStride = 260;  // words between copies: shifts each copy by four banks
 
-template <bool kSym, bool kHist>
+// kMem: the new memory is stored (false: a dry pass that only counts symbols and leaves every input untouched).
+// kDither: the instance behind the dithered entry points (stochastic choice between the two levels around a value).
+template <bool kSym, bool kHist, bool kMem, bool kDither>
 __global__ void __launch_bounds__(kThreads, 3) convert_kernel(ConvertArgs a) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     Feed& fd = *reinterpret_cast<Feed*>(smem_raw);
@@ -527,14 +582,14 @@ __global__ void __launch_bounds__(kThreads, 3) convert_kernel(ConvertArgs a) {
     const uint32_t tid = threadIdx.x;
     const uint32_t n_chunks = ctrl->n_chunks;
     const FeedArgs fa{a.grad, a.mem, a.client_stride, a.n_clients};
-    if ((uint64_t)blockIdx.x >= (uint64_t)n_chunks * a.n_clients) return;
+    if ((uint64_t)blockIdx.x * a.group >= (uint64_t)n_chunks * a.n_clients) return;
 
     ChunkDesc next{};
     if (tid == 0) {
         mbar_init(&fd.bar[0], 1);
         mbar_init(&fd.bar[1], 1);
         fd.fail = 0u;
-        fd.cur.init(n_chunks);
+        fd.cur.init(n_chunks, a.group);
         next = a.ws.chunk_desc[fd.cur.chunk];
         feed_issue(fd, fa, a.ws, n_chunks, 0, next, true);
     }
@@ -577,11 +632,11 @@ __global__ void __launch_bounds__(kThreads, 3) convert_kernel(ConvertArgs a) {
         if (!ok) {
             hw_fail = true;
         } else if (it.tma) {
-            convert8<true>(g, m, 8, a.decay, f, mo, s, n_sat, n_nf);
-            store8_vec(a.mem + e, mo);
+            convert8<true, kDither>(g, m, 8, a.decay, f, Place{a.seed, it.client, it.d.seg, (uint64_t)it.d.cis * kC + i0}, mo, s, n_sat, n_nf);
+            if (kMem) store8_vec(a.mem + e, mo);
         } else if (nv) {
-            convert8<false>(g, m, nv, a.decay, f, mo, s, n_sat, n_nf);
-            store8_any(a.mem + e, nv, mo);
+            convert8<false, kDither>(g, m, nv, a.decay, f, Place{a.seed, it.client, it.d.seg, (uint64_t)it.d.cis * kC + i0}, mo, s, n_sat, n_nf);
+            if (kMem) store8_any(a.mem + e, nv, mo);
         }
         if (kSym && nv && ok) {
             if (nv == 8 && (reinterpret_cast<uintptr_t>(a.sym_out + e) & 7u) == 0) {
@@ -633,6 +688,8 @@ struct PackArgs {
     uint8_t* streams;
     size_t stream_capacity;
     co3_result* res;
+    uint32_t group;      // consecutive items a block takes at a time
+    uint32_t seed;       // key of the draw stream (dithered entry point)
     Ws ws;
 };
 
@@ -658,6 +715,7 @@ __device__ __forceinline__ void put_bits(uint32_t buf_addr, uint32_t end, uint64
     or_if_nonzero(last - 8u, __funnelshift_l(lo, hi, q));
     or_if_nonzero(last - 12u, __funnelshift_l(hi, 0u, q));
 }
+
 
 constexpr int kBitWords = kSlotWords;  // bit buffer of one chunk: one uint4 per thread
 
@@ -700,7 +758,7 @@ struct PackSmem {
 // kFromSym), their codewords, the block-wide scan of the lengths, and the bits ORed into the chunk's buffer.
 // kWhole: the chunk is complete (and, on the fused path, was delivered through the ring).
 // Returns the chunk's total bit count; `missing` reports a symbol without codeword.
-template <bool kFromSym, bool kWhole>
+template <bool kFromSym, bool kWhole, bool kDither>
 __device__ __forceinline__ uint32_t pack_item(const PackArgs& a, PackSmem& sm, const FeedArgs& fa, const FeedItem& it,
                                               uint32_t k, uint32_t& parity, uint32_t& enc_seg, uint32_t& n_sat,
                                               uint32_t& n_nf, bool& hw_fail, bool& missing, uint32_t& off_out) {
@@ -727,10 +785,10 @@ __device__ __forceinline__ uint32_t pack_item(const PackArgs& a, PackSmem& sm, c
 #pragma unroll
             for (int j = 0; j < 8; ++j) s[j] = 0u;
         } else if (kWhole) {
-            convert8<true>(g, m, 8, a.decay, f, mo, s, n_sat, n_nf);
+            convert8<true, kDither>(g, m, 8, a.decay, f, Place{a.seed, it.client, it.d.seg, (uint64_t)it.d.cis * kC + i0}, mo, s, n_sat, n_nf);
             store8_vec(a.mem + e, mo);
         } else if (nv) {
-            convert8<false>(g, m, nv, a.decay, f, mo, s, n_sat, n_nf);
+            convert8<false, kDither>(g, m, nv, a.decay, f, Place{a.seed, it.client, it.d.seg, (uint64_t)it.d.cis * kC + i0}, mo, s, n_sat, n_nf);
             store8_any(a.mem + e, nv, mo);
         }
     }
@@ -782,16 +840,17 @@ __device__ __forceinline__ void pack_out_set(const PackArgs& a, PackSmem& sm, ui
     sm.out[slot] = o;
 }
 
-template <bool kFromSym>
+// kDither: the instance behind the dithered entry point (see convert_kernel).
+template <bool kFromSym, bool kDither>
 __global__ void __launch_bounds__(kThreads, 3) pack_kernel(PackArgs a) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     PackSmem& sm = *reinterpret_cast<PackSmem*>(smem_raw);
-    const Ctrl* ctrl = a.ws.ctrl;
+    Ctrl* ctrl = a.ws.ctrl;
     if (ctrl->abort) return;
     const uint32_t tid = threadIdx.x;
     const uint32_t n_chunks = ctrl->n_chunks;
     const FeedArgs fa{a.grad, a.mem, a.client_stride, a.n_clients};
-    if ((uint64_t)blockIdx.x >= (uint64_t)n_chunks * a.n_clients) return;
+    if ((uint64_t)blockIdx.x * a.group >= (uint64_t)n_chunks * a.n_clients) return;
     const uint64_t sub_off = ctrl->sub_off;
 
     ChunkDesc next{};
@@ -799,7 +858,7 @@ __global__ void __launch_bounds__(kThreads, 3) pack_kernel(PackArgs a) {
         mbar_init(&sm.feed.bar[0], 1);
         mbar_init(&sm.feed.bar[1], 1);
         sm.feed.fail = 0u;
-        sm.feed.cur.init(n_chunks);
+        sm.feed.cur.init(n_chunks, a.group);
         next = a.ws.chunk_desc[sm.feed.cur.chunk];
         feed_issue(sm.feed, fa, a.ws, n_chunks, 0, next, !kFromSym);
         pack_out_set(a, sm, 0, sub_off);
@@ -830,8 +889,8 @@ __global__ void __launch_bounds__(kThreads, 3) pack_kernel(PackArgs a) {
         bool missing;
         uint32_t off, total;
         const bool whole = kFromSym ? it.d.cnt == (uint32_t)kC : it.tma != 0;
-        if (whole) total = pack_item<kFromSym, true>(a, sm, fa, it, k, parity, enc_seg, n_sat, n_nf, hw_fail, missing, off);
-        else total = pack_item<kFromSym, false>(a, sm, fa, it, k, parity, enc_seg, n_sat, n_nf, hw_fail, missing, off);
+        if (whole) total = pack_item<kFromSym, true, kDither>(a, sm, fa, it, k, parity, enc_seg, n_sat, n_nf, hw_fail, missing, off);
+        else total = pack_item<kFromSym, false, kDither>(a, sm, fa, it, k, parity, enc_seg, n_sat, n_nf, hw_fail, missing, off);
         const PackOut out = sm.out[k & 1u];
         if ((tid & 15u) == 0) out.sub[tid >> 4] = (uint16_t)off;
         if (__syncthreads_or(missing)) {  // bit buffer complete
@@ -2085,6 +2144,7 @@ bool ws_layout(uint64_t n_elem, uint32_t n_seg, uint32_t n_clients, WsLayout* L)
     L->n_chunks_max = (uint32_t)nc;
     size_t o = 0;
     L->ctrl = o;        o += up256(sizeof(Ctrl));
+    L->client_fail = o; o += up256(4 * (size_t)(n_clients ? n_clients : 1));  // directly behind ctrl: cleared with it
     L->first_chunk = o; o += up256(4 * ((size_t)n_seg + 1));
     L->chunk_desc = o;  o += up256(sizeof(ChunkDesc) * (size_t)nc);
     L->tile_desc = o;   o += up256(sizeof(TileDesc) * (size_t)nc);
@@ -2093,7 +2153,6 @@ bool ws_layout(uint64_t n_elem, uint32_t n_seg, uint32_t n_clients, WsLayout* L)
     L->dec_lut = o;     o += up256(2 * (size_t)kDecLut * n_seg);
     L->dec_sub = o;     o += up256(2 * (size_t)kSubLut * n_seg);
     L->val_lut = o;     o += up256(4 * 256 * (size_t)n_seg);
-    L->client_fail = o; o += up256(4 * (size_t)(n_clients ? n_clients : 1));
     L->chunk_bits = o;  o += up256(4 * (size_t)n_clients * nc);
     L->bit_prefix = o;  o += up256(8 * (size_t)n_clients * (nc + 1));
     L->n_ranges_max = (uint32_t)(nc / kRangeChunks + 1);
@@ -2140,16 +2199,22 @@ uint64_t fixed_part_bound(uint32_t n_seg, uint64_t n_chunks_max) {
     } while (0)
 
 // Blocks of a persistent kernel: enough to fill every SM at the kernel's occupancy, never more than the work.
+// grouped: items are handed out four consecutive ones at a time when that still leaves every block many groups
+// (the kernels with private histograms, which flush them when the layer changes; the others balance better one by one).
+constexpr uint32_t kItemGroup = 4;
+
 template <typename Kernel>
-int persistent_grid(Kernel kernel, size_t smem, uint64_t items, uint32_t* grid) {
+int persistent_grid(Kernel kernel, int threads, size_t smem, uint64_t items, bool grouped, uint32_t* grid, uint32_t* group) {
     int dev = 0, sms = 0, per_sm = 0;
     CO3_CUDA(cudaGetDevice(&dev));
     CO3_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
     CO3_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    CO3_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kThreads, smem));
+    CO3_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, threads, smem));
     if (per_sm < 1) return CO3_ERR_CUDA;
     const uint64_t want = (uint64_t)sms * (uint64_t)per_sm;
-    *grid = (uint32_t)(items < want ? items : want);
+    *group = (grouped && items >= 8ull * kItemGroup * want) ? kItemGroup : 1u;
+    const uint64_t groups = (items + *group - 1) / *group;
+    *grid = (uint32_t)(groups < want ? groups : want);
     return CO3_OK;
 }
 
@@ -2194,15 +2259,14 @@ int begin_call(const WsLayout& L, const Ws& ws, co3_result* res, uint32_t n_res,
                const co3_fmt* fmts, const co3_code* codes, const co3_seg* segs, uint32_t n_seg, uint64_t n_elem,
                uint32_t tile_chunks, uint32_t n_fail, const uint8_t* const* streams = nullptr,
                const uint8_t* single = nullptr, size_t stream_bytes = 0, uint32_t n_streams = 0) {
-    CO3_CUDA(cudaMemsetAsync(ws.ctrl, 0, sizeof(Ctrl), st));
+    // the call-wide state and the per-client failure marks lie side by side in the workspace: one clearing for both
+    CO3_CUDA(cudaMemsetAsync(ws.ctrl, 0, (L.client_fail - L.ctrl) + 4 * (size_t)(n_fail ? n_fail : 1), st));
     CO3_CUDA(cudaMemsetAsync(res, 0, sizeof(co3_result) * (size_t)n_res, st));
-    CO3_CUDA(cudaMemsetAsync(ws.client_fail, 0, 4 * (size_t)(n_fail ? n_fail : 1), st));
     PrepArgs pa{fmts, codes, segs, n_seg, n_elem, tile_chunks, res, n_res, n_streams ? 1u : 0u, streams, single, stream_bytes, n_streams, ws};
     // extra blocks per segment when segments are long (their chunk descriptors are written in parallel)
     const uint64_t per_seg = L.n_chunks_max / (n_seg ? n_seg : 1);
     const uint32_t helpers = (uint32_t)std::min<uint64_t>(128, per_seg / (8 * kThreads) + 1);
     CO3_LAUNCH(CO3_KERNEL_PREPARE, st, prepare_kernel<<<dim3(n_seg ? n_seg : 1, helpers), kThreads, 0, st>>>(pa));
-    (void)L;
     return CO3_OK;
 }
 
@@ -2256,7 +2320,8 @@ int decode_common(const uint8_t* const* streams, const uint8_t* single, size_t s
 int encode_common(const float* grad, float* mem, float decay, const uint8_t* sym, const co3_fmt* fmts,
                   const co3_code* codes, const co3_seg* segs, uint32_t n_seg, uint64_t n_elem, uint32_t n_clients,
                   uint64_t client_stride, uint8_t* streams_out, size_t stream_capacity, uint32_t chunk_syms,
-                  void* workspace, size_t workspace_bytes, co3_result* res, cudaStream_t st) {
+                  void* workspace, size_t workspace_bytes, co3_result* res, cudaStream_t st, bool dither = false,
+                  uint32_t seed = 0) {
     if (!codes || !res || !workspace || !streams_out || n_clients == 0 || n_clients > 65535u ||
         chunk_syms != (uint32_t)kC)
         return CO3_ERR_INVALID_ARG;
@@ -2273,18 +2338,19 @@ int encode_common(const float* grad, float* mem, float decay, const uint8_t* sym
     const int rc = begin_call(L, ws, res, n_clients, st, sym ? nullptr : fmts, codes, segs, n_seg, n_elem, 1, n_clients);
     if (rc != CO3_OK) return rc;
     if (L.n_chunks_max) {
-        PackArgs pa{grad, mem, decay, sym, client_stride, n_clients, streams_out, stream_capacity, res, ws};
+        PackArgs pa{grad, mem, decay, sym, client_stride, n_clients, streams_out, stream_capacity, res, 1u, seed, ws};
         const uint64_t items = (uint64_t)L.n_chunks_max * n_clients;
         uint32_t grid = 0;
-        if (sym) {
-            const int g = persistent_grid(pack_kernel<true>, sizeof(PackSmem), items, &grid);
-            if (g != CO3_OK) return g;
-            CO3_LAUNCH(CO3_KERNEL_PACK, st, pack_kernel<true><<<grid, kThreads, sizeof(PackSmem), st>>>(pa));
-        } else {
-            const int g = persistent_grid(pack_kernel<false>, sizeof(PackSmem), items, &grid);
-            if (g != CO3_OK) return g;
-            CO3_LAUNCH(CO3_KERNEL_PACK, st, pack_kernel<false><<<grid, kThreads, sizeof(PackSmem), st>>>(pa));
-        }
+#define CO3_PACK_CASE(S, D)                                                                                          \
+    {                                                                                                                \
+        const int g = persistent_grid(pack_kernel<S, D>, kThreads, sizeof(PackSmem), items, false, &grid, &pa.group); \
+        if (g != CO3_OK) return g;                                                                                   \
+        CO3_LAUNCH(CO3_KERNEL_PACK, st, pack_kernel<S, D><<<grid, kThreads, sizeof(PackSmem), st>>>(pa));            \
+    }
+        if (sym) CO3_PACK_CASE(true, false)
+        else if (dither) CO3_PACK_CASE(false, true)
+        else CO3_PACK_CASE(false, false)
+#undef CO3_PACK_CASE
     }
     // inputs beyond a few tiles of chunks per client: offsets by a two-level scan over many blocks
     const uint32_t two_level = L.n_chunks_max > 4u * kRangeChunks ? 1u : 0u;
@@ -2357,10 +2423,11 @@ int co3_stream_capacity_bytes(uint64_t n_elem, uint32_t n_seg, uint32_t chunk_sy
     return CO3_OK;
 }
 
-int co3_convert(const float* grad, float* mem, float decay, const co3_fmt* fmts, const co3_seg* segs, uint32_t n_seg,
-                uint64_t n_elem, uint32_t n_clients, uint64_t client_stride_elems, uint8_t* sym_out,
-                uint64_t* hist_out, co3_result* res, void* workspace, size_t workspace_bytes, void* stream) {
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
+static int convert_common(const float* grad, float* mem, bool store_mem, float decay, const co3_fmt* fmts,
+                          const co3_seg* segs, uint32_t n_seg, uint64_t n_elem, uint32_t n_clients,
+                          uint64_t client_stride_elems, uint8_t* sym_out, uint64_t* hist_out, co3_result* res,
+                          void* workspace, size_t workspace_bytes, cudaStream_t st, bool dither = false,
+                          uint32_t seed = 0) {
     if (!grad || !mem || !fmts || !res || !workspace || n_clients == 0 || n_clients > 65535u) return CO3_ERR_INVALID_ARG;
     if (!segs && n_seg) return CO3_ERR_INVALID_ARG;
     if (!aligned(grad, 16) || !aligned(mem, 16) || !aligned(workspace, 256) || !aligned(res, 8) ||
@@ -2375,22 +2442,64 @@ int co3_convert(const float* grad, float* mem, float decay, const co3_fmt* fmts,
     const int rc = begin_call(L, ws, res, n_clients, st, fmts, nullptr, segs, n_seg, n_elem, 1, 1);
     if (rc != CO3_OK) return rc;
     if (L.n_chunks_max == 0) return CO3_OK;
-    ConvertArgs ca{grad, mem, decay, client_stride_elems, n_clients, sym_out, hist_out, res, ws};
+    ConvertArgs ca{grad, mem, decay, client_stride_elems, n_clients, sym_out, hist_out, res, 1u, seed, ws};
     const uint64_t items = (uint64_t)L.n_chunks_max * n_clients;
     const size_t smem = sizeof(Feed) + (hist_out ? 4 * (size_t)kHistStride * kHistCopies : 0);
     uint32_t grid = 0;
-#define CO3_CONVERT_CASE(S, H)                                                                                       \
+#define CO3_CONVERT_CASE2(S, H, M, D)                                                                                \
     {                                                                                                                \
-        const int g = persistent_grid(convert_kernel<S, H>, smem, items, &grid);                                     \
+        const int g = persistent_grid(convert_kernel<S, H, M, D>, kThreads, smem, items, H, &grid, &ca.group);       \
         if (g != CO3_OK) return g;                                                                                   \
-        CO3_LAUNCH(CO3_KERNEL_CONVERT, st, convert_kernel<S, H><<<grid, kThreads, smem, st>>>(ca));                  \
+        CO3_LAUNCH(CO3_KERNEL_CONVERT, st, convert_kernel<S, H, M, D><<<grid, kThreads, smem, st>>>(ca));            \
     }
-    if (sym_out && hist_out) CO3_CONVERT_CASE(true, true)
-    else if (sym_out) CO3_CONVERT_CASE(true, false)
-    else if (hist_out) CO3_CONVERT_CASE(false, true)
-    else CO3_CONVERT_CASE(false, false)
+#define CO3_CONVERT_CASE(S, H, M)                  \
+    {                                              \
+        if (dither) CO3_CONVERT_CASE2(S, H, M, true) \
+        else CO3_CONVERT_CASE2(S, H, M, false)     \
+    }
+    if (!store_mem) CO3_CONVERT_CASE(false, true, false)
+    else if (sym_out && hist_out) CO3_CONVERT_CASE(true, true, true)
+    else if (sym_out) CO3_CONVERT_CASE(true, false, true)
+    else if (hist_out) CO3_CONVERT_CASE(false, true, true)
+    else CO3_CONVERT_CASE(false, false, true)
+#undef CO3_CONVERT_CASE2
 #undef CO3_CONVERT_CASE
     return CO3_OK;
+}
+
+int co3_convert(const float* grad, float* mem, float decay, const co3_fmt* fmts, const co3_seg* segs, uint32_t n_seg,
+                uint64_t n_elem, uint32_t n_clients, uint64_t client_stride_elems, uint8_t* sym_out,
+                uint64_t* hist_out, co3_result* res, void* workspace, size_t workspace_bytes, void* stream) {
+    return convert_common(grad, mem, true, decay, fmts, segs, n_seg, n_elem, n_clients, client_stride_elems, sym_out,
+                          hist_out, res, workspace, workspace_bytes, static_cast<cudaStream_t>(stream));
+}
+
+int co3_histogram(const float* grad, const float* mem, float decay, const co3_fmt* fmts, const co3_seg* segs,
+                  uint32_t n_seg, uint64_t n_elem, uint32_t n_clients, uint64_t client_stride_elems,
+                  uint64_t* hist_out, co3_result* res, void* workspace, size_t workspace_bytes, void* stream) {
+    if (!hist_out) return CO3_ERR_INVALID_ARG;
+    // the kernel instance without the memory store never writes through this pointer
+    return convert_common(grad, const_cast<float*>(mem), false, decay, fmts, segs, n_seg, n_elem, n_clients,
+                          client_stride_elems, nullptr, hist_out, res, workspace, workspace_bytes,
+                          static_cast<cudaStream_t>(stream));
+}
+
+int co3_convert_dither(const float* grad, float* mem, float decay, const co3_fmt* fmts, const co3_seg* segs,
+                       uint32_t n_seg, uint64_t n_elem, uint32_t n_clients, uint64_t client_stride_elems,
+                       uint32_t seed, uint8_t* sym_out, uint64_t* hist_out, co3_result* res, void* workspace,
+                       size_t workspace_bytes, void* stream) {
+    return convert_common(grad, mem, true, decay, fmts, segs, n_seg, n_elem, n_clients, client_stride_elems, sym_out,
+                          hist_out, res, workspace, workspace_bytes, static_cast<cudaStream_t>(stream), true, seed);
+}
+
+int co3_histogram_dither(const float* grad, const float* mem, float decay, const co3_fmt* fmts, const co3_seg* segs,
+                         uint32_t n_seg, uint64_t n_elem, uint32_t n_clients, uint64_t client_stride_elems,
+                         uint32_t seed, uint64_t* hist_out, co3_result* res, void* workspace, size_t workspace_bytes,
+                         void* stream) {
+    if (!hist_out) return CO3_ERR_INVALID_ARG;
+    return convert_common(grad, const_cast<float*>(mem), false, decay, fmts, segs, n_seg, n_elem, n_clients,
+                          client_stride_elems, nullptr, hist_out, res, workspace, workspace_bytes,
+                          static_cast<cudaStream_t>(stream), true, seed);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -2467,9 +2576,9 @@ int co3_fit_scale(const float* grad, const float* mem, float decay, co3_fmt* fmt
     // the per-(chunk, client) partial sums take the place of the encoder's chunk slots (16 of 4096 bytes each)
     // and behind them the per-layer range sums and completion counters of the fit
     double2* part = reinterpret_cast<double2*>(ws.slots);
+    static_assert(16 * (kFitRanges + 1) + 4 <= 4 * kSlotWords, "the fit's scratch fits in the slots of n_seg chunks");
     double2* range_part = part + (size_t)n_clients * L.n_chunks_max;
     uint32_t* range_done = reinterpret_cast<uint32_t*>(range_part + (size_t)n_seg * kFitRanges);
-    static_assert(16 * (kFitRanges + 1) + 4 <= 4 * kSlotWords, "the fit's scratch fits in the slots of n_seg chunks");
     CO3_CUDA(cudaMemsetAsync(range_done, 0, 4 * (size_t)n_seg, st));
     FitArgs fa{grad, mem, decay, client_stride_elems, n_clients, fmts, segs, n_seg, log_tab, seg_tab, n_tab, n_beta,
                beta0, dbeta, stats_out, part, range_part, range_done, res, ws};
@@ -2537,6 +2646,16 @@ int co3_encode(const float* grad, float* mem, float decay, const co3_fmt* fmts, 
     return encode_common(grad, mem, decay, nullptr, fmts, codes, segs, n_seg, n_elem, n_clients, client_stride_elems,
                          streams_out, stream_capacity, chunk_syms, workspace, workspace_bytes, res,
                          static_cast<cudaStream_t>(stream));
+}
+
+int co3_encode_dither(const float* grad, float* mem, float decay, const co3_fmt* fmts, const co3_code* codes,
+                      const co3_seg* segs, uint32_t n_seg, uint64_t n_elem, uint32_t n_clients,
+                      uint64_t client_stride_elems, uint32_t seed, uint8_t* streams_out, size_t stream_capacity,
+                      uint32_t chunk_syms, void* workspace, size_t workspace_bytes, co3_result* res, void* stream) {
+    if (!grad || !mem || !fmts) return CO3_ERR_INVALID_ARG;
+    return encode_common(grad, mem, decay, nullptr, fmts, codes, segs, n_seg, n_elem, n_clients, client_stride_elems,
+                         streams_out, stream_capacity, chunk_syms, workspace, workspace_bytes, res,
+                         static_cast<cudaStream_t>(stream), true, seed);
 }
 
 int co3_encode_symbols(const uint8_t* sym, const co3_code* codes, const co3_seg* segs, uint32_t n_seg, uint64_t n_elem,

@@ -83,6 +83,15 @@ class Co3Session:
             return None
         return self.hist.cpu().numpy().astype(np.uint64).reshape(-1, 256)[:self.n_seg]
 
+    def histogram_only(self, grads: torch.Tensor, mems: torch.Tensor, stream=None, to_host: bool = True):
+        """The same counts without running the round: neither `mems` nor anything else is written."""
+        st = B.co3_histogram(grads, mems, self.decay, self.fmts, self.segs, self.n_seg, self.n_elem, self.n_clients,
+                             self.stride, self.hist, self.res_enc, self.workspace, stream)
+        self._check(st, "co3_histogram")
+        if not to_host:
+            return None
+        return self.hist.cpu().numpy().astype(np.uint64).reshape(-1, 256)[:self.n_seg]
+
     def set_codes_from_weights(self, weights: np.ndarray) -> None:
         """weights: uint64[n_seg][256] (histogram counts or model weights); one Huffman code per layer."""
         codes = np.zeros(self.n_seg, dtype=B.CODE_DTYPE)

@@ -105,25 +105,33 @@ class Gpu:
         c = self.case
         return np.stack([t[u * c.stride:u * c.stride + c.n_elem].cpu().numpy() for u in range(c.n_clients)])
 
-    def convert(self, grads, mems, want_sym=True, want_hist=True):
+    def convert(self, grads, mems, want_sym=True, want_hist=True, dither_seed=None):
         c = self.case
         g, m = self._buf(grads), self._buf(mems)
         sym = torch.full((c.n_clients * c.stride + 8,), 0xEE, dtype=torch.uint8, device="cuda") if want_sym else None
         hist = torch.full((max(1, c.n_seg) * 256,), 7, dtype=torch.int64, device="cuda") if want_hist else None
-        st = co3.co3_convert(g, m, c.decay, self.fmts, self.segs, c.n_seg, c.n_elem, c.n_clients, c.stride, sym, hist,
-                             self.res, self.ws)
+        if dither_seed is None:
+            st = co3.co3_convert(g, m, c.decay, self.fmts, self.segs, c.n_seg, c.n_elem, c.n_clients, c.stride, sym,
+                                 hist, self.res, self.ws)
+        else:
+            st = co3.co3_convert_dither(g, m, c.decay, self.fmts, self.segs, c.n_seg, c.n_elem, c.n_clients, c.stride,
+                                        dither_seed, sym, hist, self.res, self.ws)
         torch.cuda.synchronize()
         res = co3.read_results(self.res, c.n_clients)
         return dict(status=st, res=res, mem=self._unbuf(m),
                     sym=self._unbuf(sym) if want_sym else None,
                     hist=hist.cpu().numpy().astype(np.uint64).reshape(-1, 256)[:c.n_seg] if want_hist else None)
 
-    def encode(self, grads, mems, codes, capacity=None, from_sym=None):
+    def encode(self, grads, mems, codes, capacity=None, from_sym=None, dither_seed=None):
         c = self.case
         cap = self.capacity if capacity is None else capacity
         streams = torch.full((c.n_clients * cap + 64,), 0xA5, dtype=torch.uint8, device="cuda")
         codes_d = self.codes_dev(codes)
-        if from_sym is None:
+        if from_sym is None and dither_seed is not None:
+            g, m = self._buf(grads), self._buf(mems)
+            st = co3.co3_encode_dither(g, m, c.decay, self.fmts, codes_d, self.segs, c.n_seg, c.n_elem, c.n_clients,
+                                       c.stride, dither_seed, streams, cap, self.ws, self.res)
+        elif from_sym is None:
             g, m = self._buf(grads), self._buf(mems)
             st = co3.co3_encode(g, m, c.decay, self.fmts, codes_d, self.segs, c.n_seg, c.n_elem, c.n_clients, c.stride,
                                 streams, cap, self.ws, self.res)

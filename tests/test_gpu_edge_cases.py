@@ -136,7 +136,7 @@ def test_symbol_without_codeword():
 
 def test_invalid_descriptors_are_refused_on_the_device():
     g = gennorm(4096, 1.0, 1e-3, seed=1).numpy()[None, :]
-    for bad in [(1, 3, 0, 1.0, 1.0), (4, 4, 0, 1.0, 1.0), (4, 3, 2, 1.0, 1.0), (4, 3, 0, 0.0, 1.0),
+    for bad in [(1, 3, 0, 1.0, 1.0), (4, 4, 0, 1.0, 1.0), (4, 3, 4, 1.0, 1.0), (4, 3, 0, 0.0, 1.0),
                 (4, 3, 0, float("inf"), 1.0), (4, 3, 0, 1.0, float("nan")), (7, 0, 0, 1.0, 3e38)]:
         case = Case([4096], [bad], n_clients=1)
         out = Gpu(case).convert(g, np.zeros_like(g))
