@@ -409,6 +409,33 @@ def measure(cfg, sizes, fmts, clients, dev, rank, world, steps, warmup, peak, he
     er, dr = check()
     ms = max_over_ranks(ms, world, dev)
 
+    # ---- small workloads are launch-bound: the same step once more as a CUDA-graph replay
+    graph_ms = None
+    if flush and world == 1:
+        try:
+            side = torch.cuda.Stream(device=dev)
+            graph = torch.cuda.CUDAGraph()
+
+            def captured():     # the calls take the capturing stream (the current one)
+                if fit:
+                    sess.histogram(grads[0], mems, None, sym_step, to_host=False)
+                    sess.set_codes_from_histogram_device(None)
+                    sess.encode_symbols(sym_step, None)
+                else:
+                    sess.encode(grads[0], mems, None)
+                sess.decode_aggregate(None)
+
+            with torch.cuda.graph(graph, stream=side):
+                captured()
+            torch.cuda.synchronize()
+            for _ in range(3):
+                graph.replay()
+            graph_ms = timed.run(lambda i: graph.replay(), steps) / steps
+            check()
+        except Exception as exc:     # a capture that fails must not take the benchmark down
+            graph_ms = "capture failed: %s" % str(exc)[:120]
+            torch.cuda.synchronize()
+
     # ---- per-kernel times: the encode calls and the decode calls again, an event pair around every launch
     co3.co3_profile_enable(True)
     timed.run(lambda i: encode_on(grads[(warmup + i) % n_rounds]), steps)
@@ -449,6 +476,8 @@ def measure(cfg, sizes, fmts, clients, dev, rank, world, steps, warmup, peak, he
         "decode_call": dict(call_row(dec_ms, alg_dec), kernels=dec_rows),
         "launches_per_step": launches,
     }
+    if graph_ms is not None:
+        row["cuda_graph_replay_ms_per_step"] = graph_ms
     if "compact" in enc_rows:   # the slots pack leaves behind are read and written once more: not algorithmic
         row["encode_call"]["non_algorithmic_gb"] = 2.0 * container / 1e9
     state = dict(sess=sess, grads=grads, mems=mems, stream=stream, step_on=step_on, check=check, barrier=barrier,

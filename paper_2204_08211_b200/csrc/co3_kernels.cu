@@ -573,7 +573,7 @@ constexpr int kHistStride = 260;  // words between copies: shifts each copy by f
 // kMem: the new memory is stored (false: a dry pass that only counts symbols and leaves every input untouched).
 // kDither: the instance behind the dithered entry points (stochastic choice between the two levels around a value).
 template <bool kSym, bool kHist, bool kMem, bool kDither>
-__global__ void __launch_bounds__(kThreads, 3) convert_kernel(ConvertArgs a) {
+__global__ void __launch_bounds__(kThreads, (kMem || kDither) ? 3 : 4) convert_kernel(ConvertArgs a) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     Feed& fd = *reinterpret_cast<Feed*>(smem_raw);
     uint32_t* s_hist = reinterpret_cast<uint32_t*>(smem_raw + sizeof(Feed));

@@ -55,6 +55,31 @@ def test_convert_special_values(E, M, flush):
         assert np.array_equal(out["hist"], oracle_hist(case, syms))
 
 
+@pytest.mark.parametrize("E,M", FORMATS)
+@pytest.mark.parametrize("flush", [False, True])
+def test_encode_special_values_through_the_fused_path(E, M, flush):
+    """The same values through co3_encode, whole chunks of them (the path that converts and codes in one pass, with
+    its own converter for complete chunks): every level, midpoint and fp32 neighbour, then the non-finite ones."""
+    for scale, decay in ((1.0, 0.0), (5317.4585, 0.0), (1.37, 0.5)):
+        ft = fmt_tuple(E, M, scale, flush)
+        ofmt = oracle.Fmt(E, M, int(flush), ft[3], ft[4])
+        x = _special_values(ofmt)
+        finite = x[np.isfinite(x)]
+        reps = -(-6200 // finite.size)
+        g = np.concatenate([np.tile(finite, reps), x]).astype(np.float32)[None, :]
+        case = Case([g.size], [ft], 1, decay=decay)
+        m0 = (gennorm(g.size, 1.0, 1e-3 / scale, seed=77).numpy() * (decay != 0.0)).astype(np.float32)[None, :]
+        mem_o = m0.copy()
+        syms, ghats, nsat, nnf = oracle_convert(case, g, mem_o)
+        codes = oracle_codes(case, oracle_hist(case, syms))
+        want = oracle_encode(case, syms, codes)
+        out = Gpu(case).encode(g, m0, codes)
+        assert out["status"] == co3.OK and out["guard_ok"]
+        assert same_bits(out["mem"], mem_o)
+        assert np.array_equal(out["streams"][0], want[0][1])
+        assert out["res"][0]["n_saturated"] == nsat[0] and out["res"][0]["n_nonfinite"] == nnf[0]
+
+
 @pytest.mark.parametrize("n", [0, 1, 2, 31, 32, 33, 4095, 4096, 4097, 50001])
 def test_convert_sizes_and_rounds(n):
     ft = fmt_tuple(4, 3, *scale_for(4, 3, 1.0, 1e-3)[:1])
