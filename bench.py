@@ -33,7 +33,7 @@ NOMINAL_HBM_GBS = 8000.0     # the peak the metric is defined against; fractions
 # dram__bytes_read.sum + dram__bytes_write.sum per element of one launch, from the ncu captures summarised under
 # profiles/ (taken on a 10-client case; traffic grows in proportion to the elements of a launch).  None: the kernel
 # has changed since its counters were taken.
-NCU_TRAFFIC_BYTES_PER_ELEMENT = {"pack": None, "decode": None, "convert": None}
+NCU_TRAFFIC_BYTES_PER_ELEMENT = {"pack": 12.529, "decode": 1.044, "convert": 12.577}   # decode: per client and element
 RANK_SEED_STRIDE = 100_000   # ranks draw their synthetic clients from disjoint seed ranges
 L2_BYTES = 126e6
 
@@ -574,6 +574,47 @@ def standalone_kernels(state, cfg, clients, steps, warmup, peak):
     return out
 
 
+def uniform_symbol_decode(dev, steps, warmup, peak):
+    """Decoding when the chunks' payloads do not fit the decoder's shared-memory staging pool: symbols uniform over
+    the 239 symbols of [1,4,3] (7.9 bit each), 11.2 M per client, one and ten clients."""
+    import torch
+    import paper_2204_08211_b200 as co3
+    from paper_2204_08211_b200.session import Co3Session
+    n = 11_181_642
+    out = {}
+    for clients in (1, 10):
+        sess = Co3Session([n], [(4, 3, 0, 1.0, 1.0)], clients, 0.9, dev)
+        valid = np.array([c | (sg << 7) for sg in (0, 1) for c in range(120) if not (sg and c == 0)], dtype=np.uint8)
+        rng = np.random.default_rng(0)
+        sym = torch.from_numpy(valid[rng.integers(0, valid.size, size=clients * sess.stride)]).to(dev)
+        hist = np.zeros((1, 256), dtype=np.uint64)
+        hist[0, valid] = 1000
+        sess.set_codes_from_weights(hist)
+        sess.encode_symbols(sym)
+        for _ in range(warmup):
+            sess.decode_aggregate()
+        torch.cuda.synchronize()
+        er = sess.encode_results()
+        if (er["status"] != co3.OK).any():
+            raise RuntimeError("device status (uniform symbols): %s" % er["status"])
+        co3.co3_profile_enable(True)
+        for _ in range(steps):
+            sess.decode_aggregate()
+        n_l, tot = co3.co3_profile_read()["decode"]
+        co3.co3_profile_enable(False)
+        if sess.decode_result()["status"][0] != co3.OK:
+            raise RuntimeError("device status after decode (uniform symbols)")
+        gb = (4.0 * n + float(er["container_bytes"].astype(np.float64).sum())) / 1e9
+        gbs = gb / (tot / n_l * 1e-3)
+        out["decode_uniform_symbols_%dclient%s" % (clients, "s" if clients > 1 else "")] = {
+            "ms_per_call": tot / n_l, "launches_per_call": 1.0, "algorithmic_gb_per_call": gb, "achieved_gbs": gbs,
+            "frac_of_measured": gbs / peak, "frac_of_8tbs": gbs / NOMINAL_HBM_GBS,
+            "mean_code_bits": float(er["payload_bits"].astype(np.float64).sum()) / (clients * n),
+            "note": "payloads read in place from global memory (they exceed the staging pool); 11.2 M symbols per client"}
+        del sess, sym
+    return out
+
+
 def end_to_end(state, clients, steps, world, dev):
     """Pinned host gradients in, averaged gradient out, every step, through the same calls."""
     import torch
@@ -660,6 +701,10 @@ def run_ours(args):
     del state
     gc.collect()
     torch.cuda.empty_cache()
+    if world == 1 and not args.no_table:
+        alone.update(uniform_symbol_decode(dev, args.steps, args.warmup, peak))
+    gc.collect()
+    torch.cuda.empty_cache()
 
     table = []
     if not args.no_table and world == 1:
@@ -681,7 +726,7 @@ def run_ours(args):
     kern = dict(row["encode_call"]["kernels"], **row["decode_call"]["kernels"])
     dom = max((k for k in ("pack", "decode", "convert") if k in kern), key=lambda k: kern[k]["ms_per_call"])
     per_elem = NCU_TRAFFIC_BYTES_PER_ELEMENT.get(dom)
-    traffic_units = n_elem if dom == "decode" else n_elem * clients
+    traffic_units = n_elem * clients
     roofline = {"kernel": dom + "_kernel", "bound": "hbm", "achieved": kern[dom]["achieved_gbs"], "peak": peak,
                 "unit": "GB/s", "frac": kern[dom]["frac_of_measured"], "frac_of_8tbs": kern[dom]["frac_of_8tbs"],
                 "traffic": per_elem * traffic_units if per_elem is not None else None,
