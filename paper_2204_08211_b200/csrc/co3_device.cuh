@@ -52,8 +52,9 @@ struct TileDesc {
     uint32_t pad;
 };
 
-// Converter constants of one segment, derived from co3_fmt by the prepare kernel.
-struct FmtDev {
+// Converter constants of one segment, derived from co3_fmt by the prepare kernel.  (16-byte alignment: a thread
+// fetches its copy from shared memory with a few wide loads.)
+struct alignas(16) FmtDev {
     uint32_t mant_bits;        // M
     uint32_t mag_bits;         // E + M
     uint32_t fast;             // 1: M >= 1 and sub-normal levels kept, the branch-free converter applies

@@ -365,10 +365,14 @@ struct Place {
 // in mo[]; counters accumulate in n_sat / n_nf.
 // kDither: the instance of the dithered entry points: one draw per element (four per block of the draw stream)
 // decides between the two levels around its value.
+// ring_g / ring_m (kWhole only): the thread's eight gradient and memory values in the shared-memory ring, from which
+// the rare second look at a group reads them again, so that the registers holding them are free once the first
+// look is done.
 template <bool kWhole, bool kDither>
 __device__ __forceinline__ void convert8(const float (&g)[8], const float (&m)[8], uint32_t nv, float decay,
                                          const FmtDev& f, const Place& at, float (&mo)[8], uint32_t (&s)[8],
-                                         uint32_t& n_sat, uint32_t& n_nf) {
+                                         uint32_t& n_sat, uint32_t& n_nf, const float* ring_g = nullptr,
+                                         const float* ring_m = nullptr) {
     if (kDither) {
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
@@ -385,25 +389,43 @@ __device__ __forceinline__ void convert8(const float (&g)[8], const float (&m)[8
         }
         return;
     }
-    bool redo = true;
     if (kWhole && f.fast) {
         bool beyond = false;
 #pragma unroll
         for (int j = 0; j < 8; ++j) mo[j] = convert_fast(g[j], m[j], decay, f, s[j], beyond);
-        redo = false;
         if (beyond) {  // a saturating or non-finite input: the clamp above already gave a finite one its level and
                        // memory, it only has to be counted; a NaN or an infinity sends the group through convert_one
             const float top = __uint_as_float(f.top_bits);
+            float g2[8], m2[8];
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const float4 x = reinterpret_cast<const float4*>(ring_g)[h], y = reinterpret_cast<const float4*>(ring_m)[h];
+                g2[4 * h] = x.x; g2[4 * h + 1] = x.y; g2[4 * h + 2] = x.z; g2[4 * h + 3] = x.w;
+                m2[4 * h] = y.x; m2[4 * h + 1] = y.y; m2[4 * h + 2] = y.z; m2[4 * h + 3] = y.w;
+            }
             uint32_t sat = 0;
+            bool again = false;
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
-                const float v = __fmaf_rn(decay, m[j], g[j]);
-                redo |= !(fabsf(v) < __uint_as_float(0x7f800000u));
+                const float v = __fmaf_rn(decay, m2[j], g2[j]);
+                again |= !(fabsf(v) < __uint_as_float(0x7f800000u));
                 sat += (fabsf(__fmul_rn(v, f.scale)) > top) ? 1u : 0u;
             }
-            if (!redo) n_sat += sat;
+            if (!again) {
+                n_sat += sat;
+            } else {
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    uint32_t fl = 0;
+                    mo[j] = convert_one(g2[j], m2[j], decay, f, s[j], fl);
+                    n_sat += fl & 1u;
+                    n_nf += fl >> 1;
+                }
+            }
         }
+        return;
     }
+    const bool redo = true;
     if (redo) {  // generic formats, ragged groups, and groups that hold a non-finite input
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
@@ -421,7 +443,7 @@ __device__ __forceinline__ void convert8(const float (&g)[8], const float (&m)[8
 // of a two-stage shared-memory ring, completed on that stage's mbarrier.  Chunks that are short or not
 // 16-byte aligned are not copied; their threads load from global memory directly.
 // ------------------------------------------------------------------------------------------------
-struct FeedItem {
+struct alignas(16) FeedItem {
     ChunkDesc d;
     uint64_t base;    // index of the chunk's first element from the batch base pointer
     uint32_t client;
@@ -632,7 +654,8 @@ __global__ void __launch_bounds__(kThreads, (kMem || kDither) ? 3 : 4) convert_k
         if (!ok) {
             hw_fail = true;
         } else if (it.tma) {
-            convert8<true, kDither>(g, m, 8, a.decay, f, Place{a.seed, it.client, it.d.seg, (uint64_t)it.d.cis * kC + i0}, mo, s, n_sat, n_nf);
+            convert8<true, kDither>(g, m, 8, a.decay, f, Place{a.seed, it.client, it.d.seg, (uint64_t)it.d.cis * kC + i0}, mo, s, n_sat, n_nf,
+                                    &fd.g[k & 1u][i0], &fd.m[k & 1u][i0]);
             if (kMem) store8_vec(a.mem + e, mo);
         } else if (nv) {
             convert8<false, kDither>(g, m, nv, a.decay, f, Place{a.seed, it.client, it.d.seg, (uint64_t)it.d.cis * kC + i0}, mo, s, n_sat, n_nf);
@@ -739,7 +762,7 @@ __device__ __forceinline__ uint32_t block_exclusive_scan_once(uint32_t x, uint32
 }
 
 // Where the results of one work item go, worked out once per item by thread 0.
-struct PackOut {
+struct alignas(16) PackOut {
     uint16_t* sub;       // the chunk's 16 sub-chunk offsets in the client's container
     uint32_t* slot;      // the chunk's worst-case slot in the workspace
     uint32_t* chunk_bits;
@@ -785,7 +808,8 @@ __device__ __forceinline__ uint32_t pack_item(const PackArgs& a, PackSmem& sm, c
 #pragma unroll
             for (int j = 0; j < 8; ++j) s[j] = 0u;
         } else if (kWhole) {
-            convert8<true, kDither>(g, m, 8, a.decay, f, Place{a.seed, it.client, it.d.seg, (uint64_t)it.d.cis * kC + i0}, mo, s, n_sat, n_nf);
+            convert8<true, kDither>(g, m, 8, a.decay, f, Place{a.seed, it.client, it.d.seg, (uint64_t)it.d.cis * kC + i0}, mo, s, n_sat, n_nf,
+                                    &sm.feed.g[k & 1u][i0], &sm.feed.m[k & 1u][i0]);
             store8_vec(a.mem + e, mo);
         } else if (nv) {
             convert8<false, kDither>(g, m, nv, a.decay, f, Place{a.seed, it.client, it.d.seg, (uint64_t)it.d.cis * kC + i0}, mo, s, n_sat, n_nf);
@@ -1178,6 +1202,8 @@ __device__ __forceinline__ const uint8_t* stream_of(const DecArgs& a, uint32_t u
 }
 
 constexpr int kMaxPairs = 16;          // (chunk, client) pairs decoded side by side in one block
+constexpr int kMultiPairs = 20;        // the same when the clients come in several batches (one chunk per block)
+constexpr int kMultiThreads = 16 * kMultiPairs;
 constexpr int kPaySlotWords = 456;     // staging per pair: 7 bits/symbol plus alignment; larger chunks are read in place
 constexpr int kPaySlack = 72;          // words a reader may run past its chunk before the end check
 
@@ -1189,13 +1215,13 @@ struct DecSmem {
     uint64_t bar;                          // completion barrier of the bulk copies of one batch
     uint32_t tile_elems;                   // elements of the tile: full chunks and the last one's count
     uint32_t pad;
-    uint64_t chunk_elem0[kMaxPairs];       // first element of each chunk of the tile
-    const uint32_t* pair_src[kMaxPairs];   // the pair's first payload word in global memory
-    uint32_t pair_off[kMaxPairs];          // staged pairs: index of that word in pay[]
-    uint32_t pair_words[kMaxPairs];
-    uint32_t pair_staged[kMaxPairs];
-    uint32_t pair_cnt[kMaxPairs];
-    uint16_t sub[kMaxPairs][kSubs];        // sub-chunk bit offsets of each pair
+    uint64_t chunk_elem0[kMultiPairs];       // first element of each chunk of the tile
+    const uint32_t* pair_src[kMultiPairs];   // the pair's first payload word in global memory
+    uint32_t pair_off[kMultiPairs];          // staged pairs: index of that word in pay[]
+    uint32_t pair_words[kMultiPairs];
+    uint32_t pair_staged[kMultiPairs];
+    uint32_t pair_cnt[kMultiPairs];
+    uint16_t sub[kMultiPairs][kSubs];        // sub-chunk bit offsets of each pair
 };
 static_assert(sizeof(DecSmem) % 16 == 0 && offsetof(DecSmem, sub) % 16 == 0, "dynamic arrays behind DecSmem must stay 16-byte aligned");
 
@@ -1321,6 +1347,20 @@ __device__ __forceinline__ uint32_t sum_word(const float* __restrict__ val, cons
     return symw;
 }
 
+// The same for one half of the word (symbols 2 * half and 2 * half + 1): the batched decoder of many clients splits
+// every word between two threads so that the whole block takes part in the sum.
+__device__ __forceinline__ void sum_half(const float* __restrict__ val, const uint32_t* __restrict__ sym, uint32_t s,
+                                         uint32_t j, uint32_t half, uint32_t nb, float (&acc)[2]) {
+    const uint32_t* row = sym + s * kPhaseWords;
+    const uint32_t rot = j + (s >> 2), sh = 16u * half;
+#pragma unroll 2
+    for (uint32_t p = 0; p < nb; ++p, row += kPairPhaseWords) {
+        const uint32_t symw = row[(rot + 4u * (p & 1u)) & (kPhaseWords - 1)] >> sh;
+        acc[0] = __fadd_rn(acc[0], val[symw & 0xffu]);
+        acc[1] = __fadd_rn(acc[1], val[(symw >> 8) & 0xffu]);
+    }
+}
+
 // Where a tile's results go.  The chunks of a tile follow one another in one segment and all but the last
 // are full, so element e of the tile (chunk index * kC + place in the chunk) is element e behind the tile's
 // first one in the output as well.
@@ -1382,16 +1422,46 @@ __device__ __forceinline__ void write_word(const TileOut& to, uint32_t e, const 
     }
 }
 
+// write_word for two elements (e even, below to.n_elem): averages and stores them, and applies the update.
+__device__ __forceinline__ void write_half(const TileOut& to, uint32_t e, const float (&acc)[2]) {
+    const uint32_t nv = min(2u, to.n_elem - e);
+    float r[2];
+    if (to.pow2) {
+        r[0] = __fmul_rn(acc[0], to.inv);
+        r[1] = __fmul_rn(acc[1], to.inv);
+    } else {
+        r[0] = __fdiv_rn(acc[0], to.u);
+        r[1] = __fdiv_rn(acc[1], to.u);
+    }
+    if (to.out) {
+        float* o = to.out + e;
+        if (nv == 2 && to.out16) *reinterpret_cast<float2*>(o) = make_float2(r[0], r[1]);
+        else for (uint32_t q = 0; q < nv; ++q) o[q] = r[q];
+    }
+    if (to.params) {  // w <- w - lr * avg: one multiplication and one subtraction, each rounded on its own
+        float* w = to.params + e;
+        if (nv == 2 && to.params16) {
+            float2 x = *reinterpret_cast<const float2*>(w);
+            x.x = __fsub_rn(x.x, __fmul_rn(to.lr, r[0]));
+            x.y = __fsub_rn(x.y, __fmul_rn(to.lr, r[1]));
+            *reinterpret_cast<float2*>(w) = x;
+        } else {
+            for (uint32_t q = 0; q < nv; ++q) w[q] = __fsub_rn(w[q], __fmul_rn(to.lr, r[q]));
+        }
+    }
+}
+
 // One block decodes a tile of G chunks for B clients at a time.  Warp 0 looks up where each (chunk, client)
 // pair's payload lies and starts one bulk copy per pair into shared memory (plus the segment's tables);
 // then 16 threads per pair (one per sub-chunk) decode into a symbol buffer, and finally every thread sums
-// its share of the tile over the clients in client order.  kMulti: more clients than fit side by side
-// (B = 16, G = 1): the partial sums stay in registers between batches.  kSingle: one client, nothing to sum.
+// its share of the tile over the clients in client order.  kMulti: more clients than fit side by side: they
+// come in equal batches of 16 to 20 (G = 1), the partial sums stay in registers between batches, and every symbol
+// word is summed by two threads (two symbols each).  kSingle: one client, nothing to sum.
 template <bool kMulti, bool kSingle>
-__global__ void __launch_bounds__(kThreads, 4) decode_kernel(DecArgs a) {
+__global__ void __launch_bounds__(kMulti ? kMultiThreads : kThreads, kMulti ? 3 : 4) decode_kernel(DecArgs a) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     DecSmem& sm = *reinterpret_cast<DecSmem*>(smem_raw);
-    const uint32_t B = kMulti ? 16u : (kSingle ? 1u : a.B), G = kMulti ? 1u : a.G;
+    const uint32_t B = kSingle ? 1u : a.B, G = kMulti ? 1u : a.G;
     const uint32_t n_pairs = B * G, n_thr = 16u * n_pairs;
     uint32_t* const sm_sym = reinterpret_cast<uint32_t*>(smem_raw + sizeof(DecSmem));
     uint32_t* const sm_pay = sm_sym + n_pairs * kPairPhaseWords;
@@ -1407,7 +1477,7 @@ __global__ void __launch_bounds__(kThreads, 4) decode_kernel(DecArgs a) {
     const uint16_t* sub_tab = a.ws.dec_sub + (size_t)td.seg * kSubLut;
 
     if (tid == 0) mbar_init(&sm.bar, 1);
-    float carry[kPhases][4];  // running sums across client batches (kMulti only)
+    float carry[kPhases][2];  // running sums across client batches (kMulti only)
     TileOut to;
     to.u = (float)a.n_clients;
     to.pow2 = (a.n_clients & (a.n_clients - 1u)) == 0;
@@ -1527,18 +1597,18 @@ __global__ void __launch_bounds__(kThreads, 4) decode_kernel(DecArgs a) {
             //      tile's phase is word (s, j) of chunk cl and starts at element e of the tile
             static_assert(kPairPhaseWords == 128 && kPhaseWords == 8 && kC == 2048 && kS == 128, "shifts below");
             if (kMulti) {
-                if (tid < (uint32_t)kPairPhaseWords) {
-                    const uint32_t s = tid >> 3, j = tid & 7u;
-                    const uint32_t e = (s << 7) + ph * kPhaseSyms + (j << 2);
-                    float acc[4];
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) acc[q] = first_batch ? 0.0f : carry[ph][q];
-                    const uint32_t symw = sum_word(sm.val, sm_sym, 0, s, j, B, nb, acc);
+                if (tid < 2u * kPairPhaseWords) {  // B >= 16: the block has at least that many threads
+                    const uint32_t half = tid >> 7, s = (tid >> 3) & 15u, j = tid & 7u;
+                    const uint32_t e = (s << 7) + ph * kPhaseSyms + (j << 2) + 2u * half;
+                    float acc[2];
+                    acc[0] = first_batch ? 0.0f : carry[ph][0];
+                    acc[1] = first_batch ? 0.0f : carry[ph][1];
+                    sum_half(sm.val, sm_sym, s, j, half, nb, acc);
                     if (!last_batch) {
-#pragma unroll
-                        for (int q = 0; q < 4; ++q) carry[ph][q] = acc[q];
+                        carry[ph][0] = acc[0];
+                        carry[ph][1] = acc[1];
                     } else if (e < to.n_elem) {
-                        write_word<false>(to, e, acc, symw);
+                        write_half(to, e, acc);
                     }
                 }
             } else {
@@ -2287,7 +2357,11 @@ int decode_common(const uint8_t* const* streams, const uint8_t* single, size_t s
     // B clients side by side and G chunks per block, 16 sub-chunk threads per (chunk, client) pair, at most
     // 16 pairs; small inputs take fewer chunks per block so that the grid still covers the GPU
     const bool multi = n_clients > (uint32_t)kMaxPairs;
-    uint32_t B = multi ? (uint32_t)kMaxPairs : n_clients;
+    uint32_t B = n_clients;
+    if (multi) {  // equal batches of at most kMultiPairs clients, never fewer than 16 side by side
+        const uint32_t batches = (n_clients + kMultiPairs - 1) / kMultiPairs;
+        B = std::max<uint32_t>(16u, (n_clients + batches - 1) / batches);
+    }
     uint32_t G = multi ? 1u : (uint32_t)kMaxPairs / B;
     const uint32_t g_min = (B == 1) ? 2u : 1u;  // a block needs at least one full warp
     if (!multi && G > g_min) {
@@ -2306,7 +2380,7 @@ int decode_common(const uint8_t* const* streams, const uint8_t* single, size_t s
     const size_t smem = sizeof(DecSmem) + 4 * ((size_t)n_pairs * (kPairPhaseWords + kPaySlotWords) + kPaySlack);
     if (multi) {
         CO3_CUDA(cudaFuncSetAttribute(decode_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        CO3_LAUNCH(CO3_KERNEL_DECODE, st, decode_kernel<true, false><<<tiles, kThreads, smem, st>>>(da));
+        CO3_LAUNCH(CO3_KERNEL_DECODE, st, decode_kernel<true, false><<<tiles, 16 * n_pairs, smem, st>>>(da));
     } else if (n_clients == 1) {
         CO3_CUDA(cudaFuncSetAttribute(decode_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         CO3_LAUNCH(CO3_KERNEL_DECODE, st, decode_kernel<false, true><<<tiles, 16 * n_pairs, smem, st>>>(da));
