@@ -303,8 +303,38 @@ __global__ void __launch_bounds__(kThreads) prepare_kernel(PrepArgs a) {
 }
 
 // ------------------------------------------------------------------------------------------------
-// Element access for one thread: 8 consecutive elements of a chunk.
+// Element access for one thread.  In the client kernels thread t owns two groups of four consecutive elements of a
+// chunk, half a chunk apart: elements 4t .. 4t+3 and kC/2 + 4t .. kC/2 + 4t+3 (register j holds element
+// 4t + (j & 3) + (j >> 2) * kC/2).  A warp's 16-byte accesses are then contiguous, in the shared-memory ring (no bank
+// conflicts) and in global memory (whole lines per store).  The moment sums keep eight consecutive elements.
 // ------------------------------------------------------------------------------------------------
+constexpr uint32_t kHalf = kC / 2;
+static_assert(kC == 8 * kThreads, "eight elements of a chunk per thread");
+
+// Bit j set: register j of thread `q0 / 4` holds an element of a chunk of `cnt` elements (q0 = 4 * thread index).
+__device__ __forceinline__ uint32_t quads_valid(uint32_t cnt, uint32_t q0) {
+    const uint32_t na = cnt > q0 ? min(4u, cnt - q0) : 0u;
+    const uint32_t nb = cnt > q0 + kHalf ? min(4u, cnt - q0 - kHalf) : 0u;
+    return ((1u << na) - 1u) | (((1u << nb) - 1u) << 4);
+}
+
+// p: the chunk's first element + q0
+__device__ __forceinline__ void store_quads_vec(float* __restrict__ p, const float (&x)[8]) {
+    *reinterpret_cast<float4*>(p) = make_float4(x[0], x[1], x[2], x[3]);
+    *reinterpret_cast<float4*>(p + kHalf) = make_float4(x[4], x[5], x[6], x[7]);
+}
+
+__device__ __forceinline__ void load_quads_any(const float* __restrict__ p, uint32_t valid, float (&x)[8]) {
+#pragma unroll
+    for (int j = 0; j < 8; ++j) x[j] = ((valid >> j) & 1u) ? p[(j & 3) + (j >> 2) * kHalf] : 0.0f;
+}
+
+__device__ __forceinline__ void store_quads_any(float* __restrict__ p, uint32_t valid, const float (&x)[8]) {
+#pragma unroll
+    for (int j = 0; j < 8; ++j)
+        if ((valid >> j) & 1u) p[(j & 3) + (j >> 2) * kHalf] = x[j];
+}
+
 __device__ __forceinline__ void load8_vec(const float* __restrict__ p, float (&x)[8]) {
     const float4 a = __ldg(reinterpret_cast<const float4*>(p));
     const float4 b = __ldg(reinterpret_cast<const float4*>(p) + 1);
@@ -312,20 +342,9 @@ __device__ __forceinline__ void load8_vec(const float* __restrict__ p, float (&x
     x[4] = b.x; x[5] = b.y; x[6] = b.z; x[7] = b.w;
 }
 
-__device__ __forceinline__ void store8_vec(float* __restrict__ p, const float (&x)[8]) {
-    reinterpret_cast<float4*>(p)[0] = make_float4(x[0], x[1], x[2], x[3]);
-    reinterpret_cast<float4*>(p)[1] = make_float4(x[4], x[5], x[6], x[7]);
-}
-
 __device__ __forceinline__ void load8_any(const float* __restrict__ p, uint32_t n_valid, float (&x)[8]) {
 #pragma unroll
     for (int j = 0; j < 8; ++j) x[j] = (uint32_t)j < n_valid ? p[j] : 0.0f;
-}
-
-__device__ __forceinline__ void store8_any(float* __restrict__ p, uint32_t n_valid, const float (&x)[8]) {
-#pragma unroll
-    for (int j = 0; j < 8; ++j)
-        if ((uint32_t)j < n_valid) p[j] = x[j];
 }
 
 __device__ __forceinline__ uint2 pack_sym8(const uint32_t (&s)[8]) {
@@ -354,29 +373,29 @@ __device__ __forceinline__ void add_counts(co3_result* r, uint32_t n_sat, uint32
 }
 
 // Where a thread's eight elements lie, for the draws of a dithered conversion: the call's seed, client, layer, and
-// the place of the first of them inside the layer (a multiple of 8).
+// the place of the first of them inside the layer (a multiple of 4; the second group of four lies kHalf further on).
 struct Place {
     uint32_t seed, client, layer;
     uint64_t first;
 };
 
 // Correct + convert + memory update of 8 elements held in registers (Algorithm 1, client side).
-// kWhole: all eight are valid, so the branch-free converter may be used.  Symbols land in s[], the new memory
-// in mo[]; counters accumulate in n_sat / n_nf.
+// kWhole: all eight are valid, so the branch-free converter may be used; otherwise bit j of `valid` says whether
+// register j holds an element.  Symbols land in s[], the new memory in mo[]; counters accumulate in n_sat / n_nf.
 // kDither: the instance of the dithered entry points: one draw per element (four per block of the draw stream)
 // decides between the two levels around its value.
-// ring_g / ring_m (kWhole only): the thread's eight gradient and memory values in the shared-memory ring, from which
+// ring_g / ring_m (kWhole only): the thread's first gradient and memory value in the shared-memory ring, from which
 // the rare second look at a group reads them again, so that the registers holding them are free once the first
 // look is done.
 template <bool kWhole, bool kDither>
-__device__ __forceinline__ void convert8(const float (&g)[8], const float (&m)[8], uint32_t nv, float decay,
+__device__ __forceinline__ void convert8(const float (&g)[8], const float (&m)[8], uint32_t valid, float decay,
                                          const FmtDev& f, const Place& at, float (&mo)[8], uint32_t (&s)[8],
                                          uint32_t& n_sat, uint32_t& n_nf, const float* ring_g = nullptr,
                                          const float* ring_m = nullptr) {
     if (kDither) {
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
-            const uint64_t b = (at.first >> 2) + (uint32_t)h;
+            const uint64_t b = (at.first >> 2) + (uint32_t)h * (kHalf / 4u);
             const uint4 r = philox4x32_10(make_uint4((uint32_t)b, (uint32_t)(b >> 32), at.client, at.layer), at.seed, 0u);
             const uint32_t R[4] = {r.x >> 8, r.y >> 8, r.z >> 8, r.w >> 8};
 #pragma unroll
@@ -384,7 +403,7 @@ __device__ __forceinline__ void convert8(const float (&g)[8], const float (&m)[8
                 const int j = 4 * h + q;
                 uint32_t fl = 0;
                 mo[j] = convert_one_dither(g[j], m[j], decay, f, R[q], s[j], fl);
-                if ((uint32_t)j < nv) { n_sat += fl & 1u; n_nf += fl >> 1; }
+                if ((valid >> j) & 1u) { n_sat += fl & 1u; n_nf += fl >> 1; }
             }
         }
         return;
@@ -399,7 +418,8 @@ __device__ __forceinline__ void convert8(const float (&g)[8], const float (&m)[8
             float g2[8], m2[8];
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
-                const float4 x = reinterpret_cast<const float4*>(ring_g)[h], y = reinterpret_cast<const float4*>(ring_m)[h];
+                const float4 x = *reinterpret_cast<const float4*>(ring_g + h * kHalf);
+                const float4 y = *reinterpret_cast<const float4*>(ring_m + h * kHalf);
                 g2[4 * h] = x.x; g2[4 * h + 1] = x.y; g2[4 * h + 2] = x.z; g2[4 * h + 3] = x.w;
                 m2[4 * h] = y.x; m2[4 * h + 1] = y.y; m2[4 * h + 2] = y.z; m2[4 * h + 3] = y.w;
             }
@@ -431,7 +451,7 @@ __device__ __forceinline__ void convert8(const float (&g)[8], const float (&m)[8
         for (int j = 0; j < 8; ++j) {
             uint32_t fl = 0;
             mo[j] = convert_one(g[j], m[j], decay, f, s[j], fl);
-            if ((uint32_t)j < nv) { n_sat += fl & 1u; n_nf += fl >> 1; }
+            if ((valid >> j) & 1u) { n_sat += fl & 1u; n_nf += fl >> 1; }
         }
     }
 }
@@ -540,11 +560,11 @@ __device__ __forceinline__ void feed_fetch_fmt(Feed& fd, const Ws& ws, uint32_t 
             reinterpret_cast<const uint32_t*>(&ws.fmt[fd.item[slot].d.seg])[threadIdx.x];
 }
 
-// All threads: this thread's 8 gradient and memory values of the current item.  Returns false if the
-// copies never arrived (never expected).
+// All threads: this thread's 8 gradient and memory values of the current item (q0 = 4 * thread index, `valid` as
+// quads_valid gives it).  Returns false if the copies never arrived (never expected).
 // `parity` holds, per ring slot, the phase parity of the next copy to wait for.
-__device__ __forceinline__ bool feed_read(Feed& fd, const FeedArgs& fa, const FeedItem& it, uint32_t k, uint32_t i0,
-                                          uint32_t nv, uint32_t& parity, float (&g)[8], float (&m)[8]) {
+__device__ __forceinline__ bool feed_read(Feed& fd, const FeedArgs& fa, const FeedItem& it, uint32_t k, uint32_t q0,
+                                          uint32_t valid, uint32_t& parity, float (&g)[8], float (&m)[8]) {
     if (it.tma) {
         const uint32_t slot = (uint32_t)k & 1u;
         const bool ok = mbar_wait(&fd.bar[slot], (parity >> slot) & 1u);
@@ -553,14 +573,15 @@ __device__ __forceinline__ bool feed_read(Feed& fd, const FeedArgs& fa, const Fe
             fd.fail = 1u;
             return false;
         }
-        const float4* gs = reinterpret_cast<const float4*>(&fd.g[slot][i0]);
-        const float4* ms = reinterpret_cast<const float4*>(&fd.m[slot][i0]);
-        const float4 a = gs[0], b = gs[1], c = ms[0], d = ms[1];
+        const float4 a = *reinterpret_cast<const float4*>(&fd.g[slot][q0]);
+        const float4 b = *reinterpret_cast<const float4*>(&fd.g[slot][q0 + kHalf]);
+        const float4 c = *reinterpret_cast<const float4*>(&fd.m[slot][q0]);
+        const float4 d = *reinterpret_cast<const float4*>(&fd.m[slot][q0 + kHalf]);
         g[0] = a.x; g[1] = a.y; g[2] = a.z; g[3] = a.w; g[4] = b.x; g[5] = b.y; g[6] = b.z; g[7] = b.w;
         m[0] = c.x; m[1] = c.y; m[2] = c.z; m[3] = c.w; m[4] = d.x; m[5] = d.y; m[6] = d.z; m[7] = d.w;
     } else {
-        load8_any(fa.grad + it.base + i0, nv, g);
-        load8_any(fa.mem + it.base + i0, nv, m);
+        load_quads_any(fa.grad + it.base + q0, valid, g);
+        load_quads_any(fa.mem + it.base + q0, valid, m);
     }
     return true;
 }
@@ -591,6 +612,43 @@ struct ConvertArgs {
 
 constexpr int kHistCopies = 8;    // private histograms per block, spread over the lanes
 constexpr int kHistStride = 260;  // words between copies: shifts each copy by four banks
+
+// One thread's part of one work item once its inputs are in registers: conversion, new memory, symbols, counts.
+// kWhole: the chunk is complete and came through the ring (every register holds an element, 16-byte accesses).
+template <bool kSym, bool kHist, bool kMem, bool kDither, bool kWhole>
+__device__ __forceinline__ void convert_item(const ConvertArgs& a, Feed& fd, const FeedItem& it, uint64_t k, const FmtDev& f,
+                                             uint32_t valid, const float (&g)[8], const float (&m)[8], uint32_t* s_hist,
+                                             uint32_t& n_sat, uint32_t& n_nf) {
+    const uint32_t q0 = threadIdx.x * 4;
+    const uint64_t e = it.base + q0;
+    const Place at{a.seed, it.client, it.d.seg, (uint64_t)it.d.cis * kC + q0};
+    float mo[8];
+    uint32_t s[8];
+    if (kWhole) {
+        convert8<true, kDither>(g, m, 0xffu, a.decay, f, at, mo, s, n_sat, n_nf, &fd.g[k & 1u][q0], &fd.m[k & 1u][q0]);
+        if (kMem) store_quads_vec(a.mem + e, mo);
+    } else {
+        convert8<false, kDither>(g, m, valid, a.decay, f, at, mo, s, n_sat, n_nf);
+        if (kMem) store_quads_any(a.mem + e, valid, mo);
+    }
+    if (kSym) {
+        if (kWhole && (reinterpret_cast<uintptr_t>(a.sym_out + e) & 3u) == 0) {
+            const uint2 w = pack_sym8(s);
+            *reinterpret_cast<uint32_t*>(a.sym_out + e) = w.x;
+            *reinterpret_cast<uint32_t*>(a.sym_out + e + kHalf) = w.y;
+        } else {
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+                if (kWhole || ((valid >> j) & 1u)) a.sym_out[e + (j & 3) + (j >> 2) * kHalf] = (uint8_t)s[j];
+        }
+    }
+    if (kHist) {
+        uint32_t* h = s_hist + (threadIdx.x & (kHistCopies - 1)) * kHistStride;
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+            if (kWhole || ((valid >> j) & 1u)) atomicAdd(&h[s[j]], 1u);
+    }
+}
 
 // kMem: the new memory is stored (false: a dry pass that only counts symbols and leaves every input untouched).
 // kDither: the instance behind the dithered entry points (stochastic choice between the two levels around a value).
@@ -623,7 +681,7 @@ __global__ void __launch_bounds__(kThreads, (kMem || kDither) ? 3 : 4) convert_k
 
     uint32_t n_sat = 0, n_nf = 0, hist_seg = 0xffffffffu, cur_client = 0, parity = 0;
     bool hw_fail = false;
-    const uint32_t i0 = tid * 8;
+    const uint32_t q0 = tid * 4;
     for (uint64_t k = 0;; ++k) {
         if (tid == 0) feed_issue(fd, fa, a.ws, n_chunks, (uint32_t)(k + 1) & 1u, next, true);
         const FeedItem it = fd.item[k & 1u];
@@ -645,37 +703,12 @@ __global__ void __launch_bounds__(kThreads, (kMem || kDither) ? 3 : 4) convert_k
             __syncthreads();
         }
         const FmtDev f = fd.fmt[k & 1u];
-        const uint32_t nv = it.d.cnt > i0 ? min(8u, it.d.cnt - i0) : 0u;
-        float g[8], m[8], mo[8];
-        uint32_t s[8];
+        const uint32_t valid = it.tma ? 0xffu : quads_valid(it.d.cnt, q0);
+        float g[8], m[8];
         // a copy that never arrived (never expected): this thread writes nothing for the item, the block stops
-        const bool ok = feed_read(fd, fa, it, k, i0, nv, parity, g, m);
-        const uint64_t e = it.base + i0;
-        if (!ok) {
-            hw_fail = true;
-        } else if (it.tma) {
-            convert8<true, kDither>(g, m, 8, a.decay, f, Place{a.seed, it.client, it.d.seg, (uint64_t)it.d.cis * kC + i0}, mo, s, n_sat, n_nf,
-                                    &fd.g[k & 1u][i0], &fd.m[k & 1u][i0]);
-            if (kMem) store8_vec(a.mem + e, mo);
-        } else if (nv) {
-            convert8<false, kDither>(g, m, nv, a.decay, f, Place{a.seed, it.client, it.d.seg, (uint64_t)it.d.cis * kC + i0}, mo, s, n_sat, n_nf);
-            if (kMem) store8_any(a.mem + e, nv, mo);
-        }
-        if (kSym && nv && ok) {
-            if (nv == 8 && (reinterpret_cast<uintptr_t>(a.sym_out + e) & 7u) == 0) {
-                *reinterpret_cast<uint2*>(a.sym_out + e) = pack_sym8(s);
-            } else {
-#pragma unroll
-                for (int j = 0; j < 8; ++j)
-                    if ((uint32_t)j < nv) a.sym_out[e + j] = (uint8_t)s[j];
-            }
-        }
-        if (kHist && nv && ok) {
-            uint32_t* h = s_hist + (tid & (kHistCopies - 1)) * kHistStride;
-#pragma unroll
-            for (int j = 0; j < 8; ++j)
-                if ((uint32_t)j < nv) atomicAdd(&h[s[j]], 1u);
-        }
+        if (!feed_read(fd, fa, it, k, q0, valid, parity, g, m)) hw_fail = true;
+        else if (it.tma) convert_item<kSym, kHist, kMem, kDither, true>(a, fd, it, k, f, 0xffu, g, m, s_hist, n_sat, n_nf);
+        else if (valid) convert_item<kSym, kHist, kMem, kDither, false>(a, fd, it, k, f, valid, g, m, s_hist, n_sat, n_nf);
         feed_fetch_fmt(fd, a.ws, (uint32_t)(k + 1) & 1u);  // item k + 1 was published before the previous barrier
         __syncthreads();  // everyone has read ring slot k & 1 and item[k & 1] before thread 0 reuses them
         if (fd.fail) {    // the same for every thread: written before the barrier
@@ -699,7 +732,8 @@ __global__ void __launch_bounds__(kThreads, (kMem || kDither) ? 3 : 4) convert_k
 }
 
 // ------------------------------------------------------------------------------------------------
-// pack: persistent blocks over (chunk, client) items.  Thread t owns symbols 8t .. 8t+7 of the chunk.
+// pack: persistent blocks over (chunk, client) items.  Thread t owns symbols 4t .. 4t+3 and kC/2 + 4t .. kC/2 + 4t+3
+// of the chunk.
 // ------------------------------------------------------------------------------------------------
 struct PackArgs {
     const float* grad;   // fused path
@@ -780,46 +814,49 @@ struct PackSmem {
 // One work item of the pack kernel for one thread: symbols of its 8 elements (converted here unless
 // kFromSym), their codewords, the block-wide scan of the lengths, and the bits ORed into the chunk's buffer.
 // kWhole: the chunk is complete (and, on the fused path, was delivered through the ring).
-// Returns the chunk's total bit count; `missing` reports a symbol without codeword.
+// Returns the chunk's total bit count; `missing` reports a symbol without codeword; off_a / off_b: where the
+// thread's two groups of four start in the chunk's bits.
 template <bool kFromSym, bool kWhole, bool kDither>
 __device__ __forceinline__ uint32_t pack_item(const PackArgs& a, PackSmem& sm, const FeedArgs& fa, const FeedItem& it,
                                               uint32_t k, uint32_t& parity, uint32_t& enc_seg, uint32_t& n_sat,
-                                              uint32_t& n_nf, bool& hw_fail, bool& missing, uint32_t& off_out) {
-    const uint32_t tid = threadIdx.x, i0 = tid * 8;
-    const uint32_t nv = kWhole ? 8u : (it.d.cnt > i0 ? min(8u, it.d.cnt - i0) : 0u);
-    const uint64_t e = it.base + i0;
+                                              uint32_t& n_nf, bool& hw_fail, bool& missing, uint32_t& off_a,
+                                              uint32_t& off_b) {
+    const uint32_t tid = threadIdx.x, q0 = tid * 4;
+    const uint32_t valid = kWhole ? 0xffu : quads_valid(it.d.cnt, q0);
+    const uint64_t e = it.base + q0;
     uint32_t s[8];
     if (kFromSym) {
-        if (kWhole && (reinterpret_cast<uintptr_t>(a.sym + e) & 7u) == 0) {
-            const uint2 w = __ldg(reinterpret_cast<const uint2*>(a.sym + e));
+        if (kWhole && (reinterpret_cast<uintptr_t>(a.sym + e) & 3u) == 0) {
+            const uint32_t wx = __ldg(reinterpret_cast<const uint32_t*>(a.sym + e));
+            const uint32_t wy = __ldg(reinterpret_cast<const uint32_t*>(a.sym + e + kHalf));
 #pragma unroll
-            for (int j = 0; j < 4; ++j) { s[j] = (w.x >> (8 * j)) & 0xffu; s[4 + j] = (w.y >> (8 * j)) & 0xffu; }
+            for (int j = 0; j < 4; ++j) { s[j] = (wx >> (8 * j)) & 0xffu; s[4 + j] = (wy >> (8 * j)) & 0xffu; }
         } else {
 #pragma unroll
-            for (int j = 0; j < 8; ++j) s[j] = (uint32_t)j < nv ? a.sym[e + j] : 0u;
+            for (int j = 0; j < 8; ++j) s[j] = ((valid >> j) & 1u) ? a.sym[e + (j & 3) + (j >> 2) * kHalf] : 0u;
         }
     } else {
         const FmtDev f = sm.feed.fmt[k & 1u];
         float g[8], m[8], mo[8];
         // a copy that never arrived (never expected): the memory is left alone, the block stops after this item
-        const bool ok = feed_read(sm.feed, fa, it, k, i0, nv, parity, g, m);
+        const bool ok = feed_read(sm.feed, fa, it, k, q0, valid, parity, g, m);
         if (!ok) {
             hw_fail = true;
 #pragma unroll
             for (int j = 0; j < 8; ++j) s[j] = 0u;
         } else if (kWhole) {
-            convert8<true, kDither>(g, m, 8, a.decay, f, Place{a.seed, it.client, it.d.seg, (uint64_t)it.d.cis * kC + i0}, mo, s, n_sat, n_nf,
-                                    &sm.feed.g[k & 1u][i0], &sm.feed.m[k & 1u][i0]);
-            store8_vec(a.mem + e, mo);
-        } else if (nv) {
-            convert8<false, kDither>(g, m, nv, a.decay, f, Place{a.seed, it.client, it.d.seg, (uint64_t)it.d.cis * kC + i0}, mo, s, n_sat, n_nf);
-            store8_any(a.mem + e, nv, mo);
+            convert8<true, kDither>(g, m, 0xffu, a.decay, f, Place{a.seed, it.client, it.d.seg, (uint64_t)it.d.cis * kC + q0}, mo, s, n_sat, n_nf,
+                                    &sm.feed.g[k & 1u][q0], &sm.feed.m[k & 1u][q0]);
+            store_quads_vec(a.mem + e, mo);
+        } else if (valid) {
+            convert8<false, kDither>(g, m, valid, a.decay, f, Place{a.seed, it.client, it.d.seg, (uint64_t)it.d.cis * kC + q0}, mo, s, n_sat, n_nf);
+            store_quads_any(a.mem + e, valid, mo);
         }
     }
-    // codewords of this thread's symbols, concatenated in two halves of at most 64 bits
+    // codewords of this thread's symbols, each group of four concatenated into at most 64 bits
     uint32_t ent[8];
 #pragma unroll
-    for (int j = 0; j < 8; ++j) ent[j] = (kWhole || (uint32_t)j < nv) ? sm.enc[s[j]] : 0u;
+    for (int j = 0; j < 8; ++j) ent[j] = (kWhole || ((valid >> j) & 1u)) ? sm.enc[s[j]] : 0u;
     const uint32_t any = ent[0] | ent[1] | ent[2] | ent[3] | ent[4] | ent[5] | ent[6] | ent[7];
     missing = (any & kEncMissing) != 0;
     // the low byte of an entry is its length, at most 16: sums of four stay inside the byte
@@ -831,8 +868,12 @@ __device__ __forceinline__ uint32_t pack_item(const PackArgs& a, PackSmem& sm, c
     const uint32_t c67 = ((ent[6] >> 8) << (ent[7] & 0xffu)) | (ent[7] >> 8);
     const uint64_t wa = ((uint64_t)c01 << ((ent[2] + ent[3]) & 0xffu)) | c23;
     const uint64_t wb = ((uint64_t)c45 << ((ent[6] + ent[7]) & 0xffu)) | c67;
-    uint32_t total;
-    const uint32_t off = block_exclusive_scan_once(la + lb, sm.scan[k & 1u], &total);
+    // One scan for both groups, the first in the low and the second in the high half of a word: neither sum can pass
+    // kC / 2 * 16 bits.  The second groups follow all the first ones in the chunk.
+    uint32_t totals;
+    const uint32_t ex = block_exclusive_scan_once(la | (lb << 16), sm.scan[k & 1u], &totals);
+    off_a = ex & 0xffffu;
+    off_b = (totals & 0xffffu) + (ex >> 16);
     // Behind the scan's barrier every thread has finished the previous item's copy-out and this item's table
     // look-ups: clear the other bit buffer and fetch the next item's tables.
     static_assert(kBitWords == 4 * kThreads, "one uint4 of the bit buffer per thread");
@@ -845,11 +886,10 @@ __device__ __forceinline__ uint32_t pack_item(const PackArgs& a, PackSmem& sm, c
     if (!kFromSym) feed_fetch_fmt(sm.feed, a.ws, (uint32_t)(k + 1) & 1u);
     if (!missing) {
         const uint32_t bits_addr = smem_addr(sm.bits[k & 1u]);
-        put_bits(bits_addr, off + la, wa);
-        put_bits(bits_addr, off + la + lb, wb);
+        put_bits(bits_addr, off_a + la, wa);
+        put_bits(bits_addr, off_b + lb, wb);
     }
-    off_out = off;
-    return total;
+    return (totals & 0xffffu) + (totals >> 16);
 }
 
 // Thread 0 only: output locations of the item just published in ring slot `slot`.
@@ -911,12 +951,17 @@ __global__ void __launch_bounds__(kThreads, 3) pack_kernel(PackArgs a) {
             cur_client = it.client;
         }
         bool missing;
-        uint32_t off, total;
+        uint32_t off_a, off_b, total;
         const bool whole = kFromSym ? it.d.cnt == (uint32_t)kC : it.tma != 0;
-        if (whole) total = pack_item<kFromSym, true, kDither>(a, sm, fa, it, k, parity, enc_seg, n_sat, n_nf, hw_fail, missing, off);
-        else total = pack_item<kFromSym, false, kDither>(a, sm, fa, it, k, parity, enc_seg, n_sat, n_nf, hw_fail, missing, off);
+        if (whole) total = pack_item<kFromSym, true, kDither>(a, sm, fa, it, k, parity, enc_seg, n_sat, n_nf, hw_fail, missing, off_a, off_b);
+        else total = pack_item<kFromSym, false, kDither>(a, sm, fa, it, k, parity, enc_seg, n_sat, n_nf, hw_fail, missing, off_a, off_b);
         const PackOut out = sm.out[k & 1u];
-        if ((tid & 15u) == 0) out.sub[tid >> 4] = (uint16_t)off;
+        // a sub-chunk of kS symbols is one warp's first or second groups
+        static_assert(kS == 4 * 32 && kSubs == 2 * (kThreads / 32), "a warp's groups of four make up one sub-chunk each");
+        if ((tid & 31u) == 0) {
+            out.sub[tid >> 5] = (uint16_t)off_a;
+            out.sub[kSubs / 2 + (tid >> 5)] = (uint16_t)off_b;
+        }
         if (__syncthreads_or(missing)) {  // bit buffer complete
             if (tid == 0) {
                 set_status(out.res, CO3_ERR_NO_CODEWORD);
