@@ -974,12 +974,9 @@ __global__ void __launch_bounds__(kThreads, 3) pack_kernel(PackArgs a) {
             break;
         }
         if (tid == 0) *out.chunk_bits = total;
-        const uint32_t words = (total + 31u) >> 5;
-        uint32_t* slot = out.slot + tid;
-        const uint32_t* bits = sm.bits[k & 1u] + tid;
-#pragma unroll
-        for (int r = 0; r < kSlotWords / kThreads; ++r)
-            if (tid + r * kThreads < words) slot[r * kThreads] = bits[r * kThreads];
+        // the chunk's words, four per thread; what the last of these copies carries beyond the chunk's end is zero
+        // and stays inside the slot
+        if (tid * 128u < total) reinterpret_cast<uint4*>(out.slot)[tid] = reinterpret_cast<const uint4*>(sm.bits[k & 1u])[tid];
     }
     if (!kFromSym) add_counts(&a.res[cur_client], n_sat, n_nf);
     if (__syncthreads_or(hw_fail)) {  // the block stopped early, chunks of any client may be missing: the call fails
