@@ -311,28 +311,36 @@ __global__ void __launch_bounds__(kThreads) prepare_kernel(PrepArgs a) {
 constexpr uint32_t kHalf = kC / 2;
 static_assert(kC == 8 * kThreads, "eight elements of a chunk per thread");
 
-// Bit j set: register j of thread `q0 / 4` holds an element of a chunk of `cnt` elements (q0 = 4 * thread index).
+// The helpers below take the distance kQ between the two groups (kHalf in the 256-thread kernels; the packer's
+// 128 threads own two such pairs each, kQuarter apart) and q0, the place of the first group in the chunk.
+constexpr uint32_t kQuarter = kC / 4;
+
+// Bit j set: register j holds an element of a chunk of `cnt` elements.
+template <uint32_t kQ>
 __device__ __forceinline__ uint32_t quads_valid(uint32_t cnt, uint32_t q0) {
     const uint32_t na = cnt > q0 ? min(4u, cnt - q0) : 0u;
-    const uint32_t nb = cnt > q0 + kHalf ? min(4u, cnt - q0 - kHalf) : 0u;
+    const uint32_t nb = cnt > q0 + kQ ? min(4u, cnt - q0 - kQ) : 0u;
     return ((1u << na) - 1u) | (((1u << nb) - 1u) << 4);
 }
 
 // p: the chunk's first element + q0
+template <uint32_t kQ>
 __device__ __forceinline__ void store_quads_vec(float* __restrict__ p, const float (&x)[8]) {
     *reinterpret_cast<float4*>(p) = make_float4(x[0], x[1], x[2], x[3]);
-    *reinterpret_cast<float4*>(p + kHalf) = make_float4(x[4], x[5], x[6], x[7]);
+    *reinterpret_cast<float4*>(p + kQ) = make_float4(x[4], x[5], x[6], x[7]);
 }
 
+template <uint32_t kQ>
 __device__ __forceinline__ void load_quads_any(const float* __restrict__ p, uint32_t valid, float (&x)[8]) {
 #pragma unroll
-    for (int j = 0; j < 8; ++j) x[j] = ((valid >> j) & 1u) ? p[(j & 3) + (j >> 2) * kHalf] : 0.0f;
+    for (int j = 0; j < 8; ++j) x[j] = ((valid >> j) & 1u) ? p[(j & 3) + (j >> 2) * kQ] : 0.0f;
 }
 
+template <uint32_t kQ>
 __device__ __forceinline__ void store_quads_any(float* __restrict__ p, uint32_t valid, const float (&x)[8]) {
 #pragma unroll
     for (int j = 0; j < 8; ++j)
-        if ((valid >> j) & 1u) p[(j & 3) + (j >> 2) * kHalf] = x[j];
+        if ((valid >> j) & 1u) p[(j & 3) + (j >> 2) * kQ] = x[j];
 }
 
 __device__ __forceinline__ void load8_vec(const float* __restrict__ p, float (&x)[8]) {
@@ -373,7 +381,7 @@ __device__ __forceinline__ void add_counts(co3_result* r, uint32_t n_sat, uint32
 }
 
 // Where a thread's eight elements lie, for the draws of a dithered conversion: the call's seed, client, layer, and
-// the place of the first of them inside the layer (a multiple of 4; the second group of four lies kHalf further on).
+// the place of the first of them inside the layer (a multiple of 4; the second group of four lies kQ further on).
 struct Place {
     uint32_t seed, client, layer;
     uint64_t first;
@@ -387,7 +395,7 @@ struct Place {
 // ring_g / ring_m (kWhole only): the thread's first gradient and memory value in the shared-memory ring, from which
 // the rare second look at a group reads them again, so that the registers holding them are free once the first
 // look is done.
-template <bool kWhole, bool kDither>
+template <bool kWhole, bool kDither, uint32_t kQ>
 __device__ __forceinline__ void convert8(const float (&g)[8], const float (&m)[8], uint32_t valid, float decay,
                                          const FmtDev& f, const Place& at, float (&mo)[8], uint32_t (&s)[8],
                                          uint32_t& n_sat, uint32_t& n_nf, const float* ring_g = nullptr,
@@ -395,7 +403,7 @@ __device__ __forceinline__ void convert8(const float (&g)[8], const float (&m)[8
     if (kDither) {
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
-            const uint64_t b = (at.first >> 2) + (uint32_t)h * (kHalf / 4u);
+            const uint64_t b = (at.first >> 2) + (uint32_t)h * (kQ / 4u);
             const uint4 r = philox4x32_10(make_uint4((uint32_t)b, (uint32_t)(b >> 32), at.client, at.layer), at.seed, 0u);
             const uint32_t R[4] = {r.x >> 8, r.y >> 8, r.z >> 8, r.w >> 8};
 #pragma unroll
@@ -418,8 +426,8 @@ __device__ __forceinline__ void convert8(const float (&g)[8], const float (&m)[8
             float g2[8], m2[8];
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
-                const float4 x = *reinterpret_cast<const float4*>(ring_g + h * kHalf);
-                const float4 y = *reinterpret_cast<const float4*>(ring_m + h * kHalf);
+                const float4 x = *reinterpret_cast<const float4*>(ring_g + h * kQ);
+                const float4 y = *reinterpret_cast<const float4*>(ring_m + h * kQ);
                 g2[4 * h] = x.x; g2[4 * h + 1] = x.y; g2[4 * h + 2] = x.z; g2[4 * h + 3] = x.w;
                 m2[4 * h] = y.x; m2[4 * h + 1] = y.y; m2[4 * h + 2] = y.z; m2[4 * h + 3] = y.w;
             }
@@ -560,30 +568,34 @@ __device__ __forceinline__ void feed_fetch_fmt(Feed& fd, const Ws& ws, uint32_t 
             reinterpret_cast<const uint32_t*>(&ws.fmt[fd.item[slot].d.seg])[threadIdx.x];
 }
 
-// All threads: this thread's 8 gradient and memory values of the current item (q0 = 4 * thread index, `valid` as
-// quads_valid gives it).  Returns false if the copies never arrived (never expected).
-// `parity` holds, per ring slot, the phase parity of the next copy to wait for.
-__device__ __forceinline__ bool feed_read(Feed& fd, const FeedArgs& fa, const FeedItem& it, uint32_t k, uint32_t q0,
-                                          uint32_t valid, uint32_t& parity, float (&g)[8], float (&m)[8]) {
+// All threads: waits for the current item's copies, if it has any.  Returns false if they never arrived (never
+// expected).  `parity` holds, per ring slot, the phase parity of the next copy to wait for.
+__device__ __forceinline__ bool feed_wait(Feed& fd, const FeedItem& it, uint32_t k, uint32_t& parity) {
+    if (!it.tma) return true;
+    const uint32_t slot = k & 1u;
+    const bool ok = mbar_wait(&fd.bar[slot], (parity >> slot) & 1u);
+    parity ^= 1u << slot;
+    if (!ok) fd.fail = 1u;
+    return ok;
+}
+
+// All threads, after feed_wait: the gradient and memory values of the current item that lie in the thread's two groups
+// at q0 and q0 + kQ (`valid` as quads_valid gives it).
+template <uint32_t kQ>
+__device__ __forceinline__ void feed_get(const Feed& fd, const FeedArgs& fa, const FeedItem& it, uint32_t k, uint32_t q0,
+                                         uint32_t valid, float (&g)[8], float (&m)[8]) {
     if (it.tma) {
-        const uint32_t slot = (uint32_t)k & 1u;
-        const bool ok = mbar_wait(&fd.bar[slot], (parity >> slot) & 1u);
-        parity ^= 1u << slot;
-        if (!ok) {
-            fd.fail = 1u;
-            return false;
-        }
+        const uint32_t slot = k & 1u;
         const float4 a = *reinterpret_cast<const float4*>(&fd.g[slot][q0]);
-        const float4 b = *reinterpret_cast<const float4*>(&fd.g[slot][q0 + kHalf]);
+        const float4 b = *reinterpret_cast<const float4*>(&fd.g[slot][q0 + kQ]);
         const float4 c = *reinterpret_cast<const float4*>(&fd.m[slot][q0]);
-        const float4 d = *reinterpret_cast<const float4*>(&fd.m[slot][q0 + kHalf]);
+        const float4 d = *reinterpret_cast<const float4*>(&fd.m[slot][q0 + kQ]);
         g[0] = a.x; g[1] = a.y; g[2] = a.z; g[3] = a.w; g[4] = b.x; g[5] = b.y; g[6] = b.z; g[7] = b.w;
         m[0] = c.x; m[1] = c.y; m[2] = c.z; m[3] = c.w; m[4] = d.x; m[5] = d.y; m[6] = d.z; m[7] = d.w;
     } else {
-        load_quads_any(fa.grad + it.base + q0, valid, g);
-        load_quads_any(fa.mem + it.base + q0, valid, m);
+        load_quads_any<kQ>(fa.grad + it.base + q0, valid, g);
+        load_quads_any<kQ>(fa.mem + it.base + q0, valid, m);
     }
-    return true;
 }
 
 // A wait gave up and the block has left its item loop after item k: thread 0 still waits (bounded again) for the
@@ -625,11 +637,11 @@ __device__ __forceinline__ void convert_item(const ConvertArgs& a, Feed& fd, con
     float mo[8];
     uint32_t s[8];
     if (kWhole) {
-        convert8<true, kDither>(g, m, 0xffu, a.decay, f, at, mo, s, n_sat, n_nf, &fd.g[k & 1u][q0], &fd.m[k & 1u][q0]);
-        if (kMem) store_quads_vec(a.mem + e, mo);
+        convert8<true, kDither, kHalf>(g, m, 0xffu, a.decay, f, at, mo, s, n_sat, n_nf, &fd.g[k & 1u][q0], &fd.m[k & 1u][q0]);
+        if (kMem) store_quads_vec<kHalf>(a.mem + e, mo);
     } else {
-        convert8<false, kDither>(g, m, valid, a.decay, f, at, mo, s, n_sat, n_nf);
-        if (kMem) store_quads_any(a.mem + e, valid, mo);
+        convert8<false, kDither, kHalf>(g, m, valid, a.decay, f, at, mo, s, n_sat, n_nf);
+        if (kMem) store_quads_any<kHalf>(a.mem + e, valid, mo);
     }
     if (kSym) {
         if (kWhole && (reinterpret_cast<uintptr_t>(a.sym_out + e) & 3u) == 0) {
@@ -703,12 +715,16 @@ __global__ void __launch_bounds__(kThreads, (kMem || kDither) ? 3 : 4) convert_k
             __syncthreads();
         }
         const FmtDev f = fd.fmt[k & 1u];
-        const uint32_t valid = it.tma ? 0xffu : quads_valid(it.d.cnt, q0);
-        float g[8], m[8];
+        const uint32_t valid = it.tma ? 0xffu : quads_valid<kHalf>(it.d.cnt, q0);
         // a copy that never arrived (never expected): this thread writes nothing for the item, the block stops
-        if (!feed_read(fd, fa, it, k, q0, valid, parity, g, m)) hw_fail = true;
-        else if (it.tma) convert_item<kSym, kHist, kMem, kDither, true>(a, fd, it, k, f, 0xffu, g, m, s_hist, n_sat, n_nf);
-        else if (valid) convert_item<kSym, kHist, kMem, kDither, false>(a, fd, it, k, f, valid, g, m, s_hist, n_sat, n_nf);
+        if (!feed_wait(fd, it, (uint32_t)k, parity)) {
+            hw_fail = true;
+        } else {
+            float g[8], m[8];
+            feed_get<kHalf>(fd, fa, it, (uint32_t)k, q0, valid, g, m);
+            if (it.tma) convert_item<kSym, kHist, kMem, kDither, true>(a, fd, it, k, f, 0xffu, g, m, s_hist, n_sat, n_nf);
+            else if (valid) convert_item<kSym, kHist, kMem, kDither, false>(a, fd, it, k, f, valid, g, m, s_hist, n_sat, n_nf);
+        }
         feed_fetch_fmt(fd, a.ws, (uint32_t)(k + 1) & 1u);  // item k + 1 was published before the previous barrier
         __syncthreads();  // everyone has read ring slot k & 1 and item[k & 1] before thread 0 reuses them
         if (fd.fail) {    // the same for every thread: written before the barrier
@@ -774,25 +790,31 @@ __device__ __forceinline__ void put_bits(uint32_t buf_addr, uint32_t end, uint64
 }
 
 
-constexpr int kBitWords = kSlotWords;  // bit buffer of one chunk: one uint4 per thread
+constexpr int kBitWords = kSlotWords;  // bit buffer of one chunk
+constexpr int kPackThreads = 128;      // threads of a packing block: 16 symbols of a chunk each
+constexpr int kPackWarps = kPackThreads / 32;
+static_assert(kC == 16 * kPackThreads && kQuarter == 4 * kPackThreads, "four groups of four symbols per packing thread, a quarter chunk apart");
+static_assert(kBitWords == 8 * kPackThreads, "two uint4 of the bit buffer per packing thread");
 
-// Exclusive prefix sum over the 256 threads of a block with one barrier; *total receives the block sum.
-// scratch: 8 words that no thread writes again before the block's next barrier after this call.
-__device__ __forceinline__ uint32_t block_exclusive_scan_once(uint32_t x, uint32_t* scratch, uint32_t* total) {
+// Exclusive prefix sums of two words over the threads of a packing block with one barrier; tot[] receives the block
+// sums.  scratch: 2 * kPackWarps words that no thread writes again before the block's next barrier after this call.
+__device__ __forceinline__ void pack_scan2(const uint32_t (&x)[2], uint32_t* scratch, uint32_t (&ex)[2], uint32_t (&tot)[2]) {
     const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
-    uint32_t inc = x;
+    uint32_t inc0 = x[0], inc1 = x[1];
 #pragma unroll
     for (int d = 1; d < 32; d <<= 1) {
-        const uint32_t y = __shfl_up_sync(0xffffffffu, inc, d);
-        if (lane >= (uint32_t)d) inc += y;
+        const uint32_t y0 = __shfl_up_sync(0xffffffffu, inc0, d), y1 = __shfl_up_sync(0xffffffffu, inc1, d);
+        if (lane >= (uint32_t)d) { inc0 += y0; inc1 += y1; }
     }
-    if (lane == 31u) scratch[warp] = inc;
+    if (lane == 31u) { scratch[warp] = inc0; scratch[kPackWarps + warp] = inc1; }
     __syncthreads();
-    // lanes 0..7 hold the warp sums; two warp-wide reductions give the block total and this warp's base
-    const uint32_t s = lane < 8u ? scratch[lane] : 0u;
-    *total = __reduce_add_sync(0xffffffffu, s);
-    const uint32_t base = __reduce_add_sync(0xffffffffu, lane < warp ? s : 0u);
-    return base + inc - x;
+    // the first lanes hold the warp sums; warp-wide reductions give the block totals and this warp's bases
+    const uint32_t s0 = lane < (uint32_t)kPackWarps ? scratch[lane] : 0u;
+    const uint32_t s1 = lane < (uint32_t)kPackWarps ? scratch[kPackWarps + lane] : 0u;
+    tot[0] = __reduce_add_sync(0xffffffffu, s0);
+    tot[1] = __reduce_add_sync(0xffffffffu, s1);
+    ex[0] = __reduce_add_sync(0xffffffffu, lane < warp ? s0 : 0u) + inc0 - x[0];
+    ex[1] = __reduce_add_sync(0xffffffffu, lane < warp ? s1 : 0u) + inc1 - x[1];
 }
 
 // Where the results of one work item go, worked out once per item by thread 0.
@@ -805,91 +827,106 @@ struct alignas(16) PackOut {
 
 struct PackSmem {
     Feed feed;
-    alignas(16) uint32_t bits[2][kBitWords];  // cleared and copied out one uint4 per thread
+    alignas(16) uint32_t bits[2][kBitWords];  // cleared and copied out 16 bytes at a time
     uint32_t enc[256];
-    uint32_t scan[2][8];
+    uint32_t scan[2][2 * kPackWarps];
     PackOut out[2];
 };
 
-// One work item of the pack kernel for one thread: symbols of its 8 elements (converted here unless
-// kFromSym), their codewords, the block-wide scan of the lengths, and the bits ORed into the chunk's buffer.
-// kWhole: the chunk is complete (and, on the fused path, was delivered through the ring).
-// Returns the chunk's total bit count; `missing` reports a symbol without codeword; off_a / off_b: where the
-// thread's two groups of four start in the chunk's bits.
+// Eight of a packing thread's sixteen symbols (two groups of four, at q0 and q0 + kQuarter in the chunk): converted
+// here unless kFromSym, then their codewords, each group's concatenated into at most 64 bits (wa, wb) of la and lb
+// bits.  kWhole: the chunk is complete (and, on the fused path, was delivered through the ring).  `any` collects
+// the table entries (for the no-codeword bit).  ok: what feed_wait returned.
 template <bool kFromSym, bool kWhole, bool kDither>
-__device__ __forceinline__ uint32_t pack_item(const PackArgs& a, PackSmem& sm, const FeedArgs& fa, const FeedItem& it,
-                                              uint32_t k, uint32_t& parity, uint32_t& enc_seg, uint32_t& n_sat,
-                                              uint32_t& n_nf, bool& hw_fail, bool& missing, uint32_t& off_a,
-                                              uint32_t& off_b) {
-    const uint32_t tid = threadIdx.x, q0 = tid * 4;
-    const uint32_t valid = kWhole ? 0xffu : quads_valid(it.d.cnt, q0);
+__device__ __forceinline__ void pack_eight(const PackArgs& a, PackSmem& sm, const FeedArgs& fa, const FeedItem& it, uint32_t k,
+                                           uint32_t q0, bool ok, uint32_t& n_sat, uint32_t& n_nf, uint32_t& la, uint32_t& lb,
+                                           uint64_t& wa, uint64_t& wb, uint32_t& any) {
+    const uint32_t valid = kWhole ? 0xffu : quads_valid<kQuarter>(it.d.cnt, q0);
     const uint64_t e = it.base + q0;
     uint32_t s[8];
     if (kFromSym) {
         if (kWhole && (reinterpret_cast<uintptr_t>(a.sym + e) & 3u) == 0) {
             const uint32_t wx = __ldg(reinterpret_cast<const uint32_t*>(a.sym + e));
-            const uint32_t wy = __ldg(reinterpret_cast<const uint32_t*>(a.sym + e + kHalf));
+            const uint32_t wy = __ldg(reinterpret_cast<const uint32_t*>(a.sym + e + kQuarter));
 #pragma unroll
             for (int j = 0; j < 4; ++j) { s[j] = (wx >> (8 * j)) & 0xffu; s[4 + j] = (wy >> (8 * j)) & 0xffu; }
         } else {
 #pragma unroll
-            for (int j = 0; j < 8; ++j) s[j] = ((valid >> j) & 1u) ? a.sym[e + (j & 3) + (j >> 2) * kHalf] : 0u;
+            for (int j = 0; j < 8; ++j) s[j] = ((valid >> j) & 1u) ? a.sym[e + (j & 3) + (j >> 2) * kQuarter] : 0u;
         }
     } else {
         const FmtDev f = sm.feed.fmt[k & 1u];
+        const Place at{a.seed, it.client, it.d.seg, (uint64_t)it.d.cis * kC + q0};
         float g[8], m[8], mo[8];
-        // a copy that never arrived (never expected): the memory is left alone, the block stops after this item
-        const bool ok = feed_read(sm.feed, fa, it, k, q0, valid, parity, g, m);
-        if (!ok) {
-            hw_fail = true;
+        if (ok) feed_get<kQuarter>(sm.feed, fa, it, k, q0, valid, g, m);
+        if (!ok) {  // the copies never arrived (never expected): the memory is left alone, the block stops after this item
 #pragma unroll
             for (int j = 0; j < 8; ++j) s[j] = 0u;
         } else if (kWhole) {
-            convert8<true, kDither>(g, m, 0xffu, a.decay, f, Place{a.seed, it.client, it.d.seg, (uint64_t)it.d.cis * kC + q0}, mo, s, n_sat, n_nf,
-                                    &sm.feed.g[k & 1u][q0], &sm.feed.m[k & 1u][q0]);
-            store_quads_vec(a.mem + e, mo);
+            convert8<true, kDither, kQuarter>(g, m, 0xffu, a.decay, f, at, mo, s, n_sat, n_nf, &sm.feed.g[k & 1u][q0], &sm.feed.m[k & 1u][q0]);
+            store_quads_vec<kQuarter>(a.mem + e, mo);
         } else if (valid) {
-            convert8<false, kDither>(g, m, valid, a.decay, f, Place{a.seed, it.client, it.d.seg, (uint64_t)it.d.cis * kC + q0}, mo, s, n_sat, n_nf);
-            store_quads_any(a.mem + e, valid, mo);
+            convert8<false, kDither, kQuarter>(g, m, valid, a.decay, f, at, mo, s, n_sat, n_nf);
+            store_quads_any<kQuarter>(a.mem + e, valid, mo);
         }
     }
-    // codewords of this thread's symbols, each group of four concatenated into at most 64 bits
     uint32_t ent[8];
 #pragma unroll
     for (int j = 0; j < 8; ++j) ent[j] = (kWhole || ((valid >> j) & 1u)) ? sm.enc[s[j]] : 0u;
-    const uint32_t any = ent[0] | ent[1] | ent[2] | ent[3] | ent[4] | ent[5] | ent[6] | ent[7];
-    missing = (any & kEncMissing) != 0;
+    any |= ent[0] | ent[1] | ent[2] | ent[3] | ent[4] | ent[5] | ent[6] | ent[7];
     // the low byte of an entry is its length, at most 16: sums of four stay inside the byte
-    const uint32_t la = (ent[0] + ent[1] + ent[2] + ent[3]) & 0xffu;
-    const uint32_t lb = (ent[4] + ent[5] + ent[6] + ent[7]) & 0xffu;
+    la = (ent[0] + ent[1] + ent[2] + ent[3]) & 0xffu;
+    lb = (ent[4] + ent[5] + ent[6] + ent[7]) & 0xffu;
     const uint32_t c01 = ((ent[0] >> 8) << (ent[1] & 0xffu)) | (ent[1] >> 8);
     const uint32_t c23 = ((ent[2] >> 8) << (ent[3] & 0xffu)) | (ent[3] >> 8);
     const uint32_t c45 = ((ent[4] >> 8) << (ent[5] & 0xffu)) | (ent[5] >> 8);
     const uint32_t c67 = ((ent[6] >> 8) << (ent[7] & 0xffu)) | (ent[7] >> 8);
-    const uint64_t wa = ((uint64_t)c01 << ((ent[2] + ent[3]) & 0xffu)) | c23;
-    const uint64_t wb = ((uint64_t)c45 << ((ent[6] + ent[7]) & 0xffu)) | c67;
-    // One scan for both groups, the first in the low and the second in the high half of a word: neither sum can pass
-    // kC / 2 * 16 bits.  The second groups follow all the first ones in the chunk.
-    uint32_t totals;
-    const uint32_t ex = block_exclusive_scan_once(la | (lb << 16), sm.scan[k & 1u], &totals);
-    off_a = ex & 0xffffu;
-    off_b = (totals & 0xffffu) + (ex >> 16);
+    wa = ((uint64_t)c01 << ((ent[2] + ent[3]) & 0xffu)) | c23;
+    wb = ((uint64_t)c45 << ((ent[6] + ent[7]) & 0xffu)) | c67;
+}
+
+// One work item of the pack kernel for one thread: its 16 symbols (groups of four at 4t, 4t + kQuarter, ...), the
+// block-wide scan of the groups' lengths, and the bits ORed into the chunk's buffer.
+// Returns the chunk's total bit count; `missing` reports a symbol without codeword; off[c]: where the thread's group
+// in quarter c starts in the chunk's bits.
+template <bool kFromSym, bool kWhole, bool kDither>
+__device__ __forceinline__ uint32_t pack_item(const PackArgs& a, PackSmem& sm, const FeedArgs& fa, const FeedItem& it,
+                                              uint32_t k, bool ok, uint32_t& enc_seg, uint32_t& n_sat, uint32_t& n_nf,
+                                              bool& missing, uint32_t (&off)[4]) {
+    const uint32_t tid = threadIdx.x;
+    uint32_t len[4], any = 0;
+    uint64_t w[4];
+    pack_eight<kFromSym, kWhole, kDither>(a, sm, fa, it, k, 4u * tid, ok, n_sat, n_nf, len[0], len[1], w[0], w[1], any);
+    pack_eight<kFromSym, kWhole, kDither>(a, sm, fa, it, k, 4u * tid + kHalf, ok, n_sat, n_nf, len[2], len[3], w[2], w[3], any);
+    missing = (any & kEncMissing) != 0;
+    // One scan for the four groups, two to a word (low and high half): no sum can pass kC / 4 * 16 bits.  In the
+    // chunk all groups of a quarter come before those of the next.
+    const uint32_t x[2] = {len[0] | (len[1] << 16), len[2] | (len[3] << 16)};
+    uint32_t ex[2], tot[2];
+    pack_scan2(x, sm.scan[k & 1u], ex, tot);
+    const uint32_t t0 = tot[0] & 0xffffu, t01 = t0 + (tot[0] >> 16), t012 = t01 + (tot[1] & 0xffffu);
+    off[0] = ex[0] & 0xffffu;
+    off[1] = t0 + (ex[0] >> 16);
+    off[2] = t01 + (ex[1] & 0xffffu);
+    off[3] = t012 + (ex[1] >> 16);
     // Behind the scan's barrier every thread has finished the previous item's copy-out and this item's table
     // look-ups: clear the other bit buffer and fetch the next item's tables.
-    static_assert(kBitWords == 4 * kThreads, "one uint4 of the bit buffer per thread");
-    reinterpret_cast<uint4*>(sm.bits[(k + 1) & 1u])[tid] = make_uint4(0, 0, 0, 0);
+    uint4* clr = reinterpret_cast<uint4*>(sm.bits[(k + 1) & 1u]);
+    clr[tid] = make_uint4(0, 0, 0, 0);
+    clr[tid + kPackThreads] = make_uint4(0, 0, 0, 0);
     const FeedItem& nx = sm.feed.item[(k + 1) & 1u];
     if (nx.valid && nx.d.seg != enc_seg) {
         enc_seg = nx.d.seg;
         sm.enc[tid] = a.ws.enc_lut[enc_seg * 256 + tid];
+        sm.enc[tid + kPackThreads] = a.ws.enc_lut[enc_seg * 256 + tid + kPackThreads];
     }
     if (!kFromSym) feed_fetch_fmt(sm.feed, a.ws, (uint32_t)(k + 1) & 1u);
     if (!missing) {
         const uint32_t bits_addr = smem_addr(sm.bits[k & 1u]);
-        put_bits(bits_addr, off_a + la, wa);
-        put_bits(bits_addr, off_b + lb, wb);
+#pragma unroll
+        for (int c = 0; c < 4; ++c) put_bits(bits_addr, off[c] + len[c], w[c]);
     }
-    return (totals & 0xffffu) + (totals >> 16);
+    return t012 + (tot[1] >> 16);
 }
 
 // Thread 0 only: output locations of the item just published in ring slot `slot`.
@@ -906,7 +943,7 @@ __device__ __forceinline__ void pack_out_set(const PackArgs& a, PackSmem& sm, ui
 
 // kDither: the instance behind the dithered entry point (see convert_kernel).
 template <bool kFromSym, bool kDither>
-__global__ void __launch_bounds__(kThreads, 3) pack_kernel(PackArgs a) {
+__global__ void __launch_bounds__(kPackThreads, 5) pack_kernel(PackArgs a) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     PackSmem& sm = *reinterpret_cast<PackSmem*>(smem_raw);
     Ctrl* ctrl = a.ws.ctrl;
@@ -928,9 +965,11 @@ __global__ void __launch_bounds__(kThreads, 3) pack_kernel(PackArgs a) {
         pack_out_set(a, sm, 0, sub_off);
     }
     reinterpret_cast<uint4*>(sm.bits[0])[tid] = make_uint4(0, 0, 0, 0);
+    reinterpret_cast<uint4*>(sm.bits[0])[tid + kPackThreads] = make_uint4(0, 0, 0, 0);
     __syncthreads();
     uint32_t enc_seg = sm.feed.item[0].valid ? sm.feed.item[0].d.seg : 0u;
     sm.enc[tid] = a.ws.enc_lut[enc_seg * 256 + tid];
+    sm.enc[tid + kPackThreads] = a.ws.enc_lut[enc_seg * 256 + tid + kPackThreads];
     feed_fetch_fmt(sm.feed, a.ws, 0);
     __syncthreads();
 
@@ -950,17 +989,19 @@ __global__ void __launch_bounds__(kThreads, 3) pack_kernel(PackArgs a) {
             n_sat = n_nf = 0;
             cur_client = it.client;
         }
+        const bool ok = kFromSym || feed_wait(sm.feed, it, k, parity);
+        if (!ok) hw_fail = true;
         bool missing;
-        uint32_t off_a, off_b, total;
+        uint32_t off[4], total;
         const bool whole = kFromSym ? it.d.cnt == (uint32_t)kC : it.tma != 0;
-        if (whole) total = pack_item<kFromSym, true, kDither>(a, sm, fa, it, k, parity, enc_seg, n_sat, n_nf, hw_fail, missing, off_a, off_b);
-        else total = pack_item<kFromSym, false, kDither>(a, sm, fa, it, k, parity, enc_seg, n_sat, n_nf, hw_fail, missing, off_a, off_b);
+        if (whole) total = pack_item<kFromSym, true, kDither>(a, sm, fa, it, k, ok, enc_seg, n_sat, n_nf, missing, off);
+        else total = pack_item<kFromSym, false, kDither>(a, sm, fa, it, k, ok, enc_seg, n_sat, n_nf, missing, off);
         const PackOut out = sm.out[k & 1u];
-        // a sub-chunk of kS symbols is one warp's first or second groups
-        static_assert(kS == 4 * 32 && kSubs == 2 * (kThreads / 32), "a warp's groups of four make up one sub-chunk each");
+        // a sub-chunk of kS symbols is the groups of one warp in one quarter of the chunk
+        static_assert(kS == 4 * 32 && kSubs == 4 * kPackWarps, "a warp's groups in a quarter make up one sub-chunk");
         if ((tid & 31u) == 0) {
-            out.sub[tid >> 5] = (uint16_t)off_a;
-            out.sub[kSubs / 2 + (tid >> 5)] = (uint16_t)off_b;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) out.sub[c * kPackWarps + (tid >> 5)] = (uint16_t)off[c];
         }
         if (__syncthreads_or(missing)) {  // bit buffer complete
             if (tid == 0) {
@@ -974,13 +1015,15 @@ __global__ void __launch_bounds__(kThreads, 3) pack_kernel(PackArgs a) {
             break;
         }
         if (tid == 0) *out.chunk_bits = total;
-        // the chunk's words, four per thread; what the last of these copies carries beyond the chunk's end is zero
-        // and stays inside the slot
-        if (tid * 128u < total) reinterpret_cast<uint4*>(out.slot)[tid] = reinterpret_cast<const uint4*>(sm.bits[k & 1u])[tid];
+        // the chunk's words, 16 bytes at a time; what the last of these copies carries beyond the chunk's end is
+        // zero and stays inside the slot
+        const uint4* bits4 = reinterpret_cast<const uint4*>(sm.bits[k & 1u]);
+        if (tid * 128u < total) reinterpret_cast<uint4*>(out.slot)[tid] = bits4[tid];
+        if ((tid + kPackThreads) * 128u < total) reinterpret_cast<uint4*>(out.slot)[tid + kPackThreads] = bits4[tid + kPackThreads];
     }
     if (!kFromSym) add_counts(&a.res[cur_client], n_sat, n_nf);
     if (__syncthreads_or(hw_fail)) {  // the block stopped early, chunks of any client may be missing: the call fails
-        for (uint32_t u = tid; u < a.n_clients; u += kThreads) set_status(&a.res[u], CO3_ERR_CUDA);
+        for (uint32_t u = tid; u < a.n_clients; u += kPackThreads) set_status(&a.res[u], CO3_ERR_CUDA);
         if (tid == 0) a.ws.ctrl->abort = 1u;  // the kernels that would assemble the containers return at once
     }
 }
@@ -2459,9 +2502,9 @@ int encode_common(const float* grad, float* mem, float decay, const uint8_t* sym
         uint32_t grid = 0;
 #define CO3_PACK_CASE(S, D)                                                                                          \
     {                                                                                                                \
-        const int g = persistent_grid(pack_kernel<S, D>, kThreads, sizeof(PackSmem), items, false, &grid, &pa.group); \
+        const int g = persistent_grid(pack_kernel<S, D>, kPackThreads, sizeof(PackSmem), items, false, &grid, &pa.group); \
         if (g != CO3_OK) return g;                                                                                   \
-        CO3_LAUNCH(CO3_KERNEL_PACK, st, pack_kernel<S, D><<<grid, kThreads, sizeof(PackSmem), st>>>(pa));            \
+        CO3_LAUNCH(CO3_KERNEL_PACK, st, pack_kernel<S, D><<<grid, kPackThreads, sizeof(PackSmem), st>>>(pa));            \
     }
         if (sym) CO3_PACK_CASE(true, false)
         else if (dither) CO3_PACK_CASE(false, true)
