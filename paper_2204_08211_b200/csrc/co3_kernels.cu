@@ -84,31 +84,65 @@ __device__ __forceinline__ uint64_t block_sum_u64(uint64_t x, uint64_t* scratch 
     return sum;
 }
 
+// Block sums of three 64-bit values at once (two barriers); every thread receives them in x[].
+__device__ __forceinline__ void block_sum3_u64(uint64_t (&x)[3], uint64_t* scratch /* [3 * 8] */) {
+#pragma unroll
+    for (int q = 0; q < 3; ++q) {
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) x[q] += __shfl_xor_sync(0xffffffffu, x[q], d);
+    }
+    __syncthreads();
+    if ((threadIdx.x & 31u) == 0) {
+#pragma unroll
+        for (int q = 0; q < 3; ++q) scratch[q * 8 + (threadIdx.x >> 5)] = x[q];
+    }
+    __syncthreads();
+#pragma unroll
+    for (int q = 0; q < 3; ++q) {
+        uint64_t sum = 0;
+#pragma unroll
+        for (int w = 0; w < kThreads / 32; ++w) sum += scratch[q * 8 + w];
+        x[q] = sum;
+    }
+}
+
 __global__ void __launch_bounds__(kThreads) prepare_kernel(PrepArgs a) {
-    __shared__ uint64_t s_red[8];
+    __shared__ uint64_t s_red[3 * 8];
     __shared__ uint32_t s_kraft;
     __shared__ uint32_t s_scan[8];
     const uint32_t tid = threadIdx.x;
     const uint32_t k = blockIdx.x;
     const uint32_t G = a.tile_chunks;
 
+    // this segment's descriptors, requested before the sums below need their first round trip to memory
+    co3_seg sg{};
+    co3_fmt f{};
+    uint32_t len = 0, bits = 0;
+    if (a.n_seg) {
+        sg = a.segs[k];
+        if (a.fmts && blockIdx.y == 0) f = a.fmts[k];
+        if (a.codes && blockIdx.y == 0) {
+            len = a.codes[k].len[tid];
+            bits = a.codes[k].bits[tid];
+        }
+    }
+
     if (k == 0 && blockIdx.y == 0)
         for (uint32_t u = tid; u < a.n_res; u += kThreads) a.res[u].first_bad_chunk = 0xffffffffu;
 
     // ---- layout: elements, chunks and tiles of the segments before this one
-    uint64_t e_before = 0, c_before = 0, t_before = 0;
+    uint64_t before[3] = {0, 0, 0};  // elements, chunks, tiles
     bool bad = false;
     for (uint32_t i = tid; i < k && i < a.n_seg; i += kThreads) {
         const uint64_t n = a.segs[i].n_elem;
         if (n > a.n_elem) bad = true;
         const uint64_t c = (n + kC - 1) / kC;
-        e_before += n;
-        c_before += c;
-        t_before += (c + G - 1) / G;
+        before[0] += n;
+        before[1] += c;
+        before[2] += (c + G - 1) / G;
     }
-    e_before = block_sum_u64(e_before, s_red);
-    c_before = block_sum_u64(c_before, s_red);
-    t_before = block_sum_u64(t_before, s_red);
+    block_sum3_u64(before, s_red);
+    const uint64_t e_before = before[0], c_before = before[1], t_before = before[2];
     bad = __syncthreads_or(bad);
     if (a.n_seg == 0) {
         if (tid == 0) {
@@ -126,7 +160,6 @@ __global__ void __launch_bounds__(kThreads) prepare_kernel(PrepArgs a) {
         }
         return;
     }
-    const co3_seg sg = a.segs[k];
     const uint64_t my_chunks = sg.n_elem <= a.n_elem ? (sg.n_elem + kC - 1) / kC : 0;
     const uint64_t my_tiles = (my_chunks + G - 1) / G;
     if (sg.n_elem > a.n_elem || sg.elem_off != e_before || c_before + my_chunks > a.ws.n_chunks_max) bad = true;
@@ -194,7 +227,6 @@ __global__ void __launch_bounds__(kThreads) prepare_kernel(PrepArgs a) {
     bool fmt_ok = true;
     FmtDev fd{};
     if (a.fmts) {
-        const co3_fmt f = a.fmts[k];
         const uint32_t E = f.exp_bits, M = f.mant_bits;
         fmt_ok = E >= 2 && 1 + E + M <= 8 && (f.flags & ~CO3_FMT_FLUSH_SUBNORMALS) == 0 && f.scale > 0.0f &&
                  f.inv_scale > 0.0f && !isinf(f.scale) && !isinf(f.inv_scale);
@@ -243,8 +275,11 @@ __global__ void __launch_bounds__(kThreads) prepare_kernel(PrepArgs a) {
     bool code_ok = true;
     if (a.codes) {
         __shared__ uint32_t s_code[256];  // bits << 8 | len of every symbol
-        const uint32_t len = a.codes[k].len[tid], bits = a.codes[k].bits[tid];
+        // one bit per node of the binary code tree down to depth CO3_MAX_CODE_LEN: node (1 << len) + bits is the
+        // codeword `bits` of `len` bits, its ancestors are its proper prefixes
+        __shared__ uint32_t s_tree[(2u << CO3_MAX_CODE_LEN) / 32];
         if (tid == 0) s_kraft = 0;
+        for (uint32_t i = tid; i < (2u << CO3_MAX_CODE_LEN) / 32; i += kThreads) s_tree[i] = 0;
         __syncthreads();
         if (len > CO3_MAX_CODE_LEN || (len && (bits >> len))) code_ok = false;
         if (tid == 255 && len) code_ok = false;  // 0xff is a symbol of no format: the decoder uses it as its error mark
@@ -261,10 +296,18 @@ __global__ void __launch_bounds__(kThreads) prepare_kernel(PrepArgs a) {
         }
         __syncthreads();
         if (s_kraft > (1u << CO3_MAX_CODE_LEN)) code_ok = false;  // over-subscribed: cannot be prefix-free
-        if (code_ok && len) {  // no other codeword may start with this one (equal codewords included)
-            for (uint32_t j = 0; j < 256; ++j) {
-                const uint32_t lj = s_code[j] & 0xffu, bj = s_code[j] >> 8;
-                if (j != tid && lj >= len && (bj >> (lj - len)) == bits) code_ok = false;
+        // no codeword may start with another one (equal codewords included): every thread marks its node, then
+        // looks for a mark on the way up to the root
+        const uint32_t node = (1u << len) + bits;
+        if (code_ok && len) {
+            const uint32_t old = atomicOr(&s_tree[node >> 5], 1u << (node & 31u));
+            if (old & (1u << (node & 31u))) code_ok = false;
+        }
+        __syncthreads();
+        if (code_ok && len) {
+            for (uint32_t up = 1; up < len; ++up) {
+                const uint32_t anc = node >> up;
+                if (s_tree[anc >> 5] & (1u << (anc & 31u))) code_ok = false;
             }
         }
         code_ok = __syncthreads_and(code_ok);
@@ -1048,8 +1091,9 @@ constexpr int kScanThreads = 1024;
 static_assert(kRangeChunks == 4 * kScanThreads, "one range is one tile of four chunks per thread");
 
 // Exclusive prefix of 32-bit per-thread sums over the 1024 threads of a block (two quantities at once);
-// *tot_w / *tot_b receive the block totals.  Contains two __syncthreads().
-__device__ __forceinline__ void block_scan_1024x2(uint32_t w, uint32_t b, uint64_t* s_w, uint64_t* s_b, uint64_t& ex_w,
+// *tot_w / *tot_b receive the block totals, which must fit 32 bits (they do for up to 2^17 chunks).  Contains two
+// __syncthreads().  s_w / s_b: 32 words each.
+__device__ __forceinline__ void block_scan_1024x2(uint32_t w, uint32_t b, uint32_t* s_w, uint32_t* s_b, uint64_t& ex_w,
                                                   uint64_t& ex_b, uint64_t& tot_w, uint64_t& tot_b) {
     const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
     uint32_t iw = w, ib = b;
@@ -1061,21 +1105,23 @@ __device__ __forceinline__ void block_scan_1024x2(uint32_t w, uint32_t b, uint64
     __syncthreads();  // earlier readers of s_w / s_b are done
     if (lane == 31u) { s_w[warp] = iw; s_b[warp] = ib; }
     __syncthreads();
-    uint64_t bw = 0, bb = 0;
-    tot_w = 0;
-    tot_b = 0;
-    for (uint32_t x = 0; x < 32; ++x) {
-        if (x < warp) { bw += s_w[x]; bb += s_b[x]; }
-        tot_w += s_w[x];
-        tot_b += s_b[x];
+    // every warp scans the 32 warp totals, one per lane
+    uint32_t xw = s_w[lane], xb = s_b[lane];
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const uint32_t yw = __shfl_up_sync(0xffffffffu, xw, d), yb = __shfl_up_sync(0xffffffffu, xb, d);
+        if (lane >= (uint32_t)d) { xw += yw; xb += yb; }
     }
-    ex_w = bw + iw - w;
-    ex_b = bb + ib - b;
+    tot_w = __shfl_sync(0xffffffffu, xw, 31);
+    tot_b = __shfl_sync(0xffffffffu, xb, 31);
+    const uint32_t bw = __shfl_sync(0xffffffffu, xw, (warp + 31u) & 31u), bb = __shfl_sync(0xffffffffu, xb, (warp + 31u) & 31u);
+    ex_w = (uint64_t)((warp ? bw : 0u) + iw - w);
+    ex_b = (uint64_t)((warp ? bb : 0u) + ib - b);
 }
 
 // Two-level scan for long inputs, step 1: words and bits of each range of kRangeChunks chunks.
 __global__ void __launch_bounds__(kScanThreads) range_totals_kernel(ScanArgs a) {
-    __shared__ uint64_t s_w[32], s_b[32];
+    __shared__ uint32_t s_w[32], s_b[32];
     const Ctrl* ctrl = a.ws.ctrl;
     if (ctrl->abort) return;
     const uint32_t y = blockIdx.x, u = blockIdx.y, tid = threadIdx.x;
@@ -1123,7 +1169,7 @@ __global__ void __launch_bounds__(kScanThreads) range_scan_kernel(ScanArgs a) {
 
 // Step 3: every range scans its own chunks from its exclusive prefix and writes the chunk offsets.
 __global__ void __launch_bounds__(kScanThreads) range_apply_kernel(ScanArgs a) {
-    __shared__ uint64_t s_w[32], s_b[32];
+    __shared__ uint32_t s_w[32], s_b[32];
     const Ctrl* ctrl = a.ws.ctrl;
     if (ctrl->abort) return;
     const uint32_t y = blockIdx.x, u = blockIdx.y, tid = threadIdx.x;
@@ -1158,7 +1204,7 @@ __global__ void __launch_bounds__(kScanThreads) range_apply_kernel(ScanArgs a) {
 }
 
 __global__ void __launch_bounds__(kScanThreads) scan_kernel(ScanArgs a) {
-    __shared__ uint64_t s_w[32], s_b[32];
+    __shared__ uint32_t s_w[32], s_b[32];
     const Ctrl* ctrl = a.ws.ctrl;
     if (ctrl->abort) return;
     const uint32_t u = blockIdx.x, tid = threadIdx.x;
@@ -1168,26 +1214,28 @@ __global__ void __launch_bounds__(kScanThreads) scan_kernel(ScanArgs a) {
     uint8_t* stream = a.streams + (size_t)u * a.stream_capacity;
     uint64_t* word_off = reinterpret_cast<uint64_t*>(stream + ctrl->chunk_off);
 
-    // tiles of 4 * 1024 chunks: four consecutive chunks per thread, warp scan, one exchange through shared memory
+    // tiles of 8 * 1024 chunks: eight consecutive chunks per thread, warp scan, one exchange through shared memory
     uint64_t carry_w = 0, carry_b = 0;  // totals of the tiles already done (same in every thread)
     if (a.two_level) {  // the range kernels have written the chunk offsets already
         carry_w = a.ws.totals[2 * u];
         carry_b = a.ws.totals[2 * u + 1];
     } else {
-        for (uint32_t base = 0; base < n; base += 4 * kScanThreads) {
-            const uint32_t c0 = base + 4 * tid;
-            uint32_t b[4], w[4];
+        constexpr uint32_t kPer = 8;  // consecutive chunks per thread
+        for (uint32_t base = 0; base < n; base += kPer * kScanThreads) {
+            const uint32_t c0 = base + kPer * tid;
+            uint32_t b[kPer], w[kPer], tw8 = 0, tb8 = 0;
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
+            for (uint32_t i = 0; i < kPer; ++i) {
                 b[i] = (c0 + i < n) ? bits[c0 + i] : 0u;
                 w[i] = (b[i] + 31u) >> 5;
+                tw8 += w[i];
+                tb8 += b[i];
             }
-            const uint32_t tw4 = w[0] + w[1] + w[2] + w[3], tb4 = b[0] + b[1] + b[2] + b[3];
             uint64_t ew, eb, tile_w, tile_b;
-            block_scan_1024x2(tw4, tb4, s_w, s_b, ew, eb, tile_w, tile_b);
+            block_scan_1024x2(tw8, tb8, s_w, s_b, ew, eb, tile_w, tile_b);
             uint64_t pw = carry_w + ew, pb = carry_b + eb;  // exclusive prefix of chunk c0
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
+            for (uint32_t i = 0; i < kPer; ++i) {
                 if (c0 + i < n) {
                     word_off[c0 + i] = pw;
                     bit_prefix[c0 + i] = pb;
