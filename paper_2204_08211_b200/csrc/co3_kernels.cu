@@ -812,14 +812,7 @@ struct PackArgs {
 // ORs an n-bit value (v, right-aligned, n <= 64, bits above n clear) into the chunk's bit buffer so that its
 // last bit lands on stream bit end-1 (most significant bit first).  Words that receive only zeros are skipped.
 __device__ __forceinline__ void or_if_nonzero(uint32_t word_addr, uint32_t v) {
-    // a predicated shared-memory reduction: no branch around it; word_addr is a shared-window byte address
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.u32 p, %1, 0;\n\t"
-        "@p red.shared.or.b32 [%0], %1;\n\t}"
-        :
-        : "r"(word_addr), "r"(v)
-        : "memory");
+    asm volatile("red.shared.or.b32 [%0], %1;" : : "r"(word_addr), "r"(v) : "memory");
 }
 
 // buf_addr: shared-window byte address of the chunk's bit buffer.
@@ -874,6 +867,7 @@ struct PackSmem {
     uint32_t enc[256];
     uint32_t scan[2][2 * kPackWarps];
     PackOut out[2];
+    FeedCursor out_cur;  // the place in the item sequence of the thread that works out the output locations
 };
 
 // Eight of a packing thread's sixteen symbols (two groups of four, at q0 and q0 + kQuarter in the chunk): converted
@@ -972,16 +966,20 @@ __device__ __forceinline__ uint32_t pack_item(const PackArgs& a, PackSmem& sm, c
     return t012 + (tot[1] >> 16);
 }
 
-// Thread 0 only: output locations of the item just published in ring slot `slot`.
-__device__ __forceinline__ void pack_out_set(const PackArgs& a, PackSmem& sm, uint32_t slot, uint64_t sub_off) {
-    const FeedItem& it = sm.feed.item[slot];
+// One thread of the block's second warp only (the first warp's thread 0 feeds the ring meanwhile): output locations of
+// the next item of the sequence, for ring slot `slot`.  It walks the item sequence with a cursor of its own, in step
+// with the feeding thread's; beyond the last item the locations are never used.
+__device__ __forceinline__ void pack_out_set(const PackArgs& a, PackSmem& sm, uint32_t slot, uint64_t sub_off, uint32_t n_chunks) {
+    FeedCursor cur = sm.out_cur;
     PackOut o;
-    const size_t ci = (size_t)it.client * a.ws.n_chunks_max + it.chunk;
-    o.sub = reinterpret_cast<uint16_t*>(a.streams + (size_t)it.client * a.stream_capacity + sub_off) + (size_t)it.chunk * kSubs;
+    const size_t ci = (size_t)cur.client * a.ws.n_chunks_max + cur.chunk;
+    o.sub = reinterpret_cast<uint16_t*>(a.streams + (size_t)cur.client * a.stream_capacity + sub_off) + (size_t)cur.chunk * kSubs;
     o.slot = a.ws.slots + ci * kSlotWords;
     o.chunk_bits = a.ws.chunk_bits + ci;
-    o.res = a.res + it.client;
+    o.res = a.res + cur.client;
     sm.out[slot] = o;
+    cur.advance(n_chunks);
+    sm.out_cur = cur;
 }
 
 // kDither: the instance behind the dithered entry point (see convert_kernel).
@@ -1005,7 +1003,10 @@ __global__ void __launch_bounds__(kPackThreads, 5) pack_kernel(PackArgs a) {
         sm.feed.cur.init(n_chunks, a.group);
         next = a.ws.chunk_desc[sm.feed.cur.chunk];
         feed_issue(sm.feed, fa, a.ws, n_chunks, 0, next, !kFromSym);
-        pack_out_set(a, sm, 0, sub_off);
+    }
+    if (tid == 32) {
+        sm.out_cur.init(n_chunks, a.group);
+        pack_out_set(a, sm, 0, sub_off, n_chunks);
     }
     reinterpret_cast<uint4*>(sm.bits[0])[tid] = make_uint4(0, 0, 0, 0);
     reinterpret_cast<uint4*>(sm.bits[0])[tid + kPackThreads] = make_uint4(0, 0, 0, 0);
@@ -1021,10 +1022,8 @@ __global__ void __launch_bounds__(kPackThreads, 5) pack_kernel(PackArgs a) {
     for (uint32_t k = 0;; ++k) {
         // item k + 1 goes into the ring slot and descriptor that item k - 1 used; every thread is past the
         // last barrier of item k - 1 and read them before it
-        if (tid == 0) {
-            feed_issue(sm.feed, fa, a.ws, n_chunks, (k + 1) & 1u, next, !kFromSym);
-            pack_out_set(a, sm, (k + 1) & 1u, sub_off);
-        }
+        if (tid == 0) feed_issue(sm.feed, fa, a.ws, n_chunks, (k + 1) & 1u, next, !kFromSym);
+        if (tid == 32) pack_out_set(a, sm, (k + 1) & 1u, sub_off, n_chunks);
         const FeedItem it = sm.feed.item[k & 1u];
         if (!it.valid) break;
         if (!kFromSym && it.client != cur_client) {
