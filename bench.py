@@ -33,7 +33,7 @@ NOMINAL_HBM_GBS = 8000.0     # the peak the metric is defined against; fractions
 # dram__bytes_read.sum + dram__bytes_write.sum per element of one launch, from the ncu captures summarised under
 # profiles/ (taken on a 10-client case; traffic grows in proportion to the elements of a launch).  None: the kernel
 # has changed since its counters were taken.
-NCU_TRAFFIC_BYTES_PER_ELEMENT = {"pack": 12.501, "decode": 1.064, "convert": 12.570}   # decode: per client and element
+NCU_TRAFFIC_BYTES_PER_ELEMENT = {"pack": 12.493, "decode": 1.056, "convert": 12.572}   # decode: per client and element
 RANK_SEED_STRIDE = 100_000   # ranks draw their synthetic clients from disjoint seed ranges
 L2_BYTES = 126e6
 
