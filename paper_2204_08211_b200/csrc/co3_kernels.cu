@@ -1828,26 +1828,29 @@ __device__ __forceinline__ void merge_queues(T* node, uint16_t* parent, uint32_t
     const uint32_t lane = threadIdx.x & 31u;
     uint32_t qa = 0, qb = n, t = n;  // leaves qa..n-1 and merged nodes qb..t-1 are waiting (same in every lane)
     while (t < 2 * n - 1) {
+        // everything a step may need is requested at once: the two heads of both queues (the same addresses in every
+        // lane) and this lane's pair in either queue
+        const uint32_t ia = qa + 2 * lane, ib = qb + 2 * lane;
         const T a0 = qa < n ? node[qa] : kNone, a1 = qa + 1 < n ? node[qa + 1] : kNone;
         const T b0 = qb < t ? node[qb] : kNone, b1 = qb + 1 < t ? node[qb + 1] : kNone;
+        const T la0 = ia < n ? node[ia] : kNone, la1 = ia + 1 < n ? node[ia + 1] : kNone;
+        const T lb0 = ib < t ? node[ib] : kNone, lb1 = ib + 1 < t ? node[ib + 1] : kNone;
         uint32_t m;
         if (a1 != kNone && a1 <= b0) {
             // leaf pairs; with an empty merged queue the first pair's node becomes the head the others face
             const T head = b0 != kNone ? b0 : a0 + a1;
-            const uint32_t i0 = qa + 2 * lane;
-            m = leading_lanes(lane == 0 || (i0 + 1 < n && node[i0 + 1] <= head));
+            m = leading_lanes(lane == 0 || (la1 != kNone && la1 <= head));
             if (lane < m) {
-                node[t + lane] = node[i0] + node[i0 + 1];
-                parent[i0] = parent[i0 + 1] = (uint16_t)(t + lane);
+                node[t + lane] = la0 + la1;
+                parent[ia] = parent[ia + 1] = (uint16_t)(t + lane);
             }
             qa += 2 * m;
         } else if (b1 != kNone && b1 < a0) {
             // pairs of merged nodes that exist already (the ones created here wait behind them)
-            const uint32_t i0 = qb + 2 * lane;
-            m = leading_lanes(lane == 0 || (i0 + 1 < t && node[i0 + 1] < a0));
+            m = leading_lanes(lane == 0 || (lb1 != kNone && lb1 < a0));
             if (lane < m) {
-                node[t + lane] = node[i0] + node[i0 + 1];
-                parent[i0] = parent[i0 + 1] = (uint16_t)(t + lane);
+                node[t + lane] = lb0 + lb1;
+                parent[ib] = parent[ib + 1] = (uint16_t)(t + lane);
             }
             qb += 2 * m;
         } else {
@@ -1866,8 +1869,9 @@ __device__ __forceinline__ void merge_queues(T* node, uint16_t* parent, uint32_t
 }
 
 // One candidate tree, built by one warp: the weights after `h` halvings, max(1, w >> h) (halving h times
-// with a floor of 1 gives exactly that).  Lanes rank their symbols among the leaves, the warp merges, the lanes
-// walk from their leaves to the root.  Returns the longest codeword; len_out[sym] receives the lengths.
+// with a floor of 1 gives exactly that).  The warp puts the leaves in order (a sort of (weight, symbol) keys for
+// 32-bit weights, a count of the leaves before each symbol for wider ones), merges, and the lanes walk from their
+// leaves to the root.  Returns the longest codeword; len_out[sym] receives the lengths.
 template <typename T>
 __device__ __forceinline__ uint32_t build_tree(const uint64_t* s_w, uint32_t h, uint32_t n, T* node, uint16_t* parent,
                                                uint8_t* len_out) {
@@ -1880,27 +1884,97 @@ __device__ __forceinline__ uint32_t build_tree(const uint64_t* s_w, uint32_t h, 
         w[i] = x ? (T)max(x >> h, (uint64_t)1) : (T)0;
         rank[i] = 0;
     }
-    for (uint32_t j = 0; j < 256; ++j) {
-        const uint64_t x = s_w[j];
-        if (x == 0) continue;  // takes no part (the same for every lane)
-        const T wj = (T)max(x >> h, (uint64_t)1);
+    if (sizeof(T) == 4) {
+        // 32-bit weights: weight and symbol make one 64-bit key, and the warp sorts the 256 keys (eight per lane,
+        // element e = 8 * lane + r) with a bitonic network: exchanges inside a lane between registers, across lanes by
+        // shuffles.  A symbol that takes no part gets the largest key and ends up behind the n leaves.
+        uint64_t key[8];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) rank[i] += (wj < w[i] || (wj == w[i] && j < lane + 32 * i)) ? 1u : 0u;
+        for (int r = 0; r < 8; ++r) {
+            const uint32_t sym = 8u * lane + (uint32_t)r;
+            const uint64_t x = s_w[sym];
+            key[r] = x ? ((max(x >> h, (uint64_t)1) << 8) | sym) : ~0ull;
+        }
+#pragma unroll
+        for (int k = 2; k <= 256; k <<= 1) {
+#pragma unroll
+            for (int j = k >> 1; j > 0; j >>= 1) {
+                if (j >= 8) {
+                    const bool up = ((8u * lane) & (uint32_t)k) == 0;           // this element's run is ascending
+                    const bool keep_min = (((lane & (uint32_t)(j >> 3)) == 0) == up);  // the pair's lower place takes the minimum
+#pragma unroll
+                    for (int r = 0; r < 8; ++r) {
+                        const uint64_t other = __shfl_xor_sync(0xffffffffu, key[r], j >> 3);
+                        key[r] = keep_min ? min(key[r], other) : max(key[r], other);
+                    }
+                } else {
+#pragma unroll
+                    for (int r = 0; r < 8; ++r) {
+                        if ((r & j) == 0) {
+                            const bool up = k < 8 ? ((r & k) == 0) : (((8u * lane) & (uint32_t)k) == 0);
+                            const uint64_t lo = min(key[r], key[r ^ j]), hi = max(key[r], key[r ^ j]);
+                            key[r] = up ? lo : hi;
+                            key[r ^ j] = up ? hi : lo;
+                        }
+                    }
+                }
+            }
+        }
+        uint16_t* place = parent + 256;  // where each symbol's leaf went; free until the merge writes parents
+#pragma unroll
+        for (int r = 0; r < 8; ++r) {
+            if (key[r] != ~0ull) {
+                node[8u * lane + (uint32_t)r] = (T)(key[r] >> 8);
+                place[key[r] & 0xffu] = (uint16_t)(8u * lane + (uint32_t)r);
+            }
+        }
+        __syncwarp();
+#pragma unroll
+        for (int i = 0; i < 8; ++i) rank[i] = place[lane + 32 * i];
+    } else {
+        // wider weights: every lane counts, for each of its symbols, the leaves that come before it.  The candidate's
+        // weights lie side by side for that (behind the leaves, where merged nodes go later); a symbol that takes no
+        // part gets a weight above every other, so that it is never counted
+        T* wp = node + 256;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) wp[lane + 32 * i] = w[i] ? w[i] : ~(T)0;
+        __syncwarp();
+#pragma unroll 8
+        for (uint32_t j = 0; j < 256; ++j) {
+            const T wj = wp[j];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) rank[i] += (wj < w[i] || (wj == w[i] && j < lane + 32 * i)) ? 1u : 0u;
+        }
+        __syncwarp();  // every lane is done with wp[] before the leaves and, later, the merged nodes are written
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+            if (w[i]) node[rank[i]] = w[i];
     }
-#pragma unroll
-    for (int i = 0; i < 8; ++i)
-        if (w[i]) node[rank[i]] = w[i];
     __syncwarp();
     merge_queues<T>(node, parent, n);
-    uint32_t longest = 0;
+    // from every leaf up to the root, the lane's eight walks side by side
+    uint32_t v[8], len[8], longest = 0;
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
-        uint32_t len = 0;
-        if (w[i]) {
-            for (uint32_t v = rank[i]; v != 2 * n - 2; v = parent[v]) ++len;
+        v[i] = w[i] ? rank[i] : 2 * n - 2;
+        len[i] = 0;
+    }
+    for (;;) {
+        bool moved = false;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            if (v[i] != 2 * n - 2) {
+                v[i] = parent[v[i]];
+                ++len[i];
+                moved = true;
+            }
         }
-        len_out[lane + 32 * i] = (uint8_t)len;
-        longest = max(longest, len);
+        if (!moved) break;
+    }
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        len_out[lane + 32 * i] = (uint8_t)len[i];
+        longest = max(longest, len[i]);
     }
     return __reduce_max_sync(0xffffffffu, longest);
 }
@@ -1964,6 +2038,7 @@ __global__ void __launch_bounds__(kThreads) code_build_kernel(CodeBuildArgs a) {
     __syncthreads();
     if (valid) {
         uint32_t before = 0;
+#pragma unroll 8
         for (uint32_t j = 0; j < 256; ++j) {
             const uint32_t lj = s_len[0][j];
             if (lj != 0 && (lj < len || (lj == len && j < sym))) before += 1u << (CO3_MAX_CODE_LEN - lj);
