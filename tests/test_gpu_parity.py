@@ -155,7 +155,7 @@ def test_encode_streams_bit_identical(n_clients):
         del m_before
 
 
-@pytest.mark.parametrize("n_clients", [1, 2, 3, 4, 5, 8, 10, 16, 17, 35])
+@pytest.mark.parametrize("n_clients", [1, 2, 3, 4, 5, 8, 10, 16, 17, 20, 21, 35, 41])
 def test_decode_aggregate_matches_oracle(n_clients):
     case = _mixed_case(n_clients, sizes=(3000, 10, 64, 0, 2048, 4099, 1, 40000, 63))
     grads = _layered_grads(case, 5)
