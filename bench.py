@@ -34,6 +34,10 @@ NOMINAL_HBM_GBS = 8000.0     # the peak the metric is defined against; fractions
 # profiles/ (taken on a 10-client case; traffic grows in proportion to the elements of a launch).  None: the kernel
 # has changed since its counters were taken.
 NCU_TRAFFIC_BYTES_PER_ELEMENT = {"pack": 12.493, "decode": 1.056, "convert": 12.572}   # decode: per client and element
+# l1tex__data_pipe_lsu_wavefronts_mem_shared.sum per decoded symbol of decode_kernel, from ncu captures on small cases
+# (10 clients side by side; 32 clients in batches).  The decoder is bound by this pipe, which takes one wavefront per
+# cycle and SM: the table look-ups of a warp collide in the 32 banks.
+NCU_DECODE_SMEM_WAVEFRONTS_PER_SYMBOL = {"side_by_side": 0.2534, "batched": 0.2736}
 RANK_SEED_STRIDE = 100_000   # ranks draw their synthetic clients from disjoint seed ranges
 L2_BYTES = 126e6
 
@@ -738,6 +742,16 @@ def run_ours(args):
                 "decode_call": {k: v for k, v in row["decode_call"].items() if k != "kernels"},
                 "kernels": dict(kern, **alone),
                 "per_config": [row] + table}
+
+    if "decode" in kern and clocks.get("sm_mhz"):
+        wf = NCU_DECODE_SMEM_WAVEFRONTS_PER_SYMBOL["batched" if clients > 16 else "side_by_side"]
+        sms = torch.cuda.get_device_properties(dev).multi_processor_count
+        peak_sym = sms * clocks["sm_mhz"] * 1e6 / wf
+        got_sym = n_elem * clients / (kern["decode"]["ms_per_call"] * 1e-3)
+        roofline["decode_kernel_shared_memory_pipe"] = {
+            "bound": "shared-memory data pipe", "achieved": got_sym, "peak": peak_sym, "unit": "symbols/s",
+            "frac": got_sym / peak_sym, "wavefronts_per_symbol": wf,
+            "peak_source": "SMs x median SM clock of this run / ncu wavefronts per symbol (one wavefront per cycle and SM)"}
 
     cpu = None
     if not args.no_cpu_baseline and world == 1:
