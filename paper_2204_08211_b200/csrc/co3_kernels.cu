@@ -670,31 +670,31 @@ constexpr int kHistStride = 260;  // words between copies: shifts each copy by f
 
 // One thread's part of one work item once its inputs are in registers: conversion, new memory, symbols, counts.
 // kWhole: the chunk is complete and came through the ring (every register holds an element, 16-byte accesses).
-template <bool kSym, bool kHist, bool kMem, bool kDither, bool kWhole>
+// q0, kQ: the thread's two groups of four lie at q0 and q0 + kQ in the chunk.
+template <bool kSym, bool kHist, bool kMem, bool kDither, bool kWhole, uint32_t kQ>
 __device__ __forceinline__ void convert_item(const ConvertArgs& a, Feed& fd, const FeedItem& it, uint64_t k, const FmtDev& f,
-                                             uint32_t valid, const float (&g)[8], const float (&m)[8], uint32_t* s_hist,
-                                             uint32_t& n_sat, uint32_t& n_nf) {
-    const uint32_t q0 = threadIdx.x * 4;
+                                             uint32_t q0, uint32_t valid, const float (&g)[8], const float (&m)[8],
+                                             uint32_t* s_hist, uint32_t& n_sat, uint32_t& n_nf) {
     const uint64_t e = it.base + q0;
     const Place at{a.seed, it.client, it.d.seg, (uint64_t)it.d.cis * kC + q0};
     float mo[8];
     uint32_t s[8];
     if (kWhole) {
-        convert8<true, kDither, kHalf>(g, m, 0xffu, a.decay, f, at, mo, s, n_sat, n_nf, &fd.g[k & 1u][q0], &fd.m[k & 1u][q0]);
-        if (kMem) store_quads_vec<kHalf>(a.mem + e, mo);
+        convert8<true, kDither, kQ>(g, m, 0xffu, a.decay, f, at, mo, s, n_sat, n_nf, &fd.g[k & 1u][q0], &fd.m[k & 1u][q0]);
+        if (kMem) store_quads_vec<kQ>(a.mem + e, mo);
     } else {
-        convert8<false, kDither, kHalf>(g, m, valid, a.decay, f, at, mo, s, n_sat, n_nf);
-        if (kMem) store_quads_any<kHalf>(a.mem + e, valid, mo);
+        convert8<false, kDither, kQ>(g, m, valid, a.decay, f, at, mo, s, n_sat, n_nf);
+        if (kMem) store_quads_any<kQ>(a.mem + e, valid, mo);
     }
     if (kSym) {
         if (kWhole && (reinterpret_cast<uintptr_t>(a.sym_out + e) & 3u) == 0) {
             const uint2 w = pack_sym8(s);
             *reinterpret_cast<uint32_t*>(a.sym_out + e) = w.x;
-            *reinterpret_cast<uint32_t*>(a.sym_out + e + kHalf) = w.y;
+            *reinterpret_cast<uint32_t*>(a.sym_out + e + kQ) = w.y;
         } else {
 #pragma unroll
             for (int j = 0; j < 8; ++j)
-                if (kWhole || ((valid >> j) & 1u)) a.sym_out[e + (j & 3) + (j >> 2) * kHalf] = (uint8_t)s[j];
+                if (kWhole || ((valid >> j) & 1u)) a.sym_out[e + (j & 3) + (j >> 2) * kQ] = (uint8_t)s[j];
         }
     }
     if (kHist) {
@@ -707,8 +707,12 @@ __device__ __forceinline__ void convert_item(const ConvertArgs& a, Feed& fd, con
 
 // kMem: the new memory is stored (false: a dry pass that only counts symbols and leaves every input untouched).
 // kDither: the instance behind the dithered entry points (stochastic choice between the two levels around a value).
-template <bool kSym, bool kHist, bool kMem, bool kDither>
-__global__ void __launch_bounds__(kThreads, (kMem || kDither) ? 3 : 4) convert_kernel(ConvertArgs a) {
+// kT: threads of a block, 256 (eight elements of a chunk per thread) or 128 (sixteen, as in the packer: the dry pass,
+// whose blocks would otherwise spend much of their time at the barrier of eight warps).
+template <bool kSym, bool kHist, bool kMem, bool kDither, int kT>
+__global__ void __launch_bounds__(kT, kT == 128 ? 5 : ((kMem || kDither) ? 3 : 4)) convert_kernel(ConvertArgs a) {
+    static_assert(kT == 256 || kT == 128, "a thread owns eight or sixteen elements of a chunk");
+    constexpr uint32_t kQ = kT == 256 ? kHalf : kQuarter;  // distance between the two groups of a pair
     extern __shared__ __align__(16) unsigned char smem_raw[];
     Feed& fd = *reinterpret_cast<Feed*>(smem_raw);
     uint32_t* s_hist = reinterpret_cast<uint32_t*>(smem_raw + sizeof(Feed));
@@ -729,7 +733,7 @@ __global__ void __launch_bounds__(kThreads, (kMem || kDither) ? 3 : 4) convert_k
         feed_issue(fd, fa, a.ws, n_chunks, 0, next, true);
     }
     if (kHist)
-        for (uint32_t i = tid; i < (uint32_t)(kHistStride * kHistCopies); i += kThreads) s_hist[i] = 0;
+        for (uint32_t i = tid; i < (uint32_t)(kHistStride * kHistCopies); i += kT) s_hist[i] = 0;
     __syncthreads();
     feed_fetch_fmt(fd, a.ws, 0);
     __syncthreads();
@@ -749,24 +753,30 @@ __global__ void __launch_bounds__(kThreads, (kMem || kDither) ? 3 : 4) convert_k
         if (kHist && it.d.seg != hist_seg) {  // flush the private histograms when the segment changes
             __syncthreads();
             if (hist_seg != 0xffffffffu) {
-                uint32_t c = 0;
+                for (uint32_t b = tid; b < 256u; b += kT) {
+                    uint32_t c = 0;
 #pragma unroll
-                for (int i = 0; i < kHistCopies; ++i) { c += s_hist[tid + i * kHistStride]; s_hist[tid + i * kHistStride] = 0; }
-                if (c) atomicAdd(reinterpret_cast<unsigned long long*>(&a.hist_out[(size_t)hist_seg * 256 + tid]), (unsigned long long)c);
+                    for (int i = 0; i < kHistCopies; ++i) { c += s_hist[b + i * kHistStride]; s_hist[b + i * kHistStride] = 0; }
+                    if (c) atomicAdd(reinterpret_cast<unsigned long long*>(&a.hist_out[(size_t)hist_seg * 256 + b]), (unsigned long long)c);
+                }
             }
             hist_seg = it.d.seg;
             __syncthreads();
         }
         const FmtDev f = fd.fmt[k & 1u];
-        const uint32_t valid = it.tma ? 0xffu : quads_valid<kHalf>(it.d.cnt, q0);
         // a copy that never arrived (never expected): this thread writes nothing for the item, the block stops
         if (!feed_wait(fd, it, (uint32_t)k, parity)) {
             hw_fail = true;
         } else {
-            float g[8], m[8];
-            feed_get<kHalf>(fd, fa, it, (uint32_t)k, q0, valid, g, m);
-            if (it.tma) convert_item<kSym, kHist, kMem, kDither, true>(a, fd, it, k, f, 0xffu, g, m, s_hist, n_sat, n_nf);
-            else if (valid) convert_item<kSym, kHist, kMem, kDither, false>(a, fd, it, k, f, valid, g, m, s_hist, n_sat, n_nf);
+#pragma unroll
+            for (uint32_t part = 0; part < 256u / kT; ++part) {  // one pair of groups, or two pairs half a chunk apart
+                const uint32_t qp = q0 + part * kHalf;
+                const uint32_t valid = it.tma ? 0xffu : quads_valid<kQ>(it.d.cnt, qp);
+                float g[8], m[8];
+                feed_get<kQ>(fd, fa, it, (uint32_t)k, qp, valid, g, m);
+                if (it.tma) convert_item<kSym, kHist, kMem, kDither, true, kQ>(a, fd, it, k, f, qp, 0xffu, g, m, s_hist, n_sat, n_nf);
+                else if (valid) convert_item<kSym, kHist, kMem, kDither, false, kQ>(a, fd, it, k, f, qp, valid, g, m, s_hist, n_sat, n_nf);
+            }
         }
         feed_fetch_fmt(fd, a.ws, (uint32_t)(k + 1) & 1u);  // item k + 1 was published before the previous barrier
         __syncthreads();  // everyone has read ring slot k & 1 and item[k & 1] before thread 0 reuses them
@@ -779,14 +789,16 @@ __global__ void __launch_bounds__(kThreads, (kMem || kDither) ? 3 : 4) convert_k
     if (kHist) {
         __syncthreads();
         if (hist_seg != 0xffffffffu) {
-            uint32_t c = 0;
+            for (uint32_t b = tid; b < 256u; b += kT) {
+                uint32_t c = 0;
 #pragma unroll
-            for (int i = 0; i < kHistCopies; ++i) c += s_hist[tid + i * kHistStride];
-            if (c) atomicAdd(reinterpret_cast<unsigned long long*>(&a.hist_out[(size_t)hist_seg * 256 + tid]), (unsigned long long)c);
+                for (int i = 0; i < kHistCopies; ++i) c += s_hist[b + i * kHistStride];
+                if (c) atomicAdd(reinterpret_cast<unsigned long long*>(&a.hist_out[(size_t)hist_seg * 256 + b]), (unsigned long long)c);
+            }
         }
     }
     if (__syncthreads_or(hw_fail)) {  // the block stopped early, items of any client may be missing: the call fails
-        for (uint32_t u = tid; u < a.n_clients; u += kThreads) set_status(&a.res[u], CO3_ERR_CUDA);
+        for (uint32_t u = tid; u < a.n_clients; u += kT) set_status(&a.res[u], CO3_ERR_CUDA);
     }
 }
 
@@ -2729,9 +2741,10 @@ static int convert_common(const float* grad, float* mem, bool store_mem, float d
     uint32_t grid = 0;
 #define CO3_CONVERT_CASE2(S, H, M, D)                                                                                \
     {                                                                                                                \
-        const int g = persistent_grid(convert_kernel<S, H, M, D>, kThreads, smem, items, H, &grid, &ca.group);       \
+        constexpr int T = (!(M) && !(D)) ? 128 : kThreads; /* the dry pass runs 128-thread blocks */                 \
+        const int g = persistent_grid(convert_kernel<S, H, M, D, T>, T, smem, items, H, &grid, &ca.group);           \
         if (g != CO3_OK) return g;                                                                                   \
-        CO3_LAUNCH(CO3_KERNEL_CONVERT, st, convert_kernel<S, H, M, D><<<grid, kThreads, smem, st>>>(ca));            \
+        CO3_LAUNCH(CO3_KERNEL_CONVERT, st, convert_kernel<S, H, M, D, T><<<grid, T, smem, st>>>(ca));                \
     }
 #define CO3_CONVERT_CASE(S, H, M)                  \
     {                                              \
