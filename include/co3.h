@@ -362,7 +362,8 @@ int co3_decode(const uint8_t* stream_in, size_t stream_bytes,
 #define CO3_KERNEL_CODE_BUILD 5 /* Huffman tables from weights on the device */
 #define CO3_KERNEL_DECODE 6   /* decode + cross-client accumulate */
 #define CO3_KERNEL_FIT 7      /* moments, multiplier fit, model weights, error magnitude */
-#define CO3_KERNEL_COUNT 8
+#define CO3_KERNEL_CLEAR 8    /* zeroing of the call state, results and histogram at the start of a call */
+#define CO3_KERNEL_COUNT 9
 int co3_profile_enable(int on);
 int co3_profile_read(double* total_ms /* [host] */, uint32_t* launches /* [host] */);
 

@@ -272,7 +272,7 @@ def co3_decode(stream_in, stream_bytes, fmts, codes, segs, n_seg, n_elem, ghat_o
                               workspace.numel() * workspace.element_size(), _dev(res), _stream(stream))
 
 
-KERNEL_NAMES = ("prepare", "convert", "pack", "scan", "compact", "code_build", "decode", "fit")
+KERNEL_NAMES = ("prepare", "convert", "pack", "scan", "compact", "code_build", "decode", "fit", "clear")
 
 
 def co3_profile_enable(on: bool) -> int:

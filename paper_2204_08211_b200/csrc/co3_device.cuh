@@ -179,6 +179,11 @@ __device__ __forceinline__ float convert_fast(float g, float m, float decay, con
     return __fsub_rn(v, ghat);
 }
 
+// First statement of a kernel that is launched right behind another kernel of the same call with programmatic
+// stream serialization: its blocks may be set up while that kernel still runs, and wait here until it has completed
+// and its writes are visible.  Without that launch attribute the instruction does nothing.
+__device__ __forceinline__ void wait_for_previous_kernel() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // Philox-4x32 with 10 rounds (Salmon, Moraes, Dror, Shaw, SC 2011): a block of four 32-bit words from a counter
 // and a key.  Each round multiplies two counter words by fixed constants, crosses the halves of the products with
 // the other two words and the key, and the key advances by Weyl constants between rounds.

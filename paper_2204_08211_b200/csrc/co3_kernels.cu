@@ -11,6 +11,7 @@
 #include <stddef.h>
 
 #include <algorithm>
+#include <utility>
 #include <stdint.h>
 
 #include "co3.h"
@@ -106,7 +107,23 @@ __device__ __forceinline__ void block_sum3_u64(uint64_t (&x)[3], uint64_t* scrat
     }
 }
 
+// Zeroes up to three word ranges: the state a call starts from (control block and failure marks, results, and where a
+// call has them its histogram or completion counters), in one launch.
+struct ClearArgs {
+    uint32_t* p[3];
+    uint64_t words[3];
+};
+
+__global__ void __launch_bounds__(kThreads) clear_kernel(ClearArgs a) {
+    wait_for_previous_kernel();  // the kernels of the call before may still read what is cleared here
+    const uint64_t step = (uint64_t)gridDim.x * kThreads;
+#pragma unroll
+    for (int r = 0; r < 3; ++r)
+        for (uint64_t i = (uint64_t)blockIdx.x * kThreads + threadIdx.x; i < a.words[r]; i += step) a.p[r][i] = 0u;
+}
+
 __global__ void __launch_bounds__(kThreads) prepare_kernel(PrepArgs a) {
+    wait_for_previous_kernel();
     __shared__ uint64_t s_red[3 * 8];
     __shared__ uint32_t s_kraft;
     __shared__ uint32_t s_scan[8];
@@ -711,6 +728,7 @@ __device__ __forceinline__ void convert_item(const ConvertArgs& a, Feed& fd, con
 // whose blocks would otherwise spend much of their time at the barrier of eight warps).
 template <bool kSym, bool kHist, bool kMem, bool kDither, int kT>
 __global__ void __launch_bounds__(kT, kT == 128 ? 5 : ((kMem || kDither) ? 3 : 4)) convert_kernel(ConvertArgs a) {
+    wait_for_previous_kernel();
     static_assert(kT == 256 || kT == 128, "a thread owns eight or sixteen elements of a chunk");
     constexpr uint32_t kQ = kT == 256 ? kHalf : kQuarter;  // distance between the two groups of a pair
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -997,6 +1015,7 @@ __device__ __forceinline__ void pack_out_set(const PackArgs& a, PackSmem& sm, ui
 // kDither: the instance behind the dithered entry point (see convert_kernel).
 template <bool kFromSym, bool kDither>
 __global__ void __launch_bounds__(kPackThreads, 5) pack_kernel(PackArgs a) {
+    wait_for_previous_kernel();
     extern __shared__ __align__(16) unsigned char smem_raw[];
     PackSmem& sm = *reinterpret_cast<PackSmem*>(smem_raw);
     Ctrl* ctrl = a.ws.ctrl;
@@ -1132,6 +1151,7 @@ __device__ __forceinline__ void block_scan_1024x2(uint32_t w, uint32_t b, uint32
 
 // Two-level scan for long inputs, step 1: words and bits of each range of kRangeChunks chunks.
 __global__ void __launch_bounds__(kScanThreads) range_totals_kernel(ScanArgs a) {
+    wait_for_previous_kernel();
     __shared__ uint32_t s_w[32], s_b[32];
     const Ctrl* ctrl = a.ws.ctrl;
     if (ctrl->abort) return;
@@ -1158,6 +1178,7 @@ __global__ void __launch_bounds__(kScanThreads) range_totals_kernel(ScanArgs a) 
 
 // Step 2: one block per client turns the range totals into exclusive prefixes and the client's totals.
 __global__ void __launch_bounds__(kScanThreads) range_scan_kernel(ScanArgs a) {
+    wait_for_previous_kernel();
     const Ctrl* ctrl = a.ws.ctrl;
     if (ctrl->abort) return;
     const uint32_t u = blockIdx.x, tid = threadIdx.x;
@@ -1180,6 +1201,7 @@ __global__ void __launch_bounds__(kScanThreads) range_scan_kernel(ScanArgs a) {
 
 // Step 3: every range scans its own chunks from its exclusive prefix and writes the chunk offsets.
 __global__ void __launch_bounds__(kScanThreads) range_apply_kernel(ScanArgs a) {
+    wait_for_previous_kernel();
     __shared__ uint32_t s_w[32], s_b[32];
     const Ctrl* ctrl = a.ws.ctrl;
     if (ctrl->abort) return;
@@ -1215,6 +1237,7 @@ __global__ void __launch_bounds__(kScanThreads) range_apply_kernel(ScanArgs a) {
 }
 
 __global__ void __launch_bounds__(kScanThreads) scan_kernel(ScanArgs a) {
+    wait_for_previous_kernel();
     __shared__ uint32_t s_w[32], s_b[32];
     const Ctrl* ctrl = a.ws.ctrl;
     if (ctrl->abort) return;
@@ -1298,6 +1321,7 @@ __global__ void __launch_bounds__(kScanThreads) scan_kernel(ScanArgs a) {
 // compact: moves the chunks' words from their slots to their final positions; one warp per chunk, eight
 // chunks of one client per block, loads batched eight deep.
 __global__ void __launch_bounds__(kThreads) compact_kernel(ScanArgs a) {
+    wait_for_previous_kernel();
     const Ctrl* ctrl = a.ws.ctrl;
     if (ctrl->abort) return;
     const uint32_t u = blockIdx.y, lane = threadIdx.x & 31u;
@@ -1603,6 +1627,7 @@ __device__ __forceinline__ void write_half(const TileOut& to, uint32_t e, const 
 // word is summed by two threads (two symbols each).  kSingle: one client, nothing to sum.
 template <bool kMulti, bool kSingle>
 __global__ void __launch_bounds__(kMulti ? kMultiThreads : kThreads, kMulti ? 3 : 4) decode_kernel(DecArgs a) {
+    wait_for_previous_kernel();
     extern __shared__ __align__(16) unsigned char smem_raw[];
     DecSmem& sm = *reinterpret_cast<DecSmem*>(smem_raw);
     const uint32_t B = kSingle ? 1u : a.B, G = kMulti ? 1u : a.G;
@@ -1994,6 +2019,7 @@ __device__ __forceinline__ uint32_t build_tree(const uint64_t* s_w, uint32_t h, 
 constexpr int kCandidates = kThreads / 32;  // trees built side by side, one per warp
 
 __global__ void __launch_bounds__(kThreads) code_build_kernel(CodeBuildArgs a) {
+    wait_for_previous_kernel();
     __shared__ uint64_t s_w[256];                    // weight of every symbol, 0 = takes no part
     __shared__ uint64_t s_node[kCandidates][512];    // per candidate: the n leaves in order, then the merged nodes by age
     __shared__ uint16_t s_parent[kCandidates][512];
@@ -2535,6 +2561,23 @@ struct Profiler {
 };
 Profiler g_prof;
 
+// Launch of a kernel that follows another kernel of the same call: programmatic stream serialization lets its launch
+// overlap the tail of that kernel; the kernel itself starts with wait_for_previous_kernel().
+template <typename... Params, typename... Args>
+cudaError_t launch_behind(void (*kernel)(Params...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
+
 #define CO3_LAUNCH(id, st, ...)        \
     do {                               \
         g_prof.begin(id, st);          \
@@ -2547,15 +2590,26 @@ Profiler g_prof;
 int begin_call(const WsLayout& L, const Ws& ws, co3_result* res, uint32_t n_res, cudaStream_t st,
                const co3_fmt* fmts, const co3_code* codes, const co3_seg* segs, uint32_t n_seg, uint64_t n_elem,
                uint32_t tile_chunks, uint32_t n_fail, const uint8_t* const* streams = nullptr,
-               const uint8_t* single = nullptr, size_t stream_bytes = 0, uint32_t n_streams = 0) {
-    // the call-wide state and the per-client failure marks lie side by side in the workspace: one clearing for both
-    CO3_CUDA(cudaMemsetAsync(ws.ctrl, 0, (L.client_fail - L.ctrl) + 4 * (size_t)(n_fail ? n_fail : 1), st));
-    CO3_CUDA(cudaMemsetAsync(res, 0, sizeof(co3_result) * (size_t)n_res, st));
+               const uint8_t* single = nullptr, size_t stream_bytes = 0, uint32_t n_streams = 0,
+               void* also_clear = nullptr, size_t also_clear_bytes = 0) {
+    // one launch clears the call-wide state with the per-client failure marks (side by side in the workspace), the
+    // results, and what else the call wants zero (a multiple of four bytes)
+    static_assert(sizeof(co3_result) % 4 == 0, "results are cleared word by word");
+    ClearArgs cl{};
+    cl.p[0] = reinterpret_cast<uint32_t*>(ws.ctrl);
+    cl.words[0] = ((L.client_fail - L.ctrl) + 4 * (size_t)(n_fail ? n_fail : 1)) / 4;
+    cl.p[1] = reinterpret_cast<uint32_t*>(res);
+    cl.words[1] = sizeof(co3_result) * (size_t)n_res / 4;
+    cl.p[2] = static_cast<uint32_t*>(also_clear);
+    cl.words[2] = also_clear_bytes / 4;
+    const uint64_t clear_words = cl.words[0] + cl.words[1] + cl.words[2];
+    const uint32_t clear_blocks = (uint32_t)std::min<uint64_t>(1024, (clear_words + 4 * kThreads - 1) / (4 * kThreads));
+    CO3_LAUNCH(CO3_KERNEL_CLEAR, st, CO3_CUDA(launch_behind(clear_kernel, clear_blocks ? clear_blocks : 1u, kThreads, 0, st, cl)));
     PrepArgs pa{fmts, codes, segs, n_seg, n_elem, tile_chunks, res, n_res, n_streams ? 1u : 0u, streams, single, stream_bytes, n_streams, ws};
     // extra blocks per segment when segments are long (their chunk descriptors are written in parallel)
     const uint64_t per_seg = L.n_chunks_max / (n_seg ? n_seg : 1);
     const uint32_t helpers = (uint32_t)std::min<uint64_t>(128, per_seg / (8 * kThreads) + 1);
-    CO3_LAUNCH(CO3_KERNEL_PREPARE, st, prepare_kernel<<<dim3(n_seg ? n_seg : 1, helpers), kThreads, 0, st>>>(pa));
+    CO3_LAUNCH(CO3_KERNEL_PREPARE, st, CO3_CUDA(launch_behind(prepare_kernel, dim3(n_seg ? n_seg : 1, helpers), kThreads, 0, st, pa)));
     return CO3_OK;
 }
 
@@ -2599,13 +2653,13 @@ int decode_common(const uint8_t* const* streams, const uint8_t* single, size_t s
     const size_t smem = sizeof(DecSmem) + 4 * ((size_t)n_pairs * (kPairPhaseWords + kPaySlotWords) + kPaySlack);
     if (multi) {
         CO3_CUDA(cudaFuncSetAttribute(decode_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        CO3_LAUNCH(CO3_KERNEL_DECODE, st, decode_kernel<true, false><<<tiles, 16 * n_pairs, smem, st>>>(da));
+        CO3_LAUNCH(CO3_KERNEL_DECODE, st, CO3_CUDA(launch_behind(decode_kernel<true, false>, tiles, 16 * n_pairs, smem, st, da)));
     } else if (n_clients == 1) {
         CO3_CUDA(cudaFuncSetAttribute(decode_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        CO3_LAUNCH(CO3_KERNEL_DECODE, st, decode_kernel<false, true><<<tiles, 16 * n_pairs, smem, st>>>(da));
+        CO3_LAUNCH(CO3_KERNEL_DECODE, st, CO3_CUDA(launch_behind(decode_kernel<false, true>, tiles, 16 * n_pairs, smem, st, da)));
     } else {
         CO3_CUDA(cudaFuncSetAttribute(decode_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        CO3_LAUNCH(CO3_KERNEL_DECODE, st, decode_kernel<false, false><<<tiles, 16 * n_pairs, smem, st>>>(da));
+        CO3_LAUNCH(CO3_KERNEL_DECODE, st, CO3_CUDA(launch_behind(decode_kernel<false, false>, tiles, 16 * n_pairs, smem, st, da)));
     }
     return CO3_OK;
 }
@@ -2638,7 +2692,7 @@ int encode_common(const float* grad, float* mem, float decay, const uint8_t* sym
     {                                                                                                                \
         const int g = persistent_grid(pack_kernel<S, D>, kPackThreads, sizeof(PackSmem), items, false, &grid, &pa.group); \
         if (g != CO3_OK) return g;                                                                                   \
-        CO3_LAUNCH(CO3_KERNEL_PACK, st, pack_kernel<S, D><<<grid, kPackThreads, sizeof(PackSmem), st>>>(pa));            \
+        CO3_LAUNCH(CO3_KERNEL_PACK, st, CO3_CUDA(launch_behind(pack_kernel<S, D>, grid, kPackThreads, sizeof(PackSmem), st, pa))); \
     }
         if (sym) CO3_PACK_CASE(true, false)
         else if (dither) CO3_PACK_CASE(false, true)
@@ -2650,13 +2704,13 @@ int encode_common(const float* grad, float* mem, float decay, const uint8_t* sym
     ScanArgs sa{segs, n_seg, n_elem, streams_out, stream_capacity, res, two_level, L.n_ranges_max, ws};
     if (two_level) {
         const dim3 rgrid(L.n_ranges_max, n_clients);
-        CO3_LAUNCH(CO3_KERNEL_SCAN, st, range_totals_kernel<<<rgrid, kScanThreads, 0, st>>>(sa));
-        CO3_LAUNCH(CO3_KERNEL_SCAN, st, range_scan_kernel<<<n_clients, kScanThreads, 0, st>>>(sa));
-        CO3_LAUNCH(CO3_KERNEL_SCAN, st, range_apply_kernel<<<rgrid, kScanThreads, 0, st>>>(sa));
+        CO3_LAUNCH(CO3_KERNEL_SCAN, st, CO3_CUDA(launch_behind(range_totals_kernel, rgrid, kScanThreads, 0, st, sa)));
+        CO3_LAUNCH(CO3_KERNEL_SCAN, st, CO3_CUDA(launch_behind(range_scan_kernel, n_clients, kScanThreads, 0, st, sa)));
+        CO3_LAUNCH(CO3_KERNEL_SCAN, st, CO3_CUDA(launch_behind(range_apply_kernel, rgrid, kScanThreads, 0, st, sa)));
     }
-    CO3_LAUNCH(CO3_KERNEL_SCAN, st, scan_kernel<<<n_clients, kScanThreads, 0, st>>>(sa));
+    CO3_LAUNCH(CO3_KERNEL_SCAN, st, CO3_CUDA(launch_behind(scan_kernel, n_clients, kScanThreads, 0, st, sa)));
     if (L.n_chunks_max) {
-        CO3_LAUNCH(CO3_KERNEL_COMPACT, st, compact_kernel<<<dim3((L.n_chunks_max + kThreads / 32 - 1) / (kThreads / 32), n_clients), kThreads, 0, st>>>(sa));
+        CO3_LAUNCH(CO3_KERNEL_COMPACT, st, CO3_CUDA(launch_behind(compact_kernel, dim3((L.n_chunks_max + kThreads / 32 - 1) / (kThreads / 32), n_clients), kThreads, 0, st, sa)));
     }
     return CO3_OK;
 }
@@ -2731,8 +2785,8 @@ static int convert_common(const float* grad, float* mem, bool store_mem, float d
     if (!ws_layout(n_elem, n_seg, 0, &L)) return CO3_ERR_INVALID_ARG;
     if (workspace_bytes < L.total) return CO3_ERR_CAPACITY;
     const Ws ws = ws_pointers(workspace, L);
-    if (hist_out) CO3_CUDA(cudaMemsetAsync(hist_out, 0, 8 * 256 * (size_t)n_seg, st));
-    const int rc = begin_call(L, ws, res, n_clients, st, fmts, nullptr, segs, n_seg, n_elem, 1, 1);
+    const int rc = begin_call(L, ws, res, n_clients, st, fmts, nullptr, segs, n_seg, n_elem, 1, 1, nullptr, nullptr, 0, 0,
+                              hist_out, hist_out ? 8 * 256 * (size_t)n_seg : 0);
     if (rc != CO3_OK) return rc;
     if (L.n_chunks_max == 0) return CO3_OK;
     ConvertArgs ca{grad, mem, decay, client_stride_elems, n_clients, sym_out, hist_out, res, 1u, seed, ws};
@@ -2744,7 +2798,7 @@ static int convert_common(const float* grad, float* mem, bool store_mem, float d
         constexpr int T = (!(M) && !(D)) ? 128 : kThreads; /* the dry pass runs 128-thread blocks */                 \
         const int g = persistent_grid(convert_kernel<S, H, M, D, T>, T, smem, items, H, &grid, &ca.group);           \
         if (g != CO3_OK) return g;                                                                                   \
-        CO3_LAUNCH(CO3_KERNEL_CONVERT, st, convert_kernel<S, H, M, D, T><<<grid, T, smem, st>>>(ca));                \
+        CO3_LAUNCH(CO3_KERNEL_CONVERT, st, CO3_CUDA(launch_behind(convert_kernel<S, H, M, D, T>, grid, T, smem, st, ca))); \
     }
 #define CO3_CONVERT_CASE(S, H, M)                  \
     {                                              \
@@ -2828,9 +2882,12 @@ int co3_code_build_device(const uint64_t* weights, const co3_fmt* fmts, uint32_t
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (!weights || !fmts || !codes_out || !res || n_seg == 0 || n_seg > (1u << 20)) return CO3_ERR_INVALID_ARG;
     if (!aligned(weights, 8) || !aligned(fmts, 4) || !aligned(codes_out, 2) || !aligned(res, 8)) return CO3_ERR_INVALID_ARG;
-    CO3_CUDA(cudaMemsetAsync(res, 0, sizeof(co3_result), st));
+    ClearArgs cl{};
+    cl.p[0] = reinterpret_cast<uint32_t*>(res);
+    cl.words[0] = sizeof(co3_result) / 4;
+    CO3_LAUNCH(CO3_KERNEL_CLEAR, st, CO3_CUDA(launch_behind(clear_kernel, 1u, kThreads, 0, st, cl)));
     CodeBuildArgs ca{weights, fmts, codes_out, res};
-    CO3_LAUNCH(CO3_KERNEL_CODE_BUILD, st, code_build_kernel<<<n_seg, kThreads, 0, st>>>(ca));
+    CO3_LAUNCH(CO3_KERNEL_CODE_BUILD, st, CO3_CUDA(launch_behind(code_build_kernel, n_seg, kThreads, 0, st, ca)));
     return CO3_OK;
 }
 
