@@ -33,7 +33,7 @@ NOMINAL_HBM_GBS = 8000.0     # the peak the metric is defined against; fractions
 # dram__bytes_read.sum + dram__bytes_write.sum per element of one launch, from the ncu captures summarised under
 # profiles/ (taken on a 10-client case; traffic grows in proportion to the elements of a launch).  None: the kernel
 # has changed since its counters were taken.
-NCU_TRAFFIC_BYTES_PER_ELEMENT = {"pack": 12.493, "decode": 1.056, "convert": 12.572}   # decode: per client and element
+NCU_TRAFFIC_BYTES_PER_ELEMENT = {"pack": 12.511, "decode": 1.050, "convert": 12.579}   # decode: per client and element
 # l1tex__data_pipe_lsu_wavefronts_mem_shared.sum per decoded symbol of decode_kernel, from ncu captures on small cases
 # (10 clients side by side; 32 clients in batches).  The decoder is bound by this pipe, which takes one wavefront per
 # cycle and SM: the table look-ups of a warp collide in the 32 banks.
